@@ -1,0 +1,207 @@
+/*
+ * dam.h -- C ABI of the B200 (sm_100a) library for long-context prefill attention under
+ * Dynamic Attention Masks (DAM, arXiv 2506.11104).
+ *
+ * Two stages, one call each:
+ *
+ *   dam_build_masks       builds, for every (sequence, query head), the true mask over the
+ *                         pattern-capture window and the matched diagonal / vertical patterns,
+ *                         and writes them with a tile list into one compact mask blob
+ *                         (paper Sec. 4.2.1 - 4.2.4, Sec. 4.3 "Case 1 / Case 2");
+ *   dam_sparse_attention  computes softmax(Q K^T / sqrt(d) with masked logits = -inf) V, visiting
+ *                         only the 128 x 128 tiles the blob lists (paper Sec. 3 and Sec. 4.3, last
+ *                         paragraph).
+ *
+ * Conventions that hold for every entry point
+ *   - plain C types only; "device" pointers are CUDA global-memory pointers on the current device,
+ *     "host" pointers are ordinary host memory; `stream` is a cudaStream_t passed as void*;
+ *   - the caller owns every buffer; the library allocates no device memory, keeps no pointer after
+ *     the enqueued work retires, and enqueues all work on `stream` without synchronising it
+ *     (exceptions are stated at the function);
+ *   - every function returns a dam_status_t; argument errors are detected on the host before
+ *     anything is enqueued and nothing is written in that case;
+ *   - problems only the device can see (a tile list that would overflow the blob, a bounded wait
+ *     that expired) are recorded in the status word at the start of the mask blob / attention
+ *     scratch and are read back with dam_poll_status;
+ *   - layouts: Q, O are [total_tokens, num_q_heads, head_dim]; K, V are
+ *     [total_tokens, num_kv_heads, head_dim]; sequences are packed back to back (token-major) and
+ *     delimited by cu_seqlens[num_seqs + 1]; strides are given in elements and head_dim is
+ *     contiguous; LSE is [num_q_heads, total_tokens] float;
+ *   - query head h reads K, V of KV head h / (num_q_heads / num_kv_heads).
+ */
+#ifndef DAM_H_
+#define DAM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum dam_status_t {
+  DAM_OK = 0,
+  DAM_ERR_INVALID_ARGUMENT = 1, /* null / misaligned pointer, inconsistent shape, bad rule value   */
+  DAM_ERR_UNSUPPORTED = 2,      /* valid request this build has no kernel for                      */
+  DAM_ERR_BUFFER_TOO_SMALL = 3, /* mask blob or scratch smaller than dam_mask_sizes reports        */
+  DAM_ERR_CUDA = 4,             /* a CUDA runtime / driver call failed                             */
+  DAM_ERR_DEVICE_TIMEOUT = 5,   /* a bounded wait inside a kernel expired (kernel returned early)  */
+  DAM_ERR_INTERNAL = 6
+} dam_status_t;
+
+typedef enum dam_dtype_t { DAM_BF16 = 0, DAM_F32 = 1 } dam_dtype_t;
+
+/* Shapes of one layer's attention call. */
+typedef struct dam_shape_t {
+  uint32_t struct_size;           /* sizeof(dam_shape_t), for ABI checking                          */
+  int32_t num_seqs;               /* B >= 1                                                        */
+  const int32_t* cu_seqlens_host; /* HOST, B + 1 entries, [0] = 0, non-decreasing                   */
+  const int32_t* cu_seqlens_dev;  /* DEVICE, same values                                            */
+  int32_t total_tokens;           /* = cu_seqlens[B]                                                */
+  int32_t max_seqlen;             /* >= every sequence length                                       */
+  int32_t num_q_heads;            /* Hq                                                             */
+  int32_t num_kv_heads;           /* Hkv, Hq % Hkv == 0                                             */
+  int32_t head_dim;               /* d; multiple of 8, <= 256 (tensor-core path: bf16, d = 128)     */
+  int32_t dtype;                  /* dam_dtype_t of Q, K, V, O                                      */
+  int64_t q_stride_tok, q_stride_head; /* elements                                                  */
+  int64_t k_stride_tok, k_stride_head;
+  int64_t v_stride_tok, v_stride_head;
+  int64_t o_stride_tok, o_stride_head;
+} dam_shape_t;
+
+/* Mask-rule parameters (paper Sec. 4.2; the paper's runs use PCL 512, tau 0.3, mu 0.8,
+ * lambda 0.5, eps 1e-8). */
+typedef struct dam_rule_t {
+  uint32_t struct_size; /* sizeof(dam_rule_t)                                                      */
+  int32_t pcl_max;      /* L_max >= 1; per sequence L = min(S, L_max) (Sec. 4.2.1)                  */
+  float tau;            /* true-mask threshold on the amplified map, > 0 (Sec. 4.2.3)              */
+  float mu;             /* pattern match threshold, gamma >= mu (Sec. 4.2.4)                       */
+  float lambda;         /* Box-Cox lambda; only 0.5 is supported (Sec. 4.2.2)                      */
+  float eps;            /* clamp constant, > 0 (Sec. 4.2.2)                                        */
+  float softmax_scale;  /* 0 selects 1 / sqrt(head_dim) (Sec. 3)                                   */
+  int32_t min_support;  /* ignore patterns with fewer cells; 1 = the paper's rule                  */
+  uint32_t flags;       /* reserved, 0                                                             */
+} dam_rule_t;
+
+/* Library version (major * 1000 + minor). No arguments, no device work. */
+int32_t dam_version(void);
+
+/* Static text for a status code. Never NULL. */
+const char* dam_status_string(dam_status_t status);
+
+/*
+ * Sizes of the caller-allocated buffers for one shape.
+ *   rule != NULL : blob built by dam_build_masks / dam_build_masks_from_scores. The bound is the
+ *                  true-mask bits plus, per 128-row query block, at most 2 * ceil(L / 128) + 1 tile
+ *                  entries (a row below the window can only reach the window's columns and the
+ *                  L diagonals next to it: Sec. 4.3, Case 2).
+ *   rule == NULL : blob built by dam_mask_all_ones (`causal` selects lower-triangular or full).
+ * Outputs (HOST pointers, each may be NULL): bytes of the mask blob, of the scratch that the two
+ * build calls need, and of the scratch dam_sparse_attention needs. Host only; no device work.
+ */
+dam_status_t dam_mask_sizes(const dam_shape_t* shape, const dam_rule_t* rule, int32_t causal,
+                            size_t* mask_bytes, size_t* build_scratch_bytes,
+                            size_t* attn_scratch_bytes);
+
+/*
+ * Stage 1 (Sec. 4.2.1 - 4.2.4, 4.3). For every sequence b and query head h:
+ *   window = first L_b = min(S_b, pcl_max) tokens; P = causal softmax(Q K^T * scale) over it (fp32);
+ *   true mask  M[i][j] = [2 (sqrt(max(P, eps)) - sqrt(eps)) >= tau]   (Box-Cox with lambda = 0.5,
+ *   shifted by its minimum, which is the constant B(eps));
+ *   cntD[r] = #{i : M[i][i-r]}, cntV[c] = #{i : M[i][c]};  D[r] = [cntD[r] >= mu * (L-r)], same for
+ *   V[c], evaluated as one fp32 multiply and compare;  then every 128 x 128 tile of the S_b x S_b
+ *   mask (rows below the window follow the matched diagonals / columns) is classified and the
+ *   non-empty ones are listed.
+ * Q, K: DEVICE, layouts and strides from `shape` (V strides ignored). 16-byte aligned.
+ * mask: DEVICE, >= mask_bytes from dam_mask_sizes, 256-byte aligned; fully overwritten.
+ * scratch: DEVICE, >= build_scratch_bytes, 256-byte aligned; contents undefined afterwards.
+ * scores_dump: DEVICE or NULL. When given, receives P as fp32, for (b, h) at element offset
+ *   sum_{b' < b} Hq * L_b'^2 + h * L_b^2, row-major [L_b][L_b], zeros above the diagonal. The mask
+ *   decisions are taken on exactly these fp32 values.
+ * Errors: INVALID_ARGUMENT (null pointers, alignment, Hq % Hkv, tau <= 0, eps <= 0, pcl_max < 1,
+ *   bad cu_seqlens, struct sizes), UNSUPPORTED (lambda != 0.5, head_dim), BUFFER_TOO_SMALL, CUDA.
+ */
+dam_status_t dam_build_masks(const void* Q, const void* K, const dam_shape_t* shape,
+                             const dam_rule_t* rule, void* mask, size_t mask_capacity,
+                             void* scratch, size_t scratch_bytes, float* scores_dump,
+                             void* stream);
+
+/*
+ * Stage 1 without the scoring pass: the rule of Sec. 4.2.2 - 4.3 applied to a caller-supplied fp32
+ * map P (DEVICE, same layout as scores_dump above; need not be a softmax). Used to compare masks
+ * bit for bit from one shared score tensor. Other arguments and errors as dam_build_masks.
+ */
+dam_status_t dam_build_masks_from_scores(const float* P, const dam_shape_t* shape,
+                                         const dam_rule_t* rule, void* mask, size_t mask_capacity,
+                                         void* scratch, size_t scratch_bytes, void* stream);
+
+/*
+ * A mask blob that lists every tile (lower-triangular tiles when causal != 0, all tiles otherwise)
+ * as fully active: dam_sparse_attention on it is dense attention. Serves as the dense baseline
+ * and as a test of the attention kernel alone. The paper has no counterpart (its masks are never
+ * all-ones); Sec. 3 defines the dense attention this reproduces.
+ * mask: DEVICE, >= mask_bytes from dam_mask_sizes(shape, NULL, causal, ...), 256-byte aligned.
+ */
+dam_status_t dam_mask_all_ones(const dam_shape_t* shape, int32_t causal, void* mask,
+                               size_t mask_capacity, void* stream);
+
+/*
+ * Stage 2 (Sec. 3; Sec. 4.3 last paragraph): O = softmax(S') V with S' = Q K^T * scale and
+ * S'[i][j] = -inf where the mask is 0 (and where j > i when causal != 0); LSE[h][t] = natural-log
+ * sum-exp of row t's active logits. A row with no active key gives O = 0, LSE = -inf.
+ * Q, K, V: DEVICE (16-byte aligned); mask: DEVICE blob from a build call or dam_mask_all_ones for the
+ * same shape; O: DEVICE, written for every token and head; lse: DEVICE float [Hq][total_tokens].
+ * gqa_group must equal num_q_heads / num_kv_heads; softmax_scale 0 selects 1 / sqrt(head_dim).
+ * scratch: DEVICE, >= attn_scratch_bytes, 256-byte aligned; it begins with a status word.
+ * Tensor-core path (tcgen05 + TMA): dtype bf16, head_dim 128, 16-byte aligned strides; other
+ * shapes run a plain CUDA-core kernel.
+ * Errors: INVALID_ARGUMENT, UNSUPPORTED, BUFFER_TOO_SMALL, CUDA; DEVICE_TIMEOUT via the status word.
+ */
+dam_status_t dam_sparse_attention(const void* Q, const void* K, const void* V, const void* mask,
+                                  const dam_shape_t* shape, int32_t causal, int32_t gqa_group,
+                                  float softmax_scale, void* O, float* lse, void* scratch,
+                                  size_t scratch_bytes, void* stream);
+
+/*
+ * Counts taken from a mask blob (DEVICE): out[0] = listed tiles, out[1] = tiles listed as fully
+ * active, out[2] = total causal tiles of the shape (for densities), out[3] = bytes of the blob in
+ * use. `out` is HOST memory (4 x uint64). Synchronises `stream`. The paper reports no such counts;
+ * they feed the density and active-FLOP figures of the benchmark.
+ */
+dam_status_t dam_mask_stats(const void* mask, const dam_shape_t* shape, uint64_t* out,
+                            void* stream);
+
+/*
+ * Test hook: expands rows [row_begin, row_begin + nrows) of (seq, head) of the S x S mask exactly as
+ * the attention kernels see it (tile list -> tile kind -> per-row 128-bit words, then the causal
+ * and sequence-end limits when causal != 0) into out_bits (DEVICE, uint32
+ * [nrows][ceil(S / 128) * 4], bit j % 32 of word j / 32 = key j). Lets a test compare the blob with
+ * the paper's Case 1 / Case 2 definition (Sec. 4.3) cell by cell.
+ */
+dam_status_t dam_mask_expand_rows(const void* mask, const dam_shape_t* shape, int32_t seq,
+                                  int32_t head, int32_t row_begin, int32_t nrows, int32_t causal,
+                                  uint32_t* out_bits, void* stream);
+
+/*
+ * Reads the status word at the start of a mask blob or of an attention scratch buffer (DEVICE).
+ * Synchronises `stream`, then returns DAM_OK or the recorded device-side status.
+ */
+dam_status_t dam_poll_status(const void* mask_or_scratch, void* stream);
+
+/*
+ * Both stages from HOST buffers: copies Q, K, V (HOST, pinned recommended, layouts from `shape`
+ * with dense strides) into the device workspace, runs dam_build_masks and dam_sparse_attention,
+ * and copies O and LSE back to HOST; everything on `stream`, which is synchronised before
+ * returning. workspace: DEVICE, >= *workspace_bytes as returned when called with workspace == NULL
+ * (in that case only the size is computed). The end-to-end figure of the benchmark is measured
+ * through this call.
+ */
+dam_status_t dam_prefill_host(const void* Q_host, const void* K_host, const void* V_host,
+                              const dam_shape_t* shape, const dam_rule_t* rule, int32_t causal,
+                              void* O_host, float* lse_host, void* workspace,
+                              size_t* workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DAM_H_ */

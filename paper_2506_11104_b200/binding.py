@@ -1,0 +1,296 @@
+"""Thin ctypes binding of the C ABI in ``include/dam.h``.
+
+Argument marshalling only: every step of the path runs inside the CUDA library.  PyTorch is used for
+device memory and streams.  There is no CPU fallback: if ``libdam_b200.so`` is missing or a call
+fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import List, Optional, Sequence
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdam_b200.so")
+
+DAM_BF16, DAM_F32 = 0, 1
+STATUS = {0: "DAM_OK", 1: "DAM_ERR_INVALID_ARGUMENT", 2: "DAM_ERR_UNSUPPORTED", 3: "DAM_ERR_BUFFER_TOO_SMALL",
+          4: "DAM_ERR_CUDA", 5: "DAM_ERR_DEVICE_TIMEOUT", 6: "DAM_ERR_INTERNAL"}
+
+EXPORTS = ["dam_version", "dam_status_string", "dam_mask_sizes", "dam_build_masks", "dam_build_masks_from_scores",
+           "dam_mask_all_ones", "dam_sparse_attention", "dam_mask_stats", "dam_mask_expand_rows", "dam_poll_status",
+           "dam_prefill_host"]
+
+
+class DamError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {STATUS.get(code, code)}")
+
+
+class dam_shape_t(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_uint32), ("num_seqs", ctypes.c_int32),
+                ("cu_seqlens_host", ctypes.c_void_p), ("cu_seqlens_dev", ctypes.c_void_p),
+                ("total_tokens", ctypes.c_int32), ("max_seqlen", ctypes.c_int32),
+                ("num_q_heads", ctypes.c_int32), ("num_kv_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("dtype", ctypes.c_int32),
+                ("q_stride_tok", ctypes.c_int64), ("q_stride_head", ctypes.c_int64),
+                ("k_stride_tok", ctypes.c_int64), ("k_stride_head", ctypes.c_int64),
+                ("v_stride_tok", ctypes.c_int64), ("v_stride_head", ctypes.c_int64),
+                ("o_stride_tok", ctypes.c_int64), ("o_stride_head", ctypes.c_int64)]
+
+
+class dam_rule_t(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_uint32), ("pcl_max", ctypes.c_int32), ("tau", ctypes.c_float),
+                ("mu", ctypes.c_float), ("lambda_", ctypes.c_float), ("eps", ctypes.c_float),
+                ("softmax_scale", ctypes.c_float), ("min_support", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+
+
+_lib = None
+
+
+def lib():
+    """The loaded shared library; raises if it was not built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2506_11104_b200.build` "
+                               "(there is no fallback path)")
+        _lib = ctypes.CDLL(LIB_PATH)
+        _lib.dam_version.restype = ctypes.c_int32
+        _lib.dam_status_string.restype = ctypes.c_char_p
+        _lib.dam_status_string.argtypes = [ctypes.c_int]
+        for name in EXPORTS[2:]:
+            getattr(_lib, name).restype = ctypes.c_int
+    return _lib
+
+
+def _check(code: int, where: str):
+    if code != 0:
+        raise DamError(code, where)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return ctypes.c_void_p(0 if t is None else t.data_ptr())
+
+
+def _stream(device) -> ctypes.c_void_p:
+    return ctypes.c_void_p(torch.cuda.current_stream(device).cuda_stream)
+
+
+@dataclass
+class Shape:
+    """Python-side owner of a dam_shape_t and the cu_seqlens buffers it points to."""
+    c: dam_shape_t
+    cu_host: np.ndarray
+    cu_dev: Optional[torch.Tensor]
+    lengths: List[int]
+
+    @property
+    def ref(self):
+        return ctypes.byref(self.c)
+
+
+def make_shape(cu_seqlens: Sequence[int], Hq: int, Hkv: int, d: int, dtype: torch.dtype, device=None,
+               q_strides=None, k_strides=None, v_strides=None, o_strides=None) -> Shape:
+    cu_host = np.ascontiguousarray(cu_seqlens, dtype=np.int32)
+    cu_dev = torch.from_numpy(cu_host.copy()).to(device) if device is not None else None
+    lengths = [int(b - a) for a, b in zip(cu_host[:-1], cu_host[1:])]
+    s = dam_shape_t()
+    s.struct_size = ctypes.sizeof(dam_shape_t)
+    s.num_seqs = len(lengths)
+    s.cu_seqlens_host = cu_host.ctypes.data
+    s.cu_seqlens_dev = cu_dev.data_ptr() if cu_dev is not None else 1   # non-null placeholder for host-only calls
+    s.total_tokens = int(cu_host[-1])
+    s.max_seqlen = max(lengths) if lengths else 0
+    s.num_q_heads, s.num_kv_heads, s.head_dim = Hq, Hkv, d
+    s.dtype = DAM_BF16 if dtype == torch.bfloat16 else DAM_F32
+    qs = q_strides or (Hq * d, d)
+    ks = k_strides or (Hkv * d, d)
+    vs = v_strides or (Hkv * d, d)
+    os_ = o_strides or (Hq * d, d)
+    s.q_stride_tok, s.q_stride_head = qs
+    s.k_stride_tok, s.k_stride_head = ks
+    s.v_stride_tok, s.v_stride_head = vs
+    s.o_stride_tok, s.o_stride_head = os_
+    return Shape(c=s, cu_host=cu_host, cu_dev=cu_dev, lengths=lengths)
+
+
+def make_rule(pcl_max: int, tau: float, mu: float, lam: float = 0.5, eps: float = 1e-8,
+              softmax_scale: float = 0.0, min_support: int = 1) -> dam_rule_t:
+    r = dam_rule_t()
+    r.struct_size = ctypes.sizeof(dam_rule_t)
+    r.pcl_max, r.tau, r.mu, r.lambda_, r.eps = pcl_max, tau, mu, lam, eps
+    r.softmax_scale, r.min_support, r.flags = softmax_scale, min_support, 0
+    return r
+
+
+def dam_version() -> int:
+    return int(lib().dam_version())
+
+
+def dam_status_string(code: int) -> str:
+    return lib().dam_status_string(code).decode()
+
+
+def dam_mask_sizes(shape: Shape, rule: Optional[dam_rule_t], causal: bool = True):
+    m, b, a = ctypes.c_size_t(0), ctypes.c_size_t(0), ctypes.c_size_t(0)
+    rc = lib().dam_mask_sizes(shape.ref, ctypes.byref(rule) if rule is not None else None, int(causal),
+                              ctypes.byref(m), ctypes.byref(b), ctypes.byref(a))
+    _check(rc, "dam_mask_sizes")
+    return m.value, b.value, a.value
+
+
+def _alloc(nbytes: int, device) -> torch.Tensor:
+    return torch.empty(max(256, nbytes), dtype=torch.uint8, device=device)
+
+
+def dam_build_masks(Q: torch.Tensor, K: torch.Tensor, shape: Shape, rule: dam_rule_t, mask: Optional[torch.Tensor] = None,
+                    scratch: Optional[torch.Tensor] = None, scores_dump: Optional[torch.Tensor] = None):
+    """Enqueues stage 1 on the current stream.  Returns (mask blob, scratch)."""
+    if mask is None or scratch is None:
+        mb, sb, _ = dam_mask_sizes(shape, rule)
+        mask = mask if mask is not None else _alloc(mb, Q.device)
+        scratch = scratch if scratch is not None else _alloc(sb, Q.device)
+    rc = lib().dam_build_masks(_ptr(Q), _ptr(K), shape.ref, ctypes.byref(rule), _ptr(mask),
+                               ctypes.c_size_t(mask.numel()), _ptr(scratch), ctypes.c_size_t(scratch.numel()),
+                               _ptr(scores_dump), _stream(Q.device))
+    _check(rc, "dam_build_masks")
+    return mask, scratch
+
+
+def dam_build_masks_from_scores(P: torch.Tensor, shape: Shape, rule: dam_rule_t, mask: Optional[torch.Tensor] = None,
+                                scratch: Optional[torch.Tensor] = None):
+    if mask is None or scratch is None:
+        mb, sb, _ = dam_mask_sizes(shape, rule)
+        mask = mask if mask is not None else _alloc(mb, P.device)
+        scratch = scratch if scratch is not None else _alloc(sb, P.device)
+    rc = lib().dam_build_masks_from_scores(_ptr(P), shape.ref, ctypes.byref(rule), _ptr(mask),
+                                           ctypes.c_size_t(mask.numel()), _ptr(scratch),
+                                           ctypes.c_size_t(scratch.numel()), _stream(P.device))
+    _check(rc, "dam_build_masks_from_scores")
+    return mask, scratch
+
+
+def dam_mask_all_ones(shape: Shape, causal: bool, device, mask: Optional[torch.Tensor] = None) -> torch.Tensor:
+    if mask is None:
+        mb, _, _ = dam_mask_sizes(shape, None, causal)
+        mask = _alloc(mb, device)
+    rc = lib().dam_mask_all_ones(shape.ref, int(causal), _ptr(mask), ctypes.c_size_t(mask.numel()), _stream(device))
+    _check(rc, "dam_mask_all_ones")
+    return mask
+
+
+def dam_sparse_attention(Q, K, V, mask, shape: Shape, causal: bool = True, softmax_scale: float = 0.0,
+                         O: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
+                         scratch: Optional[torch.Tensor] = None):
+    """Enqueues stage 2 on the current stream.  Returns (O, LSE [Hq, T] fp32, scratch)."""
+    if O is None:
+        O = torch.empty_like(Q)
+    if lse is None:
+        lse = torch.empty(shape.c.num_q_heads, shape.c.total_tokens, dtype=torch.float32, device=Q.device)
+    if scratch is None:
+        scratch = _alloc(256, Q.device)
+    rc = lib().dam_sparse_attention(_ptr(Q), _ptr(K), _ptr(V), _ptr(mask), shape.ref, int(causal),
+                                    shape.c.num_q_heads // shape.c.num_kv_heads, ctypes.c_float(softmax_scale),
+                                    _ptr(O), _ptr(lse), _ptr(scratch), ctypes.c_size_t(scratch.numel()),
+                                    _stream(Q.device))
+    _check(rc, "dam_sparse_attention")
+    return O, lse, scratch
+
+
+def dam_mask_stats(mask: torch.Tensor, shape: Shape) -> dict:
+    out = (ctypes.c_uint64 * 4)()
+    rc = lib().dam_mask_stats(_ptr(mask), shape.ref, out, _stream(mask.device))
+    _check(rc, "dam_mask_stats")
+    return {"tiles": int(out[0]), "full_tiles": int(out[1]), "causal_tiles": int(out[2]), "bytes_used": int(out[3])}
+
+
+def dam_mask_expand_rows(mask: torch.Tensor, shape: Shape, seq: int, head: int, row_begin: int, nrows: int,
+                         causal: bool = True) -> torch.Tensor:
+    S = shape.lengths[seq]
+    words = ((S + 127) // 128) * 4
+    out = torch.empty(nrows, words, dtype=torch.int32, device=mask.device)
+    rc = lib().dam_mask_expand_rows(_ptr(mask), shape.ref, seq, head, row_begin, nrows, int(causal), _ptr(out),
+                                    _stream(mask.device))
+    _check(rc, "dam_mask_expand_rows")
+    return out
+
+
+def dam_poll_status(buf: torch.Tensor) -> int:
+    return int(lib().dam_poll_status(_ptr(buf), _stream(buf.device)))
+
+
+def dam_prefill_host(Qh: torch.Tensor, Kh: torch.Tensor, Vh: torch.Tensor, shape: Shape, rule: dam_rule_t,
+                     Oh: torch.Tensor, lse_h: torch.Tensor, workspace: Optional[torch.Tensor], device,
+                     causal: bool = True):
+    """Host buffers in, host buffers out (copies inside the call).  workspace=None returns the size."""
+    n = ctypes.c_size_t(0 if workspace is None else workspace.numel())
+    rc = lib().dam_prefill_host(_ptr(Qh), _ptr(Kh), _ptr(Vh), shape.ref, ctypes.byref(rule), int(causal),
+                                _ptr(Oh), _ptr(lse_h), _ptr(workspace), ctypes.byref(n), _stream(device))
+    _check(rc, "dam_prefill_host")
+    return n.value
+
+
+# ----------------------------------------------------------------------------------------------
+# Blob reader (host side, for tests and statistics): unpacks the sections of a mask blob.
+# ----------------------------------------------------------------------------------------------
+_HDR = np.dtype([("magic", "<u4"), ("status", "<u4"), ("version", "<u4"), ("flags", "<u4"),
+                 ("num_seqs", "<i4"), ("num_q_heads", "<i4"), ("total_qblocks", "<i4"), ("rows", "<i4"),
+                 ("tile_capacity", "<u4"), ("total_tiles", "<u4"), ("full_tiles", "<u4"), ("pcl_max", "<u4"),
+                 ("off_seq", "<u8"), ("off_qbseq", "<u8"), ("off_dv", "<u8"), ("off_true", "<u8"),
+                 ("off_tile_ptr", "<u8"), ("off_work", "<u8"), ("off_tiles", "<u8"), ("bytes_used", "<u8"),
+                 ("causal_tiles", "<u8"), ("reserved", "<u8", (17,))])
+_SEQ = np.dtype([("tok_start", "<i4"), ("S", "<i4"), ("L", "<i4"), ("nq", "<i4"), ("first_qblock", "<i4"),
+                 ("W", "<i4"), ("nL", "<i4"), ("pad", "<i4"), ("dv_off", "<u8"), ("true_off", "<u8"),
+                 ("p_off", "<u8"), ("cnt_off", "<u8")])
+
+
+def _unpack_bits(words: np.ndarray, n: int) -> np.ndarray:
+    """uint32 words [..., W] -> uint8 bits [..., n] (bit j % 32 of word j / 32)."""
+    b = np.unpackbits(words.astype("<u4").view(np.uint8), axis=-1, bitorder="little")
+    return b[..., :n]
+
+
+class MaskBlob:
+    """Host copy of a mask blob with accessors for its sections."""
+
+    def __init__(self, blob: torch.Tensor):
+        hdr_bytes = blob[:256].cpu().numpy()
+        self.hdr = np.frombuffer(hdr_bytes.tobytes(), dtype=_HDR)[0]
+        assert self.hdr["magic"] == 0x4B4D4144, "not a DAM mask blob"
+        used = int(max(self.hdr["bytes_used"], self.hdr["off_tiles"]))
+        self.raw = blob[:used].cpu().numpy().tobytes()
+        B = int(self.hdr["num_seqs"])
+        self.seqs = np.frombuffer(self.raw, dtype=_SEQ, count=B, offset=int(self.hdr["off_seq"]))
+        rows = int(self.hdr["rows"])
+        self.tile_ptr = np.frombuffer(self.raw, dtype="<u4", count=rows + 1, offset=int(self.hdr["off_tile_ptr"]))
+        self.work = np.frombuffer(self.raw, dtype="<u4", count=rows, offset=int(self.hdr["off_work"]))
+        self.tiles = np.frombuffer(self.raw, dtype="<u4", count=int(self.hdr["total_tiles"]),
+                                   offset=int(self.hdr["off_tiles"]))
+
+    def pattern_bits(self, seq: int, head: int):
+        """(D, Drev, V) as uint8 [L]."""
+        s = self.seqs[seq]
+        L, W = int(s["L"]), int(s["W"])
+        off = int(self.hdr["off_dv"]) + 4 * (int(s["dv_off"]) + head * 3 * W)
+        w = np.frombuffer(self.raw, dtype="<u4", count=3 * W, offset=off).reshape(3, W)
+        bits = _unpack_bits(w, L)
+        return bits[0], bits[1], bits[2]
+
+    def true_mask(self, seq: int, head: int) -> np.ndarray:
+        s = self.seqs[seq]
+        L, W = int(s["L"]), int(s["W"])
+        off = int(self.hdr["off_true"]) + 4 * (int(s["true_off"]) + head * L * W)
+        w = np.frombuffer(self.raw, dtype="<u4", count=L * W, offset=off).reshape(L, W)
+        return _unpack_bits(w, L)
+
+    def row_tiles(self, seq: int, head: int, qb: int):
+        """(kv tile indices, kinds) of query block qb of (seq, head)."""
+        row = head * int(self.hdr["total_qblocks"]) + int(self.seqs[seq]["first_qblock"]) + qb
+        e = self.tiles[self.tile_ptr[row]: self.tile_ptr[row + 1]]
+        return (e & 0x0FFFFFFF).astype(np.int64), (e >> 28).astype(np.int64)

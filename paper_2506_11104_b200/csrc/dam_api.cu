@@ -1,0 +1,363 @@
+// Host side of the C ABI declared in include/dam.h: argument validation, buffer layout, the
+// single-compare form of the threshold, and kernel dispatch.  No device memory is allocated here.
+#include <math.h>
+#include <string.h>
+
+#include <vector>
+
+#include "dam_internal.cuh"
+
+namespace {
+
+struct Layout {
+  DamHeader hdr;
+  size_t mask_bytes;
+  size_t build_scratch_bytes;
+  size_t attn_scratch_bytes;
+  uint64_t off_cnt, off_rowstat, off_rowcnt, off_hist, off_cursor;
+  int max_L, max_W, max_nL, max_nq;
+  uint64_t score_elems;
+};
+
+dam_status_t check_shape(const dam_shape_t* s) {
+  if (!s || s->struct_size != sizeof(dam_shape_t)) return DAM_ERR_INVALID_ARGUMENT;
+  if (s->num_seqs < 1 || !s->cu_seqlens_host || !s->cu_seqlens_dev) return DAM_ERR_INVALID_ARGUMENT;
+  if (s->cu_seqlens_host[0] != 0) return DAM_ERR_INVALID_ARGUMENT;
+  for (int b = 0; b < s->num_seqs; ++b) {
+    int len = s->cu_seqlens_host[b + 1] - s->cu_seqlens_host[b];
+    if (len < 0 || len > s->max_seqlen) return DAM_ERR_INVALID_ARGUMENT;
+  }
+  if (s->cu_seqlens_host[s->num_seqs] != s->total_tokens) return DAM_ERR_INVALID_ARGUMENT;
+  if (s->num_q_heads < 1 || s->num_kv_heads < 1 || s->num_q_heads % s->num_kv_heads) return DAM_ERR_INVALID_ARGUMENT;
+  if (s->dtype != DAM_BF16 && s->dtype != DAM_F32) return DAM_ERR_INVALID_ARGUMENT;
+  if (s->head_dim < 8 || s->head_dim % 8) return DAM_ERR_INVALID_ARGUMENT;
+  if (s->head_dim > 256) return DAM_ERR_UNSUPPORTED;
+  const int64_t st[8] = {s->q_stride_tok, s->q_stride_head, s->k_stride_tok, s->k_stride_head,
+                         s->v_stride_tok, s->v_stride_head, s->o_stride_tok, s->o_stride_head};
+  const int64_t vec = s->dtype == DAM_BF16 ? 8 : 4;   // 16-byte vectors
+  for (int i = 0; i < 8; ++i)
+    if (st[i] < s->head_dim || st[i] % vec) return DAM_ERR_INVALID_ARGUMENT;
+  return DAM_OK;
+}
+
+dam_status_t check_rule(const dam_rule_t* r) {
+  if (!r || r->struct_size != sizeof(dam_rule_t)) return DAM_ERR_INVALID_ARGUMENT;
+  if (r->pcl_max < 1) return DAM_ERR_INVALID_ARGUMENT;
+  if (!(r->tau > 0.f) || !(r->eps > 0.f) || !(r->mu == r->mu)) return DAM_ERR_INVALID_ARGUMENT;
+  if (r->min_support < 1 || r->flags != 0 || r->softmax_scale < 0.f) return DAM_ERR_INVALID_ARGUMENT;
+  if (r->lambda != 0.5f) return DAM_ERR_UNSUPPORTED;
+  return DAM_OK;
+}
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// Layout of the blob and of the scratch buffers, from the host copy of cu_seqlens.
+// pcl_max == 0 selects the all-ones blob (no window sections).
+void compute_layout(const dam_shape_t* s, int pcl_max, int all_ones_causal, Layout* out) {
+  Layout& y = *out;
+  memset(&y, 0, sizeof(y));
+  const int Hq = s->num_q_heads;
+  uint64_t dv = 0, tr = 0, cnt = 0, cap = 0, causal_tiles = 0, lrows = 0, po = 0;
+  int total_qb = 0;
+  for (int b = 0; b < s->num_seqs; ++b) {
+    int S = s->cu_seqlens_host[b + 1] - s->cu_seqlens_host[b];
+    int L = S < pcl_max ? S : pcl_max;
+    int W = L > 0 ? dam_words(L) : 0;
+    int nL = (L + DAM_TILE - 1) / DAM_TILE;
+    int nq = (S + DAM_TILE - 1) / DAM_TILE;
+    dv += (uint64_t)Hq * 3 * W;
+    tr += (uint64_t)Hq * L * W;
+    po += (uint64_t)Hq * L * L;
+    cnt += (uint64_t)Hq * dam_cnt_stride(L, W, nL);
+    lrows += (uint64_t)Hq * L;
+    causal_tiles += (uint64_t)Hq * nq * (nq + 1) / 2;
+    if (pcl_max > 0) {
+      for (int qb = 0; qb < nq; ++qb) cap += (uint64_t)Hq * dam_row_tile_bound(qb, nL);
+    } else {
+      cap += (uint64_t)Hq * (all_ones_causal ? (uint64_t)nq * (nq + 1) / 2 : (uint64_t)nq * nq);
+    }
+    total_qb += nq;
+    if (L > y.max_L) y.max_L = L;
+    if (W > y.max_W) y.max_W = W;
+    if (nL > y.max_nL) y.max_nL = nL;
+    if (nq > y.max_nq) y.max_nq = nq;
+  }
+  DamHeader& h = y.hdr;
+  h.magic = DAM_MAGIC;
+  h.status = 0;
+  h.version = 1;
+  h.flags = pcl_max > 0 ? DAM_FLAG_CAUSAL_LIST : (DAM_FLAG_ALL_ONES | (all_ones_causal ? DAM_FLAG_CAUSAL_LIST : 0u));
+  h.num_seqs = s->num_seqs;
+  h.num_q_heads = Hq;
+  h.total_qblocks = total_qb;
+  h.rows = Hq * total_qb;
+  h.tile_capacity = (uint32_t)(cap > 0xFFFFFFF0ull ? 0xFFFFFFF0ull : cap);
+  h.pcl_max = (uint32_t)pcl_max;
+  h.off_seq = sizeof(DamHeader);
+  h.off_qbseq = dam_align(h.off_seq + (uint64_t)s->num_seqs * sizeof(DamSeq), 256);
+  h.off_dv = dam_align(h.off_qbseq + 4ull * total_qb, 256);
+  h.off_true = dam_align(h.off_dv + 4ull * dv, 256);
+  h.off_tile_ptr = dam_align(h.off_true + 4ull * tr, 256);
+  h.off_work = dam_align(h.off_tile_ptr + 4ull * (h.rows + 1), 256);
+  h.off_tiles = dam_align(h.off_work + 4ull * h.rows, 256);
+  h.causal_tiles = causal_tiles;
+  y.mask_bytes = dam_align(h.off_tiles + 4ull * cap, 256);
+  // build scratch: [0,256) reserved | counts | row stats (2 floats per window row) | row counts | hist | cursor
+  y.off_cnt = 256;
+  y.off_rowstat = dam_align(y.off_cnt + 4ull * cnt, 256);
+  y.off_rowcnt = dam_align(y.off_rowstat + 8ull * lrows, 256);
+  y.off_hist = dam_align(y.off_rowcnt + 4ull * h.rows, 256);
+  y.off_cursor = y.off_hist + 4ull * DAM_HIST;
+  y.build_scratch_bytes = dam_align(y.off_cursor + 4ull * DAM_HIST, 256);
+  y.attn_scratch_bytes = 256;
+  y.score_elems = po;
+}
+
+// The threshold chain of the true mask (Sec. 4.2.2 - 4.2.3 with lambda = 0.5), each step one IEEE
+// single-precision operation:  x = max(p, eps); b = (sqrt(x) - 1) * 2; a = b - (sqrt(eps) - 1) * 2;
+// active = a >= tau.  Every step is monotone in p, so the active set is {p >= p*}; p* is found by
+// bisection over the float bit patterns in [0, 1] and the kernels use the single compare.
+bool chain_active(float p, float tau, float eps) {
+  volatile float x = p > eps ? p : eps;
+  volatile float r = sqrtf(x);
+  volatile float b = (r - 1.0f) * 2.0f;
+  volatile float se = sqrtf(eps);
+  volatile float bmin = (se - 1.0f) * 2.0f;
+  volatile float a = b - bmin;
+  return a >= tau;
+}
+
+float find_pstar(float tau, float eps) {
+  if (!chain_active(1.0f, tau, eps)) {
+    // no probability reaches tau; larger (non-softmax) inputs may: search up to the largest float
+    uint32_t lo = 0x3F800000u, hi = 0x7F7FFFFFu;
+    float fh; memcpy(&fh, &hi, 4);
+    if (!chain_active(fh, tau, eps)) return INFINITY;
+    while (hi - lo > 1) {
+      uint32_t mid = lo + (hi - lo) / 2; float fm; memcpy(&fm, &mid, 4);
+      if (chain_active(fm, tau, eps)) hi = mid; else lo = mid;
+    }
+    memcpy(&fh, &hi, 4);
+    return fh;
+  }
+  uint32_t lo = 0u, hi = 0x3F800000u;     // chain(0) is inactive because tau > 0
+  while (hi - lo > 1) {
+    uint32_t mid = lo + (hi - lo) / 2; float fm; memcpy(&fm, &mid, 4);
+    if (chain_active(fm, tau, eps)) hi = mid; else lo = mid;
+  }
+  float f; memcpy(&f, &hi, 4);
+  return f;
+}
+
+dam_status_t fill_ctx(const dam_shape_t* s, const dam_rule_t* r, void* mask, size_t cap, void* scratch,
+                      size_t scratch_bytes, Layout* y, DamBuildCtx* c) {
+  dam_status_t st;
+  if ((st = check_shape(s)) != DAM_OK) return st;
+  if ((st = check_rule(r)) != DAM_OK) return st;
+  if (!mask || !scratch || !aligned(mask, 256) || !aligned(scratch, 256)) return DAM_ERR_INVALID_ARGUMENT;
+  compute_layout(s, r->pcl_max, 1, y);
+  if (cap < y->mask_bytes || scratch_bytes < y->build_scratch_bytes) return DAM_ERR_BUFFER_TOO_SMALL;
+  c->blob = reinterpret_cast<unsigned char*>(mask);
+  c->scratch = reinterpret_cast<unsigned char*>(scratch);
+  c->num_seqs = s->num_seqs; c->Hq = s->num_q_heads; c->Hkv = s->num_kv_heads; c->d = s->head_dim; c->dtype = s->dtype;
+  c->total_qblocks = y->hdr.total_qblocks; c->rows = y->hdr.rows;
+  c->max_L = y->max_L; c->max_W = y->max_W; c->max_nL = y->max_nL; c->max_nq = y->max_nq;
+  c->pstar = find_pstar(r->tau, r->eps);
+  c->mu = r->mu; c->min_support = r->min_support;
+  c->scale = r->softmax_scale > 0.f ? r->softmax_scale : 1.0f / sqrtf((float)s->head_dim);
+  c->off_cnt = y->off_cnt; c->off_rowstat = y->off_rowstat; c->off_rowcnt = y->off_rowcnt;
+  c->off_hist = y->off_hist; c->off_cursor = y->off_cursor;
+  return DAM_OK;
+}
+
+bool sm100_shape(const dam_shape_t* s) {
+  return s->dtype == DAM_BF16 && s->head_dim == 128;
+}
+
+}  // namespace
+
+extern "C" {
+
+int32_t dam_version(void) { return 1000; }
+
+const char* dam_status_string(dam_status_t s) {
+  switch (s) {
+    case DAM_OK: return "ok";
+    case DAM_ERR_INVALID_ARGUMENT: return "invalid argument";
+    case DAM_ERR_UNSUPPORTED: return "unsupported";
+    case DAM_ERR_BUFFER_TOO_SMALL: return "buffer too small";
+    case DAM_ERR_CUDA: return "CUDA error";
+    case DAM_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    case DAM_ERR_INTERNAL: return "internal error";
+  }
+  return "unknown status";
+}
+
+dam_status_t dam_mask_sizes(const dam_shape_t* shape, const dam_rule_t* rule, int32_t causal, size_t* mask_bytes,
+                            size_t* build_scratch_bytes, size_t* attn_scratch_bytes) {
+  dam_status_t st;
+  if ((st = check_shape(shape)) != DAM_OK) return st;
+  if (rule && (st = check_rule(rule)) != DAM_OK) return st;
+  Layout y;
+  compute_layout(shape, rule ? rule->pcl_max : 0, causal != 0, &y);
+  if (mask_bytes) *mask_bytes = y.mask_bytes;
+  if (build_scratch_bytes) *build_scratch_bytes = rule ? y.build_scratch_bytes : 0;
+  if (attn_scratch_bytes) *attn_scratch_bytes = y.attn_scratch_bytes;
+  return DAM_OK;
+}
+
+dam_status_t dam_build_masks(const void* Q, const void* K, const dam_shape_t* shape, const dam_rule_t* rule,
+                             void* mask, size_t mask_capacity, void* scratch, size_t scratch_bytes,
+                             float* scores_dump, void* stream) {
+  Layout y; DamBuildCtx c;
+  dam_status_t st = fill_ctx(shape, rule, mask, mask_capacity, scratch, scratch_bytes, &y, &c);
+  if (st != DAM_OK) return st;
+  if (!Q || !K || !aligned(Q, 16) || !aligned(K, 16) || (scores_dump && !aligned(scores_dump, 16)))
+    return DAM_ERR_INVALID_ARGUMENT;
+  cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
+  if (dam_launch_init_blob(shape, rule->pcl_max, y.hdr.flags, mask, y.hdr.tile_capacity, y.hdr, cs) != cudaSuccess)
+    return DAM_ERR_CUDA;
+  cudaError_t e = cudaErrorNotSupported;
+  if (sm100_shape(shape)) e = dam_launch_scores_sm100(Q, K, shape, c, scores_dump, cs);
+  if (e == cudaErrorNotSupported) e = dam_launch_scores_ref(Q, K, shape, c, scores_dump, cs);
+  if (e != cudaSuccess) return DAM_ERR_CUDA;
+  if (dam_launch_rule(c, cs) != cudaSuccess) return DAM_ERR_CUDA;
+  return DAM_OK;
+}
+
+dam_status_t dam_build_masks_from_scores(const float* P, const dam_shape_t* shape, const dam_rule_t* rule,
+                                         void* mask, size_t mask_capacity, void* scratch, size_t scratch_bytes,
+                                         void* stream) {
+  Layout y; DamBuildCtx c;
+  dam_status_t st = fill_ctx(shape, rule, mask, mask_capacity, scratch, scratch_bytes, &y, &c);
+  if (st != DAM_OK) return st;
+  if (!P || !aligned(P, 4)) return DAM_ERR_INVALID_ARGUMENT;
+  cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
+  if (dam_launch_init_blob(shape, rule->pcl_max, y.hdr.flags, mask, y.hdr.tile_capacity, y.hdr, cs) != cudaSuccess)
+    return DAM_ERR_CUDA;
+  if (dam_launch_bits_from_scores(P, c, cs) != cudaSuccess) return DAM_ERR_CUDA;
+  if (dam_launch_rule(c, cs) != cudaSuccess) return DAM_ERR_CUDA;
+  return DAM_OK;
+}
+
+dam_status_t dam_mask_all_ones(const dam_shape_t* shape, int32_t causal, void* mask, size_t mask_capacity,
+                               void* stream) {
+  dam_status_t st;
+  if ((st = check_shape(shape)) != DAM_OK) return st;
+  if (!mask || !aligned(mask, 256)) return DAM_ERR_INVALID_ARGUMENT;
+  Layout y;
+  compute_layout(shape, 0, causal != 0, &y);
+  if (mask_capacity < y.mask_bytes) return DAM_ERR_BUFFER_TOO_SMALL;
+  cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
+  if (dam_launch_init_blob(shape, 0, y.hdr.flags, mask, y.hdr.tile_capacity, y.hdr, cs) != cudaSuccess)
+    return DAM_ERR_CUDA;
+  if (dam_launch_all_ones(shape, causal != 0, mask, cs) != cudaSuccess) return DAM_ERR_CUDA;
+  return DAM_OK;
+}
+
+dam_status_t dam_sparse_attention(const void* Q, const void* K, const void* V, const void* mask,
+                                  const dam_shape_t* shape, int32_t causal, int32_t gqa_group, float softmax_scale,
+                                  void* O, float* lse, void* scratch, size_t scratch_bytes, void* stream) {
+  dam_status_t st;
+  if ((st = check_shape(shape)) != DAM_OK) return st;
+  if (!Q || !K || !V || !mask || !O || !lse || !scratch) return DAM_ERR_INVALID_ARGUMENT;
+  if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16) || !aligned(lse, 4) ||
+      !aligned(mask, 256) || !aligned(scratch, 256))
+    return DAM_ERR_INVALID_ARGUMENT;
+  if (gqa_group != shape->num_q_heads / shape->num_kv_heads || softmax_scale < 0.f) return DAM_ERR_INVALID_ARGUMENT;
+  if (scratch_bytes < 256) return DAM_ERR_BUFFER_TOO_SMALL;
+  const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)shape->head_dim);
+  cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
+  // status word and work counter start at zero
+  if (cudaMemsetAsync(scratch, 0, 256, cs) != cudaSuccess) return DAM_ERR_CUDA;
+  cudaError_t e = cudaErrorNotSupported;
+  if (sm100_shape(shape)) e = dam_launch_attn_sm100(Q, K, V, mask, shape, causal != 0, scale, O, lse, scratch, cs);
+  if (e == cudaErrorNotSupported) e = dam_launch_attn_ref(Q, K, V, mask, shape, causal != 0, scale, O, lse, scratch, cs);
+  return e == cudaSuccess ? DAM_OK : DAM_ERR_CUDA;
+}
+
+dam_status_t dam_mask_stats(const void* mask, const dam_shape_t* shape, uint64_t* out, void* stream) {
+  if (!mask || !out || !shape) return DAM_ERR_INVALID_ARGUMENT;
+  cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
+  DamHeader h;
+  if (cudaMemcpyAsync(&h, mask, sizeof(h), cudaMemcpyDeviceToHost, cs) != cudaSuccess) return DAM_ERR_CUDA;
+  if (cudaStreamSynchronize(cs) != cudaSuccess) return DAM_ERR_CUDA;
+  if (h.magic != DAM_MAGIC) return DAM_ERR_INVALID_ARGUMENT;
+  out[0] = h.total_tiles; out[1] = h.full_tiles; out[2] = h.causal_tiles; out[3] = h.bytes_used;
+  return DAM_OK;
+}
+
+dam_status_t dam_mask_expand_rows(const void* mask, const dam_shape_t* shape, int32_t seq, int32_t head,
+                                  int32_t row_begin, int32_t nrows, int32_t causal, uint32_t* out_bits,
+                                  void* stream) {
+  dam_status_t st;
+  if ((st = check_shape(shape)) != DAM_OK) return st;
+  if (!mask || !out_bits || seq < 0 || seq >= shape->num_seqs || head < 0 || head >= shape->num_q_heads ||
+      nrows < 0 || row_begin < 0)
+    return DAM_ERR_INVALID_ARGUMENT;
+  if (nrows == 0) return DAM_OK;
+  int S = shape->cu_seqlens_host[seq + 1] - shape->cu_seqlens_host[seq];
+  int words = ((S + DAM_TILE - 1) / DAM_TILE) * 4;
+  if (words == 0) return DAM_OK;
+  cudaError_t e = dam_launch_expand_rows(mask, seq, head, row_begin, nrows, words, causal != 0, out_bits,
+                                         reinterpret_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? DAM_OK : DAM_ERR_CUDA;
+}
+
+dam_status_t dam_poll_status(const void* mask_or_scratch, void* stream) {
+  if (!mask_or_scratch) return DAM_ERR_INVALID_ARGUMENT;
+  cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
+  uint32_t w[2] = {0, 0};
+  if (cudaMemcpyAsync(w, mask_or_scratch, sizeof(w), cudaMemcpyDeviceToHost, cs) != cudaSuccess) return DAM_ERR_CUDA;
+  if (cudaStreamSynchronize(cs) != cudaSuccess) return DAM_ERR_CUDA;
+  if (w[1] > DAM_ERR_INTERNAL) return DAM_ERR_INTERNAL;
+  return static_cast<dam_status_t>(w[1]);
+}
+
+dam_status_t dam_prefill_host(const void* Qh, const void* Kh, const void* Vh, const dam_shape_t* shape,
+                              const dam_rule_t* rule, int32_t causal, void* Oh, float* lse_h, void* workspace,
+                              size_t* workspace_bytes, void* stream) {
+  dam_status_t st;
+  if ((st = check_shape(shape)) != DAM_OK) return st;
+  if ((st = check_rule(rule)) != DAM_OK) return st;
+  if (!workspace_bytes) return DAM_ERR_INVALID_ARGUMENT;
+  const size_t es = shape->dtype == DAM_BF16 ? 2 : 4;
+  const int64_t T = shape->total_tokens, Hq = shape->num_q_heads, Hkv = shape->num_kv_heads, d = shape->head_dim;
+  // dense strides only
+  if (shape->q_stride_head != d || shape->q_stride_tok != Hq * d || shape->k_stride_head != d ||
+      shape->k_stride_tok != Hkv * d || shape->v_stride_head != d || shape->v_stride_tok != Hkv * d ||
+      shape->o_stride_head != d || shape->o_stride_tok != Hq * d)
+    return DAM_ERR_UNSUPPORTED;
+  Layout y;
+  compute_layout(shape, rule->pcl_max, 1, &y);
+  const size_t qb = dam_align((size_t)T * Hq * d * es, 256), kb = dam_align((size_t)T * Hkv * d * es, 256);
+  const size_t lb = dam_align((size_t)Hq * T * 4, 256);
+  size_t off_q = 0, off_k = off_q + qb, off_v = off_k + kb, off_o = off_v + kb, off_l = off_o + qb;
+  size_t off_m = off_l + lb, off_bs = off_m + y.mask_bytes, off_as = off_bs + y.build_scratch_bytes;
+  size_t total = off_as + y.attn_scratch_bytes;
+  if (!workspace) { *workspace_bytes = total; return DAM_OK; }
+  if (*workspace_bytes < total) return DAM_ERR_BUFFER_TOO_SMALL;
+  if (!Qh || !Kh || !Vh || !Oh || !lse_h || !aligned(workspace, 256)) return DAM_ERR_INVALID_ARGUMENT;
+  cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
+  unsigned char* w = reinterpret_cast<unsigned char*>(workspace);
+  if (cudaMemcpyAsync(w + off_q, Qh, (size_t)T * Hq * d * es, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
+      cudaMemcpyAsync(w + off_k, Kh, (size_t)T * Hkv * d * es, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
+      cudaMemcpyAsync(w + off_v, Vh, (size_t)T * Hkv * d * es, cudaMemcpyHostToDevice, cs) != cudaSuccess)
+    return DAM_ERR_CUDA;
+  st = dam_build_masks(w + off_q, w + off_k, shape, rule, w + off_m, y.mask_bytes, w + off_bs, y.build_scratch_bytes,
+                       nullptr, stream);
+  if (st != DAM_OK) return st;
+  st = dam_sparse_attention(w + off_q, w + off_k, w + off_v, w + off_m, shape, causal,
+                            shape->num_q_heads / shape->num_kv_heads, rule->softmax_scale, w + off_o,
+                            reinterpret_cast<float*>(w + off_l), w + off_as, y.attn_scratch_bytes, stream);
+  if (st != DAM_OK) return st;
+  if (cudaMemcpyAsync(Oh, w + off_o, (size_t)T * Hq * d * es, cudaMemcpyDeviceToHost, cs) != cudaSuccess ||
+      cudaMemcpyAsync(lse_h, w + off_l, (size_t)Hq * T * 4, cudaMemcpyDeviceToHost, cs) != cudaSuccess)
+    return DAM_ERR_CUDA;
+  if (cudaStreamSynchronize(cs) != cudaSuccess) return DAM_ERR_CUDA;
+  st = dam_poll_status(w + off_m, stream);
+  if (st != DAM_OK) return st;
+  return dam_poll_status(w + off_as, stream);
+}
+
+}  // extern "C"

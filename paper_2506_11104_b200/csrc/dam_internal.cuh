@@ -1,0 +1,189 @@
+// Internal layout of the mask blob and device helpers shared by the DAM kernels.
+//
+// The blob is one flat, relocatable buffer (byte offsets from its start, little endian):
+//
+//   DamHeader (256 B)            magic, status word, counts, section offsets
+//   DamSeq[num_seqs]             per sequence: token start, S, L = min(S, pcl_max), q-block range,
+//                                word offsets of its bit sections
+//   qb_seq[total_qblocks]        sequence index of every global 128-row query block
+//   per (seq, head) pattern bits 3 * W words: D (matched diagonal offsets r), Drev (D reversed:
+//                                bit x = D[L-1-x]), V (matched columns c); W = ceil(L/32) rounded
+//                                up to a multiple of 4 words
+//   per (seq, head) true mask    L rows x W words, bit (j % 32) of word (j / 32) = M[i][j]
+//   tile_ptr[rows + 1]           CSR over rows = head * total_qblocks + global q-block
+//   work_order[rows]             row ids, longest tile list first
+//   tiles[...]                   one u32 per listed tile: kv tile index | kind << 28
+//
+// A PARTIAL tile stores no bits of its own: inside the window they are the true-mask words of the
+// row, below it they follow from V and Drev (Sec. 4.3, Case 2), see dam_tile_row_bits.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/dam.h"
+
+#define DAM_TILE 128
+#define DAM_MAGIC 0x4B4D4144u      /* "DAMK" */
+#define DAM_SCRATCH_MAGIC 0x534D4144u /* "DAMS" */
+#define DAM_KIND_FULL 1u
+#define DAM_KIND_PARTIAL 2u
+#define DAM_FLAG_ALL_ONES 1u
+#define DAM_FLAG_CAUSAL_LIST 2u    /* tile lists hold only kb <= qb */
+#define DAM_HIST 4096
+
+struct DamHeader {
+  uint32_t magic;
+  uint32_t status;          // device-side dam_status_t, 0 = ok
+  uint32_t version;
+  uint32_t flags;
+  int32_t num_seqs;
+  int32_t num_q_heads;
+  int32_t total_qblocks;
+  int32_t rows;             // num_q_heads * total_qblocks
+  uint32_t tile_capacity;   // entries that fit in tiles[]
+  uint32_t total_tiles;     // entries in use
+  uint32_t full_tiles;
+  uint32_t pcl_max;
+  uint64_t off_seq, off_qbseq, off_dv, off_true, off_tile_ptr, off_work, off_tiles;
+  uint64_t bytes_used;
+  uint64_t causal_tiles;    // sum over heads and sequences of nq (nq + 1) / 2
+  uint64_t reserved[17];
+};
+static_assert(sizeof(DamHeader) == 256, "DamHeader must be 256 bytes");
+
+struct DamSeq {
+  int32_t tok_start, S, L, nq;
+  int32_t first_qblock, W, nL, pad;
+  uint64_t dv_off;     // u32 words from off_dv: head h at dv_off + h * 3 * W
+  uint64_t true_off;   // u32 words from off_true: head h at true_off + h * L * W
+  uint64_t p_off;      // fp32 elements into a score tensor: head h at p_off + h * L * L
+  uint64_t cnt_off;    // int32 elements into the build scratch count area: head h at cnt_off + h * cnt_stride
+};
+static_assert(sizeof(DamSeq) == 64, "DamSeq must be 64 bytes");
+
+// Per-(seq, head) words in the build scratch count area:
+//   cntD[L], cntV[L], prefD[W + 1], prefV[W + 1], tile_pop[nL * nL], padded to a multiple of 4.
+__host__ __device__ inline uint64_t dam_cnt_stride(int L, int W, int nL) {
+  uint64_t n = 2ull * L + 2ull * (W + 1) + (uint64_t)nL * nL;
+  return (n + 3) & ~3ull;
+}
+__host__ __device__ inline int dam_words(int L) { return (((L + 31) >> 5) + 3) & ~3; }
+__host__ __device__ inline uint64_t dam_align(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+
+// Upper bound on listed tiles of one q-block row of a DAM mask (see dam_mask_sizes).
+__host__ __device__ inline int dam_row_tile_bound(int qb, int nL) {
+  int a = qb + 1, b = 2 * nL + 1;
+  return a < b ? a : b;
+}
+
+struct DamHeadBits {
+  const uint32_t* D;
+  const uint32_t* Drev;
+  const uint32_t* V;
+  const uint32_t* M;
+  int L, W, S;
+};
+
+__device__ __forceinline__ DamHeadBits dam_head_bits(const unsigned char* blob, const DamHeader* hdr,
+                                                     const DamSeq& sq, int head) {
+  DamHeadBits hb;
+  const uint32_t* dv = reinterpret_cast<const uint32_t*>(blob + hdr->off_dv) + sq.dv_off + (uint64_t)head * 3 * sq.W;
+  hb.D = dv;
+  hb.Drev = dv + sq.W;
+  hb.V = dv + 2 * sq.W;
+  hb.M = reinterpret_cast<const uint32_t*>(blob + hdr->off_true) + sq.true_off + (uint64_t)head * sq.L * sq.W;
+  hb.L = sq.L;
+  hb.W = sq.W;
+  hb.S = sq.S;
+  return hb;
+}
+
+// bits [x, x + 32) of a bit array of nwords words; zero outside the array. x may be negative.
+__device__ __forceinline__ uint32_t dam_window32(const uint32_t* __restrict__ bits, int nwords, int x) {
+  int w = x >> 5;  // arithmetic shift: floor
+  int sh = x & 31;
+  uint32_t lo = (w >= 0 && w < nwords) ? __ldg(bits + w) : 0u;
+  uint32_t hi = (w + 1 >= 0 && w + 1 < nwords) ? __ldg(bits + w + 1) : 0u;
+  return __funnelshift_r(lo, hi, sh);
+}
+
+// The 128 mask bits of row i (index inside the sequence) against kv tile kb of a PARTIAL tile.
+// Inside the window (i < L): the true-mask words.  Below it: matched columns of this tile OR the
+// matched diagonals, key j active iff D[i - j]; with Drev[x] = D[L-1-x] the keys j0 .. j0+127 read
+// Drev bits x0 .. x0+127, x0 = L - 1 - i + j0 (ascending in j), which also excludes j > i.
+__device__ __forceinline__ uint4 dam_tile_row_bits(const DamHeadBits& hb, int i, int kb) {
+  uint4 r = make_uint4(0u, 0u, 0u, 0u);
+  const int j0 = kb * DAM_TILE;
+  if (i >= hb.S) return r;
+  if (i < hb.L) {
+    if (j0 < hb.L) r = __ldg(reinterpret_cast<const uint4*>(hb.M + (size_t)i * hb.W + kb * 4));
+  } else {
+    if (j0 < hb.L) r = __ldg(reinterpret_cast<const uint4*>(hb.V + kb * 4));
+    const int x0 = hb.L - 1 - i + j0;
+    if (x0 + DAM_TILE > 0 && x0 < hb.L) {
+      r.x |= dam_window32(hb.Drev, hb.W, x0);
+      r.y |= dam_window32(hb.Drev, hb.W, x0 + 32);
+      r.z |= dam_window32(hb.Drev, hb.W, x0 + 64);
+      r.w |= dam_window32(hb.Drev, hb.W, x0 + 96);
+    }
+  }
+  return r;
+}
+
+// ones for t in [0, n), n clipped to [0, 128]
+__device__ __forceinline__ uint4 dam_low_ones128(int n) {
+  uint4 r;
+  auto w = [](int k) -> uint32_t { return k >= 32 ? 0xFFFFFFFFu : (k <= 0 ? 0u : ((1u << k) - 1u)); };
+  r.x = w(n);
+  r.y = w(n - 32);
+  r.z = w(n - 64);
+  r.w = w(n - 96);
+  return r;
+}
+
+// Final 128 bits the attention kernels apply for row i against tile kb.
+__device__ __forceinline__ uint4 dam_apply_bits(const DamHeadBits& hb, uint32_t kind, int i, int kb, int causal) {
+  uint4 b = (kind == DAM_KIND_FULL) ? make_uint4(~0u, ~0u, ~0u, ~0u) : dam_tile_row_bits(hb, i, kb);
+  const int j0 = kb * DAM_TILE;
+  if (i >= hb.S) return make_uint4(0u, 0u, 0u, 0u);
+  int n = hb.S - j0;                       // keys beyond the sequence end do not exist
+  if (causal) { int c = i - j0 + 1; n = c < n ? c : n; }
+  if (n < DAM_TILE) {
+    uint4 m = dam_low_ones128(n);
+    b.x &= m.x; b.y &= m.y; b.z &= m.z; b.w &= m.w;
+  }
+  return b;
+}
+
+// ---- host-side launch entry points of the kernel files -----------------------------------------
+struct DamBuildCtx {
+  unsigned char* blob;
+  unsigned char* scratch;
+  int num_seqs, Hq, Hkv, d, dtype;
+  int total_qblocks, rows;
+  int max_L, max_W, max_nL, max_nq;
+  float pstar;       // single-compare threshold on p equivalent to the Box-Cox chain
+  float mu;
+  int min_support;
+  float scale;
+  uint64_t off_cnt, off_rowstat, off_rowcnt, off_hist, off_cursor;   // scratch sections
+};
+
+cudaError_t dam_launch_init_blob(const dam_shape_t* shape, int pcl_max, uint32_t flags, void* blob,
+                                 uint32_t tile_capacity, const DamHeader& host_hdr, cudaStream_t st);
+cudaError_t dam_launch_scores_ref(const void* Q, const void* K, const dam_shape_t* shape, const DamBuildCtx& c,
+                                  float* scores_dump, cudaStream_t st);
+cudaError_t dam_launch_bits_from_scores(const float* P, const DamBuildCtx& c, cudaStream_t st);
+cudaError_t dam_launch_rule(const DamBuildCtx& c, cudaStream_t st);
+cudaError_t dam_launch_all_ones(const dam_shape_t* shape, int causal, void* blob, cudaStream_t st);
+cudaError_t dam_launch_expand_rows(const void* blob, int seq, int head, int row_begin, int nrows, int words,
+                                   int causal, uint32_t* out, cudaStream_t st);
+cudaError_t dam_launch_attn_ref(const void* Q, const void* K, const void* V, const void* blob,
+                                const dam_shape_t* shape, int causal, float scale, void* O, float* lse,
+                                void* scratch, cudaStream_t st);
+// tensor-core paths (bf16, d = 128); return cudaErrorNotSupported when the shape does not qualify
+cudaError_t dam_launch_attn_sm100(const void* Q, const void* K, const void* V, const void* blob,
+                                  const dam_shape_t* shape, int causal, float scale, void* O, float* lse,
+                                  void* scratch, cudaStream_t st);
+cudaError_t dam_launch_scores_sm100(const void* Q, const void* K, const dam_shape_t* shape, const DamBuildCtx& c,
+                                    float* scores_dump, cudaStream_t st);

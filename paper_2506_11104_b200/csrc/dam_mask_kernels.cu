@@ -1,0 +1,491 @@
+// Stage-1 rule kernels: true-mask bits from a score tensor, diagonal / column counts, pattern
+// match, tile classification and emission of the tile lists (paper Sec. 4.2.2 - 4.2.4, Sec. 4.3).
+// Integer / bit work throughout; the only floating-point operations are the single compare
+// p >= p* (equivalent to the Box-Cox threshold chain, see dam_api.cu) and one fp32 multiply +
+// compare per pattern.
+#include "dam_internal.cuh"
+
+namespace {
+
+__device__ __forceinline__ const DamSeq* blob_seqs(const unsigned char* blob, const DamHeader* h) {
+  return reinterpret_cast<const DamSeq*>(blob + h->off_seq);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Header + per-sequence table + q-block table, computed on the device from cu_seqlens so that no
+// host buffer has to outlive the call.  One block.
+// ---------------------------------------------------------------------------------------------
+__global__ void init_blob_kernel(unsigned char* blob, DamHeader hdr, const int32_t* __restrict__ cu,
+                                 int pcl_max, int Hq, int all_ones_causal /* -1: DAM mask */) {
+  DamHeader* H = reinterpret_cast<DamHeader*>(blob);
+  DamSeq* seqs = reinterpret_cast<DamSeq*>(blob + hdr.off_seq);
+  int32_t* qbseq = reinterpret_cast<int32_t*>(blob + hdr.off_qbseq);
+  if (threadIdx.x == 0) {
+    *H = hdr;
+    uint64_t dv = 0, tr = 0, po = 0, co = 0;
+    int fq = 0;
+    for (int b = 0; b < hdr.num_seqs; ++b) {
+      int t0 = cu[b], S = cu[b + 1] - t0;
+      int L = S < pcl_max ? S : pcl_max;
+      if (L < 0) L = 0;
+      int W = L > 0 ? dam_words(L) : 0;
+      int nL = (L + DAM_TILE - 1) / DAM_TILE;
+      int nq = (S + DAM_TILE - 1) / DAM_TILE;
+      DamSeq s;
+      s.tok_start = t0; s.S = S; s.L = L; s.nq = nq;
+      s.first_qblock = fq; s.W = W; s.nL = nL; s.pad = 0;
+      s.dv_off = dv; s.true_off = tr; s.p_off = po; s.cnt_off = co;
+      seqs[b] = s;
+      dv += (uint64_t)Hq * 3 * W;
+      tr += (uint64_t)Hq * L * W;
+      po += (uint64_t)Hq * L * L;
+      if (all_ones_causal < 0) co += (uint64_t)Hq * dam_cnt_stride(L, W, nL);
+      else co += all_ones_causal ? (uint64_t)nq * (nq + 1) / 2 : (uint64_t)nq * nq;   // tile base per head
+      fq += nq;
+    }
+  }
+  __syncthreads();
+  for (int b = 0; b < hdr.num_seqs; ++b) {
+    int fq = seqs[b].first_qblock, nq = seqs[b].nq;
+    for (int q = threadIdx.x; q < nq; q += blockDim.x) qbseq[fq + q] = b;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// True-mask bits from an fp32 map P ([L][L] per (seq, head)): bit = [P >= p*], forced to 0 above
+// the diagonal.  One warp per (row, 32-column word); coalesced reads, one word written per warp.
+// ---------------------------------------------------------------------------------------------
+__global__ void bits_from_scores_kernel(unsigned char* blob, const float* __restrict__ P, float pstar) {
+  const DamHeader* H = reinterpret_cast<const DamHeader*>(blob);
+  const int sh = blockIdx.y;
+  const int b = sh / H->num_q_heads, h = sh % H->num_q_heads;
+  const DamSeq sq = blob_seqs(blob, H)[b];
+  if (sq.L == 0) return;
+  uint32_t* M = reinterpret_cast<uint32_t*>(blob + H->off_true) + sq.true_off + (uint64_t)h * sq.L * sq.W;
+  const float* Ph = P + sq.p_off + (uint64_t)h * sq.L * sq.L;
+  const int lane = threadIdx.x & 31;
+  const long long nitems = (long long)sq.L * sq.W;
+  const long long wstride = (long long)gridDim.x * (blockDim.x >> 5);
+  for (long long it = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); it < nitems; it += wstride) {
+    int i = (int)(it / sq.W), w = (int)(it % sq.W);
+    int j = w * 32 + lane;
+    float p = (j < sq.L && j <= i) ? __ldg(Ph + (size_t)i * sq.L + j) : 0.0f;
+    uint32_t word = __ballot_sync(0xFFFFFFFFu, p >= pstar);
+    if (lane == 0) M[(size_t)i * sq.W + w] = word;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Counts: one block per 128 x 128 tile (qb, kb <= qb) of the window.  Thread t owns row qb*128+t
+// and its 128 bits.  Column counts (128), diagonal counts (255) and the tile's popcount are
+// accumulated in shared memory and flushed with integer atomics (order-independent).
+// ---------------------------------------------------------------------------------------------
+__global__ void counts_kernel(const unsigned char* blob, unsigned char* scratch, uint64_t off_cnt) {
+  const DamHeader* H = reinterpret_cast<const DamHeader*>(blob);
+  const int sh = blockIdx.y;
+  const int b = sh / H->num_q_heads, h = sh % H->num_q_heads;
+  const DamSeq sq = blob_seqs(blob, H)[b];
+  const int nL = sq.nL;
+  // tile index -> (qb, kb) over the lower triangle
+  int t = blockIdx.x;
+  if (t >= nL * (nL + 1) / 2) return;
+  int qb = (int)((sqrtf(8.0f * t + 1.0f) - 1.0f) * 0.5f);
+  while ((qb + 1) * (qb + 2) / 2 <= t) ++qb;
+  while (qb * (qb + 1) / 2 > t) --qb;
+  const int kb = t - qb * (qb + 1) / 2;
+
+  const uint32_t* M = reinterpret_cast<const uint32_t*>(blob + H->off_true) + sq.true_off + (uint64_t)h * sq.L * sq.W;
+  int32_t* cnt = reinterpret_cast<int32_t*>(scratch + off_cnt) + sq.cnt_off + (uint64_t)h * dam_cnt_stride(sq.L, sq.W, nL);
+  int32_t* cntD = cnt;
+  int32_t* cntV = cnt + sq.L;
+  int32_t* tile_pop = cnt + 2 * sq.L + 2 * (sq.W + 1);
+
+  __shared__ int sV[DAM_TILE];
+  __shared__ int sD[2 * DAM_TILE];
+  __shared__ int sPop;
+  const int tid = threadIdx.x;
+  const int i = qb * DAM_TILE + tid;
+  uint4 bits = make_uint4(0, 0, 0, 0);
+  if (i < sq.L) bits = __ldg(reinterpret_cast<const uint4*>(M + (size_t)i * sq.W + kb * 4));
+  const int nz = (bits.x | bits.y | bits.z | bits.w) != 0;
+  if (!__syncthreads_or(nz)) return;
+  sV[tid] = 0; sD[tid] = 0; sD[tid + DAM_TILE] = 0;
+  if (tid == 0) sPop = 0;
+  __syncthreads();
+  if (nz) {
+    uint32_t w[4] = {bits.x, bits.y, bits.z, bits.w};
+    int pop = 0;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      uint32_t x = w[q];
+      pop += __popc(x);
+      while (x) {
+        int c = q * 32 + (__ffs(x) - 1);
+        x &= x - 1;
+        atomicAdd(&sV[c], 1);
+        atomicAdd(&sD[tid - c + (DAM_TILE - 1)], 1);
+      }
+    }
+    atomicAdd(&sPop, pop);
+  }
+  __syncthreads();
+  {
+    int c = kb * DAM_TILE + tid;
+    if (sV[tid] && c < sq.L) atomicAdd(&cntV[c], sV[tid]);
+    for (int idx = tid; idx < 2 * DAM_TILE - 1; idx += DAM_TILE) {
+      int r = (qb - kb) * DAM_TILE + idx - (DAM_TILE - 1);
+      if (sD[idx] && r >= 0 && r < sq.L) atomicAdd(&cntD[r], sD[idx]);
+    }
+    if (tid == 0) tile_pop[qb * nL + kb] = sPop;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Match: D[r] = [cntD[r] >= mu * (L - r)], V[c] likewise (one fp32 multiply, one compare), written
+// as bit sets; Drev = D reversed; prefix popcounts per word for range queries.  Block per (seq, head).
+// ---------------------------------------------------------------------------------------------
+__global__ void match_kernel(unsigned char* blob, unsigned char* scratch, uint64_t off_cnt, float mu, int min_support) {
+  const DamHeader* H = reinterpret_cast<const DamHeader*>(blob);
+  const int sh = blockIdx.x;
+  const int b = sh / H->num_q_heads, h = sh % H->num_q_heads;
+  const DamSeq sq = blob_seqs(blob, H)[b];
+  if (sq.L == 0) return;
+  const int L = sq.L, W = sq.W;
+  uint32_t* dv = reinterpret_cast<uint32_t*>(blob + H->off_dv) + sq.dv_off + (uint64_t)h * 3 * W;
+  uint32_t* Dw = dv; uint32_t* Rw = dv + W; uint32_t* Vw = dv + 2 * W;
+  int32_t* cnt = reinterpret_cast<int32_t*>(scratch + off_cnt) + sq.cnt_off + (uint64_t)h * dam_cnt_stride(L, W, sq.nL);
+  const int32_t* cntD = cnt;
+  const int32_t* cntV = cnt + L;
+  int32_t* prefD = cnt + 2 * L;
+  int32_t* prefV = prefD + (W + 1);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  for (int w = warp; w < W; w += nw) {
+    int k = w * 32 + lane;
+    bool d = false, v = false;
+    if (k < L) {
+      int size = L - k;
+      float need = __fmul_rn(mu, (float)size);
+      bool ok = size >= min_support;
+      d = ok && ((float)cntD[k] >= need);
+      v = ok && ((float)cntV[k] >= need);
+    }
+    uint32_t dw = __ballot_sync(0xFFFFFFFFu, d), vw = __ballot_sync(0xFFFFFFFFu, v);
+    if (lane == 0) { Dw[w] = dw; Vw[w] = vw; }
+  }
+  __threadfence_block();
+  __syncthreads();
+  for (int w = warp; w < W; w += nw) {
+    int x = w * 32 + lane;
+    int src = L - 1 - x;
+    bool bit = (x < L) && ((Dw[src >> 5] >> (src & 31)) & 1u);
+    uint32_t rw = __ballot_sync(0xFFFFFFFFu, bit);
+    if (lane == 0) Rw[w] = rw;
+  }
+  if (threadIdx.x == 0) {
+    int a = 0, c = 0;
+    for (int w = 0; w < W; ++w) {
+      prefD[w] = a; prefV[w] = c;
+      a += __popc(Dw[w]); c += __popc(Vw[w]);
+    }
+    prefD[W] = a; prefV[W] = c;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Tile classification.  One warp per row = (head, global q-block); lanes test candidate kv tiles in
+// ascending order.  pass 0 counts, pass 1 writes entries at tile_ptr[row] + rank.
+// ---------------------------------------------------------------------------------------------
+struct HeadView {
+  const uint32_t* Dw; const uint32_t* Vw;
+  const int32_t* prefD; const int32_t* prefV; const int32_t* tile_pop;
+  int L, W, nL, S;
+};
+
+__device__ __forceinline__ int cnt_below(const uint32_t* bits, const int32_t* pref, int x) {
+  int w = x >> 5, s = x & 31;
+  int c = pref[w];
+  if (s) c += __popc(bits[w] & ((1u << s) - 1u));
+  return c;
+}
+__device__ __forceinline__ int cnt_range(const uint32_t* bits, const int32_t* pref, int lo, int hi) {
+  return cnt_below(bits, pref, hi + 1) - cnt_below(bits, pref, lo);
+}
+
+// returns 0 (empty), DAM_KIND_FULL or DAM_KIND_PARTIAL
+__device__ __forceinline__ uint32_t classify_tile(const HeadView& v, int qb, int kb) {
+  const int i0 = qb * DAM_TILE;
+  const int i1 = min(i0 + DAM_TILE, v.S);
+  const int j0 = kb * DAM_TILE;
+  bool act = false, full = false;
+  if (i0 < v.L && j0 < v.L) {                       // rows inside the window: the true mask
+    int pop = v.tile_pop[qb * v.nL + kb];
+    act = pop > 0;
+    full = pop == DAM_TILE * DAM_TILE;
+  }
+  if (i1 > v.L && v.L > 0) {                        // rows below the window: matched patterns
+    const int a = max(i0, v.L);
+    const bool whole = (a == i0) && (i1 - i0 == DAM_TILE) && (kb < qb);
+    if (j0 < v.L) {
+      int hi = min(j0 + DAM_TILE - 1, v.L - 1);
+      int n = cnt_range(v.Vw, v.prefV, j0, hi);
+      act |= n > 0;
+      full |= whole && n == DAM_TILE;
+    }
+    int rlo = a - (j0 + DAM_TILE - 1), rhi = (i1 - 1) - j0;
+    int clo = max(rlo, 0), chi = min(rhi, v.L - 1);
+    if (clo <= chi) {
+      int n = cnt_range(v.Dw, v.prefD, clo, chi);
+      act |= n > 0;
+      full |= whole && clo == rlo && chi == rhi && n == 2 * DAM_TILE - 1;
+    }
+  }
+  return act ? (full ? DAM_KIND_FULL : DAM_KIND_PARTIAL) : 0u;
+}
+
+template <int PASS>
+__global__ void classify_kernel(unsigned char* blob, unsigned char* scratch, uint64_t off_cnt, uint64_t off_rowcnt,
+                                uint64_t off_hist, uint64_t off_cursor) {
+  DamHeader* H = reinterpret_cast<DamHeader*>(blob);
+  const int lane = threadIdx.x & 31;
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= H->rows) return;
+  const int h = row / H->total_qblocks, gqb = row % H->total_qblocks;
+  const int b = reinterpret_cast<const int32_t*>(blob + H->off_qbseq)[gqb];
+  const DamSeq sq = blob_seqs(blob, H)[b];
+  const int qb = gqb - sq.first_qblock;
+  HeadView v;
+  const uint32_t* dv = reinterpret_cast<const uint32_t*>(blob + H->off_dv) + sq.dv_off + (uint64_t)h * 3 * sq.W;
+  const int32_t* cnt = reinterpret_cast<const int32_t*>(scratch + off_cnt) + sq.cnt_off +
+                       (uint64_t)h * dam_cnt_stride(sq.L, sq.W, sq.nL);
+  v.Dw = dv; v.Vw = dv + 2 * sq.W;
+  v.prefD = cnt + 2 * sq.L; v.prefV = v.prefD + (sq.W + 1); v.tile_pop = v.prefV + (sq.W + 1);
+  v.L = sq.L; v.W = sq.W; v.nL = sq.nL; v.S = sq.S;
+
+  // candidates, ascending: [0, min(qb, nL-1)] then [max(that + 1, qb - nL), qb]
+  const int n1 = min(qb, sq.nL - 1) + 1;
+  const int lo2 = max(n1, qb - sq.nL);
+  const int n2 = max(0, qb - lo2 + 1);
+  uint32_t* rowcnt = reinterpret_cast<uint32_t*>(scratch + off_rowcnt);
+  uint32_t* tile_ptr = reinterpret_cast<uint32_t*>(blob + H->off_tile_ptr);
+  uint32_t* tiles = reinterpret_cast<uint32_t*>(blob + H->off_tiles);
+  uint32_t base = 0;
+  if (PASS == 1) {
+    base = tile_ptr[row];
+    if (base + rowcnt[row] > H->tile_capacity) return;   // overflow already flagged by the scan
+  }
+  int total = 0, nfull = 0;
+  for (int c0 = 0; c0 < n1 + n2; c0 += 32) {
+    int idx = c0 + lane;
+    uint32_t kind = 0;
+    int kb = 0;
+    if (idx < n1 + n2) {
+      kb = idx < n1 ? idx : lo2 + (idx - n1);
+      kind = classify_tile(v, qb, kb);
+    }
+    uint32_t m = __ballot_sync(0xFFFFFFFFu, kind != 0);
+    if (PASS == 1 && kind) {
+      int rank = __popc(m & ((1u << lane) - 1u));
+      tiles[base + total + rank] = (uint32_t)kb | (kind << 28);
+    }
+    if (PASS == 1) nfull += __popc(__ballot_sync(0xFFFFFFFFu, kind == DAM_KIND_FULL));
+    total += __popc(m);
+  }
+  if (lane == 0) {
+    if (PASS == 0) {
+      rowcnt[row] = total;
+      atomicAdd(reinterpret_cast<uint32_t*>(scratch + off_hist) + min(total, DAM_HIST - 1), 1u);
+    } else {
+      uint32_t pos = atomicAdd(reinterpret_cast<uint32_t*>(scratch + off_cursor) + min(total, DAM_HIST - 1), 1u);
+      reinterpret_cast<uint32_t*>(blob + H->off_work)[pos] = row;
+      if (nfull) atomicAdd(&H->full_tiles, (uint32_t)nfull);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Exclusive scans, one block of 1024 threads: tile_ptr over row counts, and the work-order
+// cursors (rows with more tiles first) over the histogram.
+// ---------------------------------------------------------------------------------------------
+__device__ uint32_t block_excl_scan(uint32_t x, uint32_t* total, uint32_t* sm /* 32 */) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t inc = x;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+    if (lane >= o) inc += y;
+  }
+  if (lane == 31) sm[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    uint32_t s = sm[lane];
+    uint32_t si = s;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      uint32_t y = __shfl_up_sync(0xFFFFFFFFu, si, o);
+      if (lane >= o) si += y;
+    }
+    sm[lane] = si - s;
+    if (lane == 31) *total = si;
+  }
+  __syncthreads();
+  uint32_t r = sm[warp] + inc - x;
+  __syncthreads();
+  return r;
+}
+
+__global__ void scan_kernel(unsigned char* blob, unsigned char* scratch, uint64_t off_rowcnt, uint64_t off_hist,
+                            uint64_t off_cursor) {
+  DamHeader* H = reinterpret_cast<DamHeader*>(blob);
+  __shared__ uint32_t sm[32];
+  __shared__ uint32_t tot;
+  const uint32_t* rowcnt = reinterpret_cast<const uint32_t*>(scratch + off_rowcnt);
+  uint32_t* tile_ptr = reinterpret_cast<uint32_t*>(blob + H->off_tile_ptr);
+  const int rows = H->rows;
+  uint32_t run = 0;
+  for (int base = 0; base < rows; base += blockDim.x) {
+    int r = base + threadIdx.x;
+    uint32_t x = r < rows ? rowcnt[r] : 0u;
+    uint32_t e = block_excl_scan(x, &tot, sm);
+    if (r < rows) tile_ptr[r] = run + e;
+    run += tot;
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    tile_ptr[rows] = run;
+    H->total_tiles = run;
+    H->bytes_used = H->off_tiles + 4ull * run;
+    if (run > H->tile_capacity) H->status = DAM_ERR_BUFFER_TOO_SMALL;
+  }
+  // cursors: bucket c starts after all buckets with more tiles
+  const uint32_t* hist = reinterpret_cast<const uint32_t*>(scratch + off_hist);
+  uint32_t* cursor = reinterpret_cast<uint32_t*>(scratch + off_cursor);
+  run = 0;
+  for (int base = 0; base < DAM_HIST; base += blockDim.x) {
+    int c = DAM_HIST - 1 - (base + threadIdx.x);
+    uint32_t x = hist[c];
+    uint32_t e = block_excl_scan(x, &tot, sm);
+    cursor[c] = run + e;
+    run += tot;
+    __syncthreads();
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// All-ones blob: every (causal: lower-triangular) tile listed as FULL.
+// ---------------------------------------------------------------------------------------------
+__global__ void all_ones_kernel(unsigned char* blob, int causal) {
+  DamHeader* H = reinterpret_cast<DamHeader*>(blob);
+  const int lane = threadIdx.x & 31;
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= H->rows) return;
+  const int h = row / H->total_qblocks, gqb = row % H->total_qblocks;
+  const int b = reinterpret_cast<const int32_t*>(blob + H->off_qbseq)[gqb];
+  const DamSeq* seqs = blob_seqs(blob, H);
+  const DamSeq sq = seqs[b];
+  const DamSeq last = seqs[H->num_seqs - 1];
+  const uint64_t per_head = last.cnt_off + (causal ? (uint64_t)last.nq * (last.nq + 1) / 2 : (uint64_t)last.nq * last.nq);
+  const int qb = gqb - sq.first_qblock;
+  const int n = causal ? qb + 1 : sq.nq;
+  const uint64_t base = (uint64_t)h * per_head + sq.cnt_off + (causal ? (uint64_t)qb * (qb + 1) / 2 : (uint64_t)qb * sq.nq);
+  uint32_t* tile_ptr = reinterpret_cast<uint32_t*>(blob + H->off_tile_ptr);
+  uint32_t* tiles = reinterpret_cast<uint32_t*>(blob + H->off_tiles);
+  for (int k = lane; k < n; k += 32) tiles[base + k] = (uint32_t)k | (DAM_KIND_FULL << 28);
+  if (lane == 0) {
+    tile_ptr[row] = (uint32_t)base;
+    // heaviest q-blocks first (exact longest-first for one sequence)
+    reinterpret_cast<uint32_t*>(blob + H->off_work)[(uint64_t)h * H->total_qblocks + (H->total_qblocks - 1 - gqb)] = row;
+    if (row == H->rows - 1) {
+      uint32_t tot = (uint32_t)(base + n);
+      tile_ptr[H->rows] = tot;
+      H->total_tiles = tot;
+      H->full_tiles = tot;
+      H->bytes_used = H->off_tiles + 4ull * tot;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Test hook: rows of the mask as the attention kernels see them.
+// ---------------------------------------------------------------------------------------------
+__global__ void expand_rows_kernel(const unsigned char* blob, int seq, int head, int row_begin, int nrows, int words,
+                                   int causal, uint32_t* __restrict__ out) {
+  const DamHeader* H = reinterpret_cast<const DamHeader*>(blob);
+  const DamSeq sq = blob_seqs(blob, H)[seq];
+  const int a = blockIdx.x;
+  if (a >= nrows) return;
+  const int i = row_begin + a;
+  uint32_t* o = out + (size_t)a * words;
+  for (int w = threadIdx.x; w < words; w += blockDim.x) o[w] = 0u;
+  __syncthreads();
+  if (i < 0 || i >= sq.S) return;
+  const int qb = i / DAM_TILE;
+  const int row = head * H->total_qblocks + sq.first_qblock + qb;
+  const uint32_t* tile_ptr = reinterpret_cast<const uint32_t*>(blob + H->off_tile_ptr);
+  const uint32_t* tiles = reinterpret_cast<const uint32_t*>(blob + H->off_tiles);
+  DamHeadBits hb = dam_head_bits(blob, H, sq, head);
+  for (uint32_t t = tile_ptr[row] + threadIdx.x; t < tile_ptr[row + 1]; t += blockDim.x) {
+    uint32_t e = tiles[t];
+    int kb = (int)(e & 0x0FFFFFFFu);
+    uint4 bits = dam_apply_bits(hb, e >> 28, i, kb, causal);
+    if (kb * 4 + 3 < words) {
+      o[kb * 4 + 0] = bits.x; o[kb * 4 + 1] = bits.y; o[kb * 4 + 2] = bits.z; o[kb * 4 + 3] = bits.w;
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t dam_launch_init_blob(const dam_shape_t* shape, int pcl_max, uint32_t flags, void* blob,
+                                 uint32_t tile_capacity, const DamHeader& host_hdr, cudaStream_t st) {
+  (void)tile_capacity;
+  int mode = (flags & DAM_FLAG_ALL_ONES) ? ((flags & DAM_FLAG_CAUSAL_LIST) ? 1 : 0) : -1;
+  init_blob_kernel<<<1, 256, 0, st>>>(reinterpret_cast<unsigned char*>(blob), host_hdr, shape->cu_seqlens_dev,
+                                      pcl_max, shape->num_q_heads, mode);
+  return cudaGetLastError();
+}
+
+cudaError_t dam_launch_bits_from_scores(const float* P, const DamBuildCtx& c, cudaStream_t st) {
+  if (c.max_L == 0) return cudaSuccess;
+  long long items = (long long)c.max_L * c.max_W;
+  int bx = (int)((items + 7) / 8);
+  if (bx > 4096) bx = 4096;
+  dim3 grid(bx, c.num_seqs * c.Hq);
+  bits_from_scores_kernel<<<grid, 256, 0, st>>>(c.blob, P, c.pstar);
+  return cudaGetLastError();
+}
+
+cudaError_t dam_launch_rule(const DamBuildCtx& c, cudaStream_t st) {
+  cudaError_t e;
+  // counters start at zero: counts + prefix + tile popcounts, row counts, histogram, cursors
+  if ((e = cudaMemsetAsync(c.scratch + c.off_cnt, 0, c.off_rowstat - c.off_cnt, st)) != cudaSuccess) return e;
+  if ((e = cudaMemsetAsync(c.scratch + c.off_hist, 0, 2ull * DAM_HIST * 4, st)) != cudaSuccess) return e;
+  if (c.max_nL > 0) {
+    dim3 g(c.max_nL * (c.max_nL + 1) / 2, c.num_seqs * c.Hq);
+    counts_kernel<<<g, DAM_TILE, 0, st>>>(c.blob, c.scratch, c.off_cnt);
+    match_kernel<<<c.num_seqs * c.Hq, 256, 0, st>>>(c.blob, c.scratch, c.off_cnt, c.mu, c.min_support);
+  }
+  if (c.rows > 0) {
+    int blocks = (c.rows + 7) / 8;
+    classify_kernel<0><<<blocks, 256, 0, st>>>(c.blob, c.scratch, c.off_cnt, c.off_rowcnt, c.off_hist, c.off_cursor);
+    scan_kernel<<<1, 1024, 0, st>>>(c.blob, c.scratch, c.off_rowcnt, c.off_hist, c.off_cursor);
+    classify_kernel<1><<<blocks, 256, 0, st>>>(c.blob, c.scratch, c.off_cnt, c.off_rowcnt, c.off_hist, c.off_cursor);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t dam_launch_all_ones(const dam_shape_t* shape, int causal, void* blob, cudaStream_t st) {
+  int rows = 0;
+  for (int b = 0; b < shape->num_seqs; ++b)
+    rows += (shape->cu_seqlens_host[b + 1] - shape->cu_seqlens_host[b] + DAM_TILE - 1) / DAM_TILE;
+  rows *= shape->num_q_heads;
+  if (rows == 0) return cudaSuccess;
+  all_ones_kernel<<<(rows + 7) / 8, 256, 0, st>>>(reinterpret_cast<unsigned char*>(blob), causal);
+  return cudaGetLastError();
+}
+
+cudaError_t dam_launch_expand_rows(const void* blob, int seq, int head, int row_begin, int nrows, int words,
+                                   int causal, uint32_t* out, cudaStream_t st) {
+  expand_rows_kernel<<<nrows, 128, 0, st>>>(reinterpret_cast<const unsigned char*>(blob), seq, head, row_begin, nrows,
+                                            words, causal, out);
+  return cudaGetLastError();
+}

@@ -1,0 +1,124 @@
+"""Stage-2 parity on the GPU, through the C ABI: with an identical mask, O and LSE must match the
+float64 oracle within max-abs 2e-2 / mean-abs 2e-3 (bf16 in, fp32 accumulate) and 1e-3 for LSE."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2506_11104_b200 import binding as B
+from paper_2506_11104_b200 import synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+TOL = {torch.bfloat16: (2e-2, 2e-3, 1e-3), torch.float32: (1e-4, 1e-5, 1e-5)}
+
+
+def _shape(w):
+    return B.make_shape(w.cu_seqlens, w.num_q_heads, w.num_kv_heads, w.head_dim, w.Q.dtype, DEV)
+
+
+def _run(w, blob, shape, causal=True):
+    Q, K, V = w.Q.to(DEV), w.K.to(DEV), w.V.to(DEV)
+    O, lse, scratch = B.dam_sparse_attention(Q, K, V, blob, shape, causal=causal)
+    assert B.dam_poll_status(scratch) == 0
+    return O, lse
+
+
+def _check(w, O, lse, masks, rows_for, heads=None, causal=True, all_ones=False):
+    mx, mn, le = TOL[w.Q.dtype]
+    worst = [0.0, 0.0, 0.0]
+    for b in range(len(w.cu_seqlens) - 1):
+        S = w.cu_seqlens[b + 1] - w.cu_seqlens[b]
+        if S == 0:
+            continue
+        for h in (heads if heads is not None else range(w.num_q_heads)):
+            e = H.attention_errors(O, lse, w, masks, b, h, rows_for(S), causal=causal, all_ones=all_ones)
+            worst = [max(a, c) for a, c in zip(worst, e)]
+    assert worst[0] <= mx and worst[1] <= mn and worst[2] <= le, worst
+    return worst
+
+
+def _all_rows(S):
+    return list(range(S))
+
+
+def _sample_rows(L):
+    def f(S, L=L):
+        rng = np.random.default_rng(S)
+        fixed = [0, L - 1, L, L + 1, 2 * L - 2, 2 * L - 1, S - 1, 127, 128, S - 129]
+        rows = set(r for r in fixed if 0 <= r < S) | set(int(x) for x in rng.choice(S, size=min(S, 40), replace=False))
+        return sorted(rows)
+    return f
+
+
+@pytest.mark.parametrize("lengths,Hq,Hkv,d,dtype,causal", [
+    ([512], 2, 2, 64, torch.float32, True),
+    ([300, 77, 129], 4, 2, 64, torch.bfloat16, True),
+    ([200], 2, 1, 32, torch.float32, False),
+    ([640], 4, 1, 128, torch.bfloat16, True),
+    ([257, 1, 500], 8, 2, 128, torch.bfloat16, True),
+    ([384], 2, 2, 128, torch.bfloat16, False),
+])
+def test_all_ones_mask_is_dense_attention(lengths, Hq, Hkv, d, dtype, causal):
+    w = synth.small_case(0, Hq, Hkv, d, 64, seed=7, dtype=dtype, lengths=lengths, amp=3.0)
+    shape = _shape(w)
+    blob = B.dam_mask_all_ones(shape, causal, DEV)
+    O, lse = _run(w, blob, shape, causal=causal)
+    _check(w, O, lse, None, _all_rows, causal=causal, all_ones=True)
+
+
+def _masked_case(w, rows_for, heads=None):
+    shape = _shape(w)
+    rule = B.make_rule(w.pcl_max, w.tau, w.mu, w.lam, w.eps)
+    n = sum(w.num_q_heads * min(S, w.pcl_max) ** 2 for S in shape.lengths)
+    dump = torch.zeros(n, dtype=torch.float32, device=DEV)
+    blob, _ = B.dam_build_masks(w.Q.to(DEV), w.K.to(DEV), shape, rule, scores_dump=dump)
+    assert B.dam_poll_status(blob) == 0
+    masks = H.oracle_masks_from_dump(w, dump.cpu().numpy())      # identical mask on both sides
+    O, lse = _run(w, blob, shape)
+    worst = _check(w, O, lse, masks, rows_for, heads=heads)
+    return blob, shape, masks, O, lse, worst
+
+
+def test_config0_every_row():
+    w = synth.config0()
+    blob, shape, masks, O, lse, worst = _masked_case(w, _all_rows)
+    # rows below the window with no matched pattern are empty: O = 0, LSE = -inf (checked inside)
+    assert torch.isfinite(O).all()
+
+
+@pytest.mark.parametrize("lengths,pcl,Hq,Hkv,d,dtype", [
+    ([700], 256, 4, 2, 128, torch.bfloat16),
+    ([333, 1000, 64], 200, 4, 1, 64, torch.bfloat16),
+    ([1500, 130], 256, 8, 2, 128, torch.bfloat16),
+    ([513], 300, 2, 2, 32, torch.float32),
+])
+def test_masked_small_cases_every_row(lengths, pcl, Hq, Hkv, d, dtype):
+    w = synth.small_case(0, Hq, Hkv, d, pcl, seed=11, dtype=dtype, lengths=lengths)
+    _masked_case(w, _all_rows)
+
+
+def test_empty_rows_and_no_patterns():
+    """mu > 1: nothing matches, every row below the window is empty."""
+    w = synth.small_case(0, 4, 2, 128, 128, seed=5, lengths=[600])
+    w.mu = 1.5
+    blob, shape, masks, O, lse, _ = _masked_case(w, _all_rows)
+    assert torch.isneginf(lse[:, 128:]).all() and (O[128:] == 0).all()
+
+
+def test_config1_sampled_rows():
+    w = synth.config1()
+    _masked_case(w, _sample_rows(1024), heads=[0, 5, 13, 22, 31])
+
+
+def test_config1_dense_causal_sampled_rows():
+    w = synth.config1()
+    shape = _shape(w)
+    blob = B.dam_mask_all_ones(shape, True, DEV)
+    O, lse = _run(w, blob, shape)
+    _check(w, O, lse, None, lambda S: [0, 1, 127, 128, 4095, 8191], heads=[3, 30], all_ones=True)
+
+
+def test_config4_varlen_sampled_rows():
+    w = synth.config4()
+    _masked_case(w, _sample_rows(1024), heads=[2, 17])

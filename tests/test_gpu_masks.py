@@ -1,0 +1,187 @@
+"""Stage-1 parity on the GPU, through the C ABI: masks must equal the oracle's bit for bit when both
+start from the same fp32 score tensor."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import dam_oracle as orc
+from paper_2506_11104_b200 import binding as B
+from paper_2506_11104_b200 import synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _shape(w):
+    return B.make_shape(w.cu_seqlens, w.num_q_heads, w.num_kv_heads, w.head_dim, w.Q.dtype, DEV)
+
+
+def _rule(w, **kw):
+    return B.make_rule(w.pcl_max, w.tau, w.mu, w.lam, w.eps, **kw)
+
+
+def _band(L, wdt):
+    i, j = np.indices((L, L))
+    return ((i - j >= 0) & (i - j < wdt)).astype(np.float32)
+
+
+def _from_scores_case(lengths, Hq, pcl, P_list, tau, mu, min_support=1):
+    cu = np.concatenate([[0], np.cumsum(lengths)]).tolist()
+    shape = B.make_shape(cu, Hq, Hq, 64, torch.float32, DEV)
+    rule = B.make_rule(pcl, tau, mu, min_support=min_support)
+    flat = np.concatenate([p.reshape(-1) for per in P_list for p in per]).astype(np.float32)
+    blob, _ = B.dam_build_masks_from_scores(torch.from_numpy(flat).to(DEV), shape, rule)
+    assert B.dam_poll_status(blob) == 0
+    masks = [[orc.head_mask_from_probs(np.ascontiguousarray(P_list[b][h]), S, tau, mu, min_support=min_support)
+              for h in range(Hq)] for b, S in enumerate(lengths)]
+    n = H.check_blob_against_oracle(blob, shape, masks)
+    return blob, shape, masks, n
+
+
+def test_injected_band_sink_and_ties():
+    """Closed-form score tensors: a band, a sink column, random lower-triangular noise, an exact tie."""
+    L = 256
+    rng = np.random.default_rng(0)
+    sink = np.zeros((L, L), np.float32)
+    sink[:, 0] = 1.0
+    noise = np.tril(rng.random((L, L)) * 0.05).astype(np.float32)
+    tie = np.zeros((L, L), np.float32)
+    r, need = 56, int(np.ceil(0.8 * (L - 56)))
+    for t in range(need):
+        tie[r + t, t] = 1.0
+    P = [[_band(L, 32), sink, noise, tie]]
+    blob, shape, masks, n = _from_scores_case([1000], 4, L, P, 0.3, 0.8)
+    assert n > 0
+    assert np.flatnonzero(masks[0][0].V).tolist() == list(range(L - 40, L))     # last floor(32 / 0.8) columns
+    assert masks[0][3].D[r] == 1
+
+
+@pytest.mark.parametrize("lengths,pcl", [([300], 200), ([129, 1, 640, 77], 130), ([2048], 512), ([100], 256)])
+def test_ragged_lengths_random_scores(lengths, pcl):
+    """Windows and sequences that are not multiples of the tile or word size, several sequences, S <= L."""
+    rng = np.random.default_rng(sum(lengths))
+    Hq = 3
+    P = []
+    for S in lengths:
+        L = min(S, pcl)
+        per = []
+        for h in range(Hq):
+            p = np.tril(rng.random((L, L)) * 0.04).astype(np.float32)
+            p += _band(L, 3 + 17 * h) * 0.5
+            p[:, min(5, L - 1)] = 1.0
+            per.append(np.tril(p).astype(np.float32))
+        P.append(per)
+    _from_scores_case(lengths, Hq, pcl, P, 0.3, 0.8)
+
+
+def test_wide_band_gives_full_tiles_and_mu_extremes():
+    L, S = 512, 2000
+    P = [[_band(L, 400), _band(L, 400)]]
+    blob, shape, masks, _ = _from_scores_case([S], 2, L, P, 0.3, 0.8)
+    st = B.dam_mask_stats(blob, shape)
+    assert st["full_tiles"] > 0 and st["tiles"] > st["full_tiles"]
+    # mu <= 0: every pattern matches; mu > 1: none
+    _from_scores_case([S], 2, L, P, 0.3, 0.0)
+    b2, s2, m2, _ = _from_scores_case([S], 2, L, P, 0.3, 1.5)
+    assert not m2[0][0].D.any()
+    _from_scores_case([S], 2, L, P, 0.3, 0.8, min_support=50)
+
+
+def test_threshold_boundary_values_bit_exact():
+    """Score values packed around the flip point of the fp32 threshold chain, for several tau."""
+    L = 128
+    for tau in (0.3, 0.1, 0.05, 0.02):
+        centre = np.float32((tau / 2 + 1e-4) ** 2)
+        bits = centre.view(np.uint32).astype(np.int64) + np.arange(-L * L // 2, L * L // 2)
+        P = np.tril(bits.astype(np.uint32).view(np.float32).reshape(L, L)).astype(np.float32)
+        _from_scores_case([L], 1, L, [[P]], tau, 0.8)
+
+
+def _build_and_check(w, qblocks=None):
+    shape, rule = _shape(w), _rule(w)
+    Q, K = w.Q.to(DEV), w.K.to(DEV)
+    lengths = shape.lengths
+    n = sum(w.num_q_heads * min(S, w.pcl_max) ** 2 for S in lengths)
+    dump = torch.zeros(n, dtype=torch.float32, device=DEV)
+    blob, _ = B.dam_build_masks(Q, K, shape, rule, scores_dump=dump)
+    assert B.dam_poll_status(blob) == 0
+    masks = H.oracle_masks_from_dump(w, dump.cpu().numpy())
+    H.check_blob_against_oracle(blob, shape, masks, qblocks_per_head=qblocks)
+    # a second build without the dump gives the identical blob (dump does not change decisions; deterministic)
+    blob2, _ = B.dam_build_masks(Q, K, shape, rule)
+    used = B.dam_mask_stats(blob, shape)["bytes_used"]
+    mb1, mb2 = B.MaskBlob(blob), B.MaskBlob(blob2)
+    assert mb1.raw[256:int(mb1.hdr["off_work"])] == mb2.raw[256:int(mb2.hdr["off_work"])]
+    assert mb1.tiles.tobytes() == mb2.tiles.tobytes() and used == int(mb2.hdr["bytes_used"])
+    assert sorted(mb1.work.tolist()) == list(range(int(mb1.hdr["rows"])))
+    return blob, shape, masks, dump
+
+
+def _score_closeness(w, dump, masks, heads):
+    """GPU fp32 map vs the float64 map; every cell whose decision differs must sit within 2 % of p*."""
+    Q, K = H.to_f32_numpy(w.Q), H.to_f32_numpy(w.K)
+    P = H.split_dump(dump.cpu().numpy(), [b - a for a, b in zip(w.cu_seqlens[:-1], w.cu_seqlens[1:])],
+                     w.num_q_heads, w.pcl_max)
+    g = w.num_q_heads // w.num_kv_heads
+    pstar = (w.tau / 2 + np.sqrt(w.eps)) ** 2
+    flipped = total = 0
+    for b in range(len(w.cu_seqlens) - 1):
+        t0, t1 = w.cu_seqlens[b], w.cu_seqlens[b + 1]
+        L = min(t1 - t0, w.pcl_max)
+        for h in heads:
+            P64 = orc.window_probs(Q[t0:t1, h], K[t0:t1, h // g], L, 1 / np.sqrt(w.head_dim))
+            assert np.abs(P[b][h] - P64).max() < 2e-5
+            M64 = orc.true_mask_f64(P64, w.tau, w.lam, w.eps)
+            diff = M64 != masks[b][h].M
+            flipped += int(diff.sum())
+            total += L * (L + 1) // 2
+            if diff.any():
+                assert np.all(np.abs(P64[diff] - pstar) <= 0.02 * pstar)
+    return flipped, total
+
+
+def test_config0_full():
+    w = synth.config0()
+    blob, shape, masks, dump = _build_and_check(w)
+    flipped, total = _score_closeness(w, dump, masks, range(w.num_q_heads))
+    assert flipped <= 1e-3 * total
+    # planted structure is recovered
+    assert masks[0][0].V[0] == 1 and masks[0][0].D[:8].all()
+    assert all(masks[0][1].V[p] for p in w.plans[0][1].stripes)
+
+
+@pytest.mark.parametrize("lengths,pcl,Hq,Hkv,d,dtype", [
+    ([700], 256, 4, 2, 128, torch.bfloat16),
+    ([333, 1000, 64], 200, 4, 1, 64, torch.bfloat16),
+    ([513], 300, 2, 2, 32, torch.float32),
+])
+def test_small_cases_scored_on_gpu(lengths, pcl, Hq, Hkv, d, dtype):
+    w = synth.small_case(0, Hq, Hkv, d, pcl, seed=len(lengths), dtype=dtype, lengths=lengths)
+    blob, shape, masks, dump = _build_and_check(w)
+    flipped, total = _score_closeness(w, dump, masks, range(Hq))
+    assert flipped <= 2e-3 * total
+
+
+def test_config1_full_size_masks():
+    """Llama-3-8B-shaped layer, 8192 tokens, PCL 1024: every head's D, V and true mask, sampled q-blocks."""
+    w = synth.config1()
+    blob, shape, masks, dump = _build_and_check(w, qblocks=12)
+    flipped, total = _score_closeness(w, dump, masks, [0, 9, 31])
+    assert flipped <= 1e-3 * total
+    st = B.dam_mask_stats(blob, shape)
+    assert 0.03 <= st["tiles"] / st["causal_tiles"] <= 0.45
+
+
+def test_config4_varlen_masks():
+    w = synth.config4(lengths=(4096, 16384, 32768, 65536))
+    _build_and_check(w, qblocks=8)
+
+
+def test_config3_shape_masks():
+    """131072 tokens, PCL 4096 (config 3): all heads' pattern bits and true masks, sampled q-blocks."""
+    w = synth.config3(device=DEV)
+    w.Q, w.K, w.V = w.Q.cpu(), w.K.cpu(), w.V.cpu()
+    blob, shape, masks, dump = _build_and_check(w, qblocks=8)
+    st = B.dam_mask_stats(blob, shape)
+    assert 0.005 <= st["tiles"] / st["causal_tiles"] <= 0.08
