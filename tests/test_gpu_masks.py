@@ -112,8 +112,12 @@ def _build_and_check(w, qblocks=None):
     blob2, _ = B.dam_build_masks(Q, K, shape, rule)
     used = B.dam_mask_stats(blob, shape)["bytes_used"]
     mb1, mb2 = B.MaskBlob(blob), B.MaskBlob(blob2)
-    assert mb1.raw[256:int(mb1.hdr["off_work"])] == mb2.raw[256:int(mb2.hdr["off_work"])]
+    assert mb1.seqs.tobytes() == mb2.seqs.tobytes() and mb1.tile_ptr.tobytes() == mb2.tile_ptr.tobytes()
     assert mb1.tiles.tobytes() == mb2.tiles.tobytes() and used == int(mb2.hdr["bytes_used"])
+    for b in range(len(lengths)):
+        for h in range(0, w.num_q_heads, max(1, w.num_q_heads // 4)):
+            assert all(np.array_equal(x, y) for x, y in zip(mb1.pattern_bits(b, h), mb2.pattern_bits(b, h)))
+            assert np.array_equal(mb1.true_mask(b, h), mb2.true_mask(b, h))
     assert sorted(mb1.work.tolist()) == list(range(int(mb1.hdr["rows"])))
     return blob, shape, masks, dump
 
