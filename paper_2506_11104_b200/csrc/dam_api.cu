@@ -167,6 +167,7 @@ dam_status_t fill_ctx(const dam_shape_t* s, const dam_rule_t* r, void* mask, siz
   c->scale = r->softmax_scale > 0.f ? r->softmax_scale : 1.0f / sqrtf((float)s->head_dim);
   c->off_cnt = y->off_cnt; c->off_rowstat = y->off_rowstat; c->off_rowcnt = y->off_rowcnt;
   c->off_hist = y->off_hist; c->off_cursor = y->off_cursor;
+  c->off_true = y->hdr.off_true; c->true_bytes = y->hdr.off_tile_ptr - y->hdr.off_true;
   return DAM_OK;
 }
 

@@ -167,6 +167,7 @@ struct DamBuildCtx {
   int min_support;
   float scale;
   uint64_t off_cnt, off_rowstat, off_rowcnt, off_hist, off_cursor;   // scratch sections
+  uint64_t off_true, true_bytes;                                     // true-mask section of the blob
 };
 
 cudaError_t dam_launch_init_blob(const dam_shape_t* shape, int pcl_max, uint32_t flags, void* blob,

@@ -1,3 +1,294 @@
+// Window scoring on the 5th-generation tensor cores (sm_100a): bf16 inputs, head_dim 128.
+//
+// For every (sequence, query head) the causal softmax map over the first L tokens is computed tile by
+// tile and thresholded straight into the bit-packed true mask (paper Sec. 4.2.1 - 4.2.3); the map itself
+// is never stored unless the caller asks for the fp32 dump.  A work item is one 128-row query block of
+// one (sequence, head).  Two sweeps over its kv tiles kb = 0 .. qb:
+//   sweep A  S = Q K^T (tcgen05, accumulator in TMEM) -> per-row running max and sum;
+//   sweep B  S again -> p = exp2(x - max) / sum in fp32 -> bit = [p >= p*] -> one 16-byte store of the
+//            row's 128 bits per tile (and the optional dump of p).
+// Warp roles as in the attention kernel: warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 one thread
+// per query row.  Every wait is bounded.
+#include <cuda_bf16.h>
+#include <math_constants.h>
+
 #include "dam_internal.cuh"
-cudaError_t dam_launch_scores_sm100(const void*, const void*, const dam_shape_t*, const DamBuildCtx&, float*,
-                                    cudaStream_t) { return cudaErrorNotSupported; }
+#include "sm100_ptx.cuh"
+
+using namespace sm100;
+
+namespace {
+
+constexpr int kSlots = 5;
+constexpr int kSlotBytes = 32768;
+constexpr int kThreads = 192;
+constexpr uint32_t kTmemCols = 256;
+
+struct SmemLayout {
+  static constexpr int q = 0;
+  static constexpr int slots = kSlotBytes;
+  static constexpr int bars = kSlotBytes * (1 + kSlots);
+  // q_full, q_empty, slot_full[kSlots], slot_empty[kSlots], s_full[2], s_empty[2]
+  static constexpr int n_bars = 2 + 2 * kSlots + 4;
+  static constexpr int tmem_slot = bars + 8 * n_bars;
+  static constexpr int abort_flag = tmem_slot + 4;
+  static constexpr int total = abort_flag + 4;
+};
+constexpr int kSmemBytes = SmemLayout::total + 1024;
+
+struct ScoreParams {
+  unsigned char* blob;
+  float* dump;
+  uint32_t* status;
+  int num_seqs, Hq, group, max_nL;
+  float scale_log2, pstar;
+};
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm volatile("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+struct Item { int b, h, qb, valid; DamSeq sq; };
+
+__device__ __forceinline__ Item decode_item(const unsigned char* blob, const DamHeader* H, const ScoreParams& p, int w) {
+  Item it;
+  const int per = p.num_seqs * p.Hq;
+  it.qb = p.max_nL - 1 - w / per;           // heaviest query blocks first
+  const int sh = w % per;
+  it.b = sh / p.Hq; it.h = sh % p.Hq;
+  it.sq = reinterpret_cast<const DamSeq*>(blob + H->off_seq)[it.b];
+  it.valid = it.qb < it.sq.nL;
+  return it;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                   const ScoreParams prm) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t sbase = smem_u32(smem);
+  const uint32_t sQ = sbase + SmemLayout::q;
+  const uint32_t sSlots = sbase + SmemLayout::slots;
+  const uint32_t bar0 = sbase + SmemLayout::bars;
+  const uint32_t bQFull = bar0, bQEmpty = bar0 + 8;
+  const uint32_t bSlotFull = bar0 + 16, bSlotEmpty = bSlotFull + 8 * kSlots;
+  const uint32_t bSFull = bSlotEmpty + 8 * kSlots, bSEmpty = bSFull + 16;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + SmemLayout::tmem_slot);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + SmemLayout::abort_flag);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  unsigned char* blob = prm.blob;
+  const DamHeader* H = reinterpret_cast<const DamHeader*>(blob);
+  const int nitems = prm.max_nL * prm.num_seqs * prm.Hq;
+
+  if (tid == 0) {
+    mbar_init(bQFull, 1); mbar_init(bQEmpty, 1);
+    for (int s = 0; s < kSlots; ++s) { mbar_init(bSlotFull + 8 * s, 1); mbar_init(bSlotEmpty + 8 * s, 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(bSFull + 8 * s, 1); mbar_init(bSEmpty + 8 * s, 128); }
+    *abort_flag = 0u;
+    mbar_fence_init();
+    tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK);
+  }
+  if (warp == 0) { tmem_alloc(smem_u32(tmem_slot), kTmemCols); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      uint32_t sc = 0, ic = 0;
+      uint32_t armed[kSlots];
+#pragma unroll
+      for (int s = 0; s < kSlots; ++s) armed[s] = 2u;
+      bool ok = true;
+      for (int w = blockIdx.x; w < nitems && ok; w += gridDim.x) {
+        const Item it = decode_item(blob, H, prm, w);
+        if (!it.valid) continue;
+        if (!(ok = mbar_wait(bQEmpty, (ic & 1u) ^ 1u, abort_flag))) break;
+        mbar_arrive_expect_tx(bQFull, kSlotBytes);
+        const int tokq = it.sq.tok_start + it.qb * DAM_TILE;
+        tma_load_3d(sQ, &tmQ, bQFull, 0, it.h, tokq);
+        tma_load_3d(sQ + 16384, &tmQ, bQFull, 64, it.h, tokq);
+        ++ic;
+        const int kvh = it.h / prm.group;
+        const int n = 2 * (it.qb + 1);
+        for (int t = 0; t < n && ok; ++t) {
+          const int kb = t % (it.qb + 1);
+          const uint32_t s = sc % kSlots, ph = (sc / kSlots) & 1u;
+          if (!(ok = mbar_wait(bSlotEmpty + 8 * s, ph ^ 1u, abort_flag))) break;
+          const uint32_t dst = sSlots + s * kSlotBytes, bar = bSlotFull + 8 * s;
+          mbar_arrive_expect_tx(bar, kSlotBytes);
+          tma_load_3d(dst, &tmK, bar, 0, kvh, it.sq.tok_start + kb * DAM_TILE);
+          tma_load_3d(dst + 16384, &tmK, bar, 64, kvh, it.sq.tok_start + kb * DAM_TILE);
+          armed[s] = ph;
+          ++sc;
+        }
+      }
+      if (!ok) {
+        uint32_t dummy = 0;
+        for (int s = 0; s < kSlots; ++s)
+          if (armed[s] != 2u) mbar_wait(bSlotFull + 8 * s, armed[s], &dummy, 20000000ull);
+        mbar_wait(bQFull, (ic + 1u) & 1u, &dummy, 20000000ull);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = idesc_bf16_f32(128, 128, 0);
+      uint32_t sc = 0, ic = 0, g = 0;
+      bool ok = true;
+      for (int w = blockIdx.x; w < nitems && ok; w += gridDim.x) {
+        const Item it = decode_item(blob, H, prm, w);
+        if (!it.valid) continue;
+        if (!(ok = mbar_wait(bQFull, ic & 1u, abort_flag))) break;
+        ++ic;
+        const int n = 2 * (it.qb + 1);
+        for (int t = 0; t < n && ok; ++t, ++g, ++sc) {
+          const uint32_t buf = g & 1u, s = sc % kSlots;
+          if (!(ok = mbar_wait(bSEmpty + 8 * buf, ((g >> 1) & 1u) ^ 1u, abort_flag))) break;
+          if (!(ok = mbar_wait(bSlotFull + 8 * s, (sc / kSlots) & 1u, abort_flag))) break;
+          tc_fence_after();
+          const uint32_t kaddr = sSlots + s * kSlotBytes;
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks) {
+            const uint32_t off = (ks >> 2) * 16384 + (ks & 3) * 32;
+            mma_ss(tmem + buf * 128, smem_desc_sw128(sQ + off, 16, 1024), smem_desc_sw128(kaddr + off, 16, 1024), idesc,
+                   ks > 0 ? 1u : 0u);
+          }
+          tc_commit(bSlotEmpty + 8 * s);
+          tc_commit(bSFull + 8 * buf);
+          if (t + 1 == n) tc_commit(bQEmpty);
+        }
+      }
+    }
+  } else {
+    const int r = (warp & 3) * 32 + lane;
+    const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+    uint32_t g = 0;
+    bool ok = true;
+    for (int w = blockIdx.x; w < nitems && ok; w += gridDim.x) {
+      const Item it = decode_item(blob, H, prm, w);
+      if (!it.valid) continue;
+      const int L = it.sq.L, W = it.sq.W;
+      const int i = it.qb * DAM_TILE + r;
+      const bool row_valid = i < L;
+      uint32_t* Mrow = reinterpret_cast<uint32_t*>(blob + H->off_true) + it.sq.true_off + (uint64_t)it.h * L * W + (size_t)i * W;
+      float* Prow = prm.dump ? prm.dump + it.sq.p_off + (uint64_t)it.h * L * L + (size_t)i * L : nullptr;
+      float m = -CUDART_INF_F, l = 0.f, inv_l = 0.f;
+      const int nk = it.qb + 1;
+      for (int t = 0; t < 2 * nk; ++t, ++g) {
+        const int kb = t % nk;
+        const bool sweepB = t >= nk;
+        const uint32_t buf = g & 1u;
+        if (!(ok = mbar_wait(bSFull + 8 * buf, (g >> 1) & 1u, abort_flag))) break;
+        tc_fence_after();
+        // keys beyond the causal limit (and beyond the window, which the limit implies) do not exist
+        const int nvalid = min(DAM_TILE, i - kb * DAM_TILE + 1);
+        if (t == nk) inv_l = l > 0.f ? 1.0f / l : 0.f;
+        uint4 words = make_uint4(0u, 0u, 0u, 0u);
+        float tmax = -CUDART_INF_F, tsum = 0.f;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t rr[32];
+          tmem_ld32(tmem + lane_addr + buf * 128 + c * 32, rr);
+          tc_wait_ld();
+          if (!sweepB) {
+            float cm = -CUDART_INF_F;
+#pragma unroll
+            for (int q = 0; q < 32; ++q) {
+              float x = __uint_as_float(rr[q]) * prm.scale_log2;
+              x = (c * 32 + q < nvalid) ? x : -CUDART_INF_F;
+              rr[q] = __float_as_uint(x);
+              cm = fmaxf(cm, x);
+            }
+            const float mn = fmaxf(tmax, cm);
+            if (mn > -CUDART_INF_F) {
+              float cs = 0.f;
+#pragma unroll
+              for (int q = 0; q < 32; ++q) cs += ex2(__uint_as_float(rr[q]) - mn);
+              tsum = tsum * ex2(tmax - mn) + cs;     // tmax = -inf gives a factor 0
+              tmax = mn;
+            }
+          } else {
+            uint32_t word = 0u;
+#pragma unroll
+            for (int q = 0; q < 32; ++q) {
+              float x = __uint_as_float(rr[q]) * prm.scale_log2;
+              float p = (c * 32 + q < nvalid) ? ex2(x - m) * inv_l : 0.f;
+              rr[q] = __float_as_uint(p);
+              word |= (p >= prm.pstar ? 1u : 0u) << q;
+            }
+            if (c == 0) words.x = word; else if (c == 1) words.y = word; else if (c == 2) words.z = word; else words.w = word;
+            if (Prow && row_valid) {
+              const int j0 = kb * DAM_TILE + c * 32;
+#pragma unroll
+              for (int q = 0; q < 32; ++q)
+                if (j0 + q < L) Prow[j0 + q] = __uint_as_float(rr[q]);
+            }
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(bSEmpty + 8 * buf);
+        if (!sweepB) {
+          if (tmax > -CUDART_INF_F) {
+            const float mn = fmaxf(m, tmax);
+            l = l * ex2(m - mn) + tsum * ex2(tmax - mn);
+            m = mn;
+          }
+        } else if (row_valid) {
+          *reinterpret_cast<uint4*>(Mrow + kb * 4) = words;
+        }
+      }
+      if (!ok) break;
+      // dump: zeros above the diagonal for the tiles this item does not visit
+      if (Prow && row_valid)
+        for (int j = (it.qb + 1) * DAM_TILE; j < L; ++j) Prow[j] = 0.f;
+    }
+  }
+
+  if (*abort_flag && tid == 64) atomicMax(prm.status, (uint32_t)DAM_ERR_DEVICE_TIMEOUT);
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+}
+
+}  // namespace
+
+cudaError_t dam_launch_scores_sm100(const void* Q, const void* K, const dam_shape_t* s, const DamBuildCtx& c,
+                                    float* dump, cudaStream_t st) {
+  if (s->dtype != DAM_BF16 || s->head_dim != 128) return cudaErrorNotSupported;
+  if (c.max_nL == 0) return cudaSuccess;
+  static int sm_count = 0;
+  if (sm_count == 0) {
+    int dev = 0, cc_major = 0, smem_optin = 0;
+    cudaError_t e;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev);
+    cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (cc_major != 10 || smem_optin < kSmemBytes) return cudaErrorNotSupported;
+    if ((e = cudaFuncSetAttribute(score_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) != cudaSuccess)
+      return e;
+    cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+  }
+  CUtensorMap tq, tk;
+  if (!dam_make_tmap_bf16(&tq, Q, 128, s->num_q_heads, s->total_tokens, s->q_stride_tok, s->q_stride_head) ||
+      !dam_make_tmap_bf16(&tk, K, 128, s->num_kv_heads, s->total_tokens, s->k_stride_tok, s->k_stride_head))
+    return cudaErrorInvalidValue;
+  // the kernel writes only the tiles on or below the diagonal: everything else of the true mask is zero
+  if (c.true_bytes) {
+    cudaError_t e = cudaMemsetAsync(c.blob + c.off_true, 0, c.true_bytes, st);
+    if (e != cudaSuccess) return e;
+  }
+  ScoreParams p;
+  p.blob = c.blob; p.dump = dump;
+  p.status = reinterpret_cast<uint32_t*>(c.blob) + 1;
+  p.num_seqs = c.num_seqs; p.Hq = c.Hq; p.group = c.Hq / c.Hkv; p.max_nL = c.max_nL;
+  p.scale_log2 = c.scale * 1.4426950408889634f;
+  p.pstar = c.pstar;
+  const int items = c.max_nL * c.num_seqs * c.Hq;
+  const int grid = items < sm_count ? items : sm_count;
+  score_sm100_kernel<<<grid, kThreads, kSmemBytes, st>>>(tq, tk, p);
+  return cudaGetLastError();
+}
