@@ -244,10 +244,15 @@ _HDR = np.dtype([("magic", "<u4"), ("status", "<u4"), ("version", "<u4"), ("flag
                  ("tile_capacity", "<u4"), ("total_tiles", "<u4"), ("full_tiles", "<u4"), ("pcl_max", "<u4"),
                  ("off_seq", "<u8"), ("off_qbseq", "<u8"), ("off_dv", "<u8"), ("off_true", "<u8"),
                  ("off_tile_ptr", "<u8"), ("off_work", "<u8"), ("off_tiles", "<u8"), ("bytes_used", "<u8"),
-                 ("causal_tiles", "<u8"), ("reserved", "<u8", (17,))])
+                 ("causal_tiles", "<u8"), ("off_pairtab", "<u8"), ("total_pairs", "<i4"), ("prows", "<i4"),
+                 ("reserved", "<u8", (15,))])
 _SEQ = np.dtype([("tok_start", "<i4"), ("S", "<i4"), ("L", "<i4"), ("nq", "<i4"), ("first_qblock", "<i4"),
-                 ("W", "<i4"), ("nL", "<i4"), ("pad", "<i4"), ("dv_off", "<u8"), ("true_off", "<u8"),
+                 ("W", "<i4"), ("nL", "<i4"), ("first_pair", "<i4"), ("dv_off", "<u8"), ("true_off", "<u8"),
                  ("p_off", "<u8"), ("cnt_off", "<u8")])
+
+
+_ITEM = np.dtype([("head", "<i4"), ("tok0", "<i4"), ("qb0", "<i4"), ("S", "<i4"), ("a0", "<u4"), ("a1", "<u4"),
+                  ("b1", "<u4"), ("seq_hasB", "<u4")])
 
 
 def _unpack_bits(words: np.ndarray, n: int) -> np.ndarray:
@@ -269,7 +274,10 @@ class MaskBlob:
         self.seqs = np.frombuffer(self.raw, dtype=_SEQ, count=B, offset=int(self.hdr["off_seq"]))
         rows = int(self.hdr["rows"])
         self.tile_ptr = np.frombuffer(self.raw, dtype="<u4", count=rows + 1, offset=int(self.hdr["off_tile_ptr"]))
-        self.work = np.frombuffer(self.raw, dtype="<u4", count=rows, offset=int(self.hdr["off_work"]))
+        self.items = np.frombuffer(self.raw, dtype=_ITEM, count=int(self.hdr["prows"]),
+                                   offset=int(self.hdr["off_work"]))
+        self.pair_tab = np.frombuffer(self.raw, dtype="<u4", count=int(self.hdr["total_pairs"]),
+                                      offset=int(self.hdr["off_pairtab"]))
         self.tiles = np.frombuffer(self.raw, dtype="<u4", count=int(self.hdr["total_tiles"]),
                                    offset=int(self.hdr["off_tiles"]))
 

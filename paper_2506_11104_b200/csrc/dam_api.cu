@@ -58,7 +58,7 @@ void compute_layout(const dam_shape_t* s, int pcl_max, int all_ones_causal, Layo
   memset(&y, 0, sizeof(y));
   const int Hq = s->num_q_heads;
   uint64_t dv = 0, tr = 0, cnt = 0, cap = 0, causal_tiles = 0, lrows = 0, po = 0;
-  int total_qb = 0;
+  int total_qb = 0, total_pairs = 0;
   for (int b = 0; b < s->num_seqs; ++b) {
     int S = s->cu_seqlens_host[b + 1] - s->cu_seqlens_host[b];
     int L = S < pcl_max ? S : pcl_max;
@@ -77,6 +77,7 @@ void compute_layout(const dam_shape_t* s, int pcl_max, int all_ones_causal, Layo
       cap += (uint64_t)Hq * (all_ones_causal ? (uint64_t)nq * (nq + 1) / 2 : (uint64_t)nq * nq);
     }
     total_qb += nq;
+    total_pairs += (nq + 1) / 2;
     if (L > y.max_L) y.max_L = L;
     if (W > y.max_W) y.max_W = W;
     if (nL > y.max_nL) y.max_nL = nL;
@@ -91,15 +92,18 @@ void compute_layout(const dam_shape_t* s, int pcl_max, int all_ones_causal, Layo
   h.num_q_heads = Hq;
   h.total_qblocks = total_qb;
   h.rows = Hq * total_qb;
+  h.total_pairs = total_pairs;
+  h.prows = Hq * total_pairs;
   h.tile_capacity = (uint32_t)(cap > 0xFFFFFFF0ull ? 0xFFFFFFF0ull : cap);
   h.pcl_max = (uint32_t)pcl_max;
   h.off_seq = sizeof(DamHeader);
   h.off_qbseq = dam_align(h.off_seq + (uint64_t)s->num_seqs * sizeof(DamSeq), 256);
-  h.off_dv = dam_align(h.off_qbseq + 4ull * total_qb, 256);
+  h.off_pairtab = dam_align(h.off_qbseq + 4ull * total_qb, 256);
+  h.off_dv = dam_align(h.off_pairtab + 4ull * total_pairs, 256);
   h.off_true = dam_align(h.off_dv + 4ull * dv, 256);
   h.off_tile_ptr = dam_align(h.off_true + 4ull * tr, 256);
   h.off_work = dam_align(h.off_tile_ptr + 4ull * (h.rows + 1), 256);
-  h.off_tiles = dam_align(h.off_work + 4ull * h.rows, 256);
+  h.off_tiles = dam_align(h.off_work + (uint64_t)sizeof(DamItem) * h.prows, 256);
   h.causal_tiles = causal_tiles;
   y.mask_bytes = dam_align(h.off_tiles + 4ull * cap, 256);
   // build scratch: [0,256) reserved | counts | row stats (2 floats per window row) | row counts | hist | cursor
@@ -160,7 +164,7 @@ dam_status_t fill_ctx(const dam_shape_t* s, const dam_rule_t* r, void* mask, siz
   c->blob = reinterpret_cast<unsigned char*>(mask);
   c->scratch = reinterpret_cast<unsigned char*>(scratch);
   c->num_seqs = s->num_seqs; c->Hq = s->num_q_heads; c->Hkv = s->num_kv_heads; c->d = s->head_dim; c->dtype = s->dtype;
-  c->total_qblocks = y->hdr.total_qblocks; c->rows = y->hdr.rows;
+  c->total_qblocks = y->hdr.total_qblocks; c->rows = y->hdr.rows; c->prows = y->hdr.prows;
   c->max_L = y->max_L; c->max_W = y->max_W; c->max_nL = y->max_nL; c->max_nq = y->max_nq;
   c->pstar = find_pstar(r->tau, r->eps);
   c->mu = r->mu; c->min_support = r->min_support;

@@ -1,18 +1,21 @@
 // Sparse flash attention on the 5th-generation tensor cores (sm_100a): bf16 inputs, head_dim 128.
 //
-// One persistent CTA per SM walks the work list of the mask blob (rows = (head, 128-row query block),
-// longest tile list first).  Warp roles:
-//   warp 0      TMA producer: Q tile once per row, then the K / V tiles of the listed kv tiles into a
-//               ring of 32 KB shared-memory slots (128-byte swizzle, two 64-column boxes per tile);
-//   warp 1      MMA issuer (one elected thread): S = Q K^T into one of two TMEM buffers, then
-//               O += P V with P read from TMEM; completion is signalled with tcgen05.commit;
-//   warps 2-5   softmax: one thread per query row reads its S row from TMEM, applies the tile's mask
-//               bits where the tile is not fully active, keeps the running max / sum, writes P (bf16)
-//               back to TMEM, rescales O in TMEM when the running max moved by more than 2^8, and
-//               finally normalises and stores O and the log-sum-exp.
+// One persistent CTA per SM walks the work list of the mask blob.  A work item is a pair of adjacent
+// 128-row query blocks (2p, 2p+1) of one (sequence, head): two query tiles ("streams" A and B) share every
+// K / V tile that either of them lists, so a kv tile is brought into shared memory once per 256 query rows.
+// Warp roles:
+//   warp 0      TMA producer: both Q tiles once per item, then K and V of every kv tile in the union of
+//               the two tile lists into a ring of 32 KB shared-memory slots (128-byte swizzle);
+//   warp 1      MMA issuer (one elected thread): S_X = Q_X K^T into the stream's TMEM columns, then
+//               O_X += P_X V with P_X read from TMEM (it overwrites the first half of S_X); the two streams
+//               are interleaved so that one stream's softmax runs under the other stream's MMAs;
+//   warps 2-5   softmax of stream A, warps 6-9 of stream B: one thread per query row reads its S row from
+//               TMEM (twice: running max, then probabilities), applies the tile's mask bits where the tile
+//               is not fully active, writes P (bf16) back to TMEM, rescales O in TMEM when the running max
+//               moved by more than 2^8, and finally normalises and stores O and the log-sum-exp.
 // Only the tiles the mask lists are ever loaded or multiplied (paper Sec. 4.3: masked logits are -inf).
-// Every wait is bounded; an expired wait sets the status word in the scratch buffer and the CTA
-// drains and exits.
+// Every wait is bounded; an expired wait sets the status word in the scratch buffer and the CTA drains
+// and exits.
 #include <cuda_bf16.h>
 #include <math_constants.h>
 
@@ -23,28 +26,41 @@ using namespace sm100;
 
 namespace {
 
-constexpr int kSlots = 6;
+constexpr int kSlots = 4;
+constexpr int kStageBytes = 16384;   // per-stream staging of one 64-column half of the O tile
 constexpr int kSlotBytes = 32768;
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColS = 0;      // S buffers at columns 0 and 128
-constexpr uint32_t kColO = 256;    // O accumulator
-constexpr uint32_t kColP = 384;    // P buffers (bf16 pairs) at columns 384 and 448
+constexpr uint32_t kColS = 0;      // S_A at 0, S_B at 128 (P_X overwrites columns [0, 64) of S_X)
+constexpr uint32_t kColO = 256;    // O_A at 256, O_B at 384
 constexpr float kRescaleThreshold = 8.0f;
+constexpr uint32_t kNone = 0xFFFFFFFFu;
 
 struct SmemLayout {
-  static constexpr int q = 0;
-  static constexpr int slots = kSlotBytes;
-  static constexpr int bars = kSlotBytes * (1 + kSlots);
-  // barriers (8 bytes each): q_full, q_empty, slot_full[kSlots], slot_empty[kSlots], s_full[2], p_full[2], pv_done
-  static constexpr int n_bars = 2 + 2 * kSlots + 2 + 2 + 1;
+  static constexpr int q = 0;                           // Q_A, Q_B
+  static constexpr int slots = 2 * kSlotBytes;
+  static constexpr int stage = kSlotBytes * (2 + kSlots);           // two staging buffers (stream A, B)
+  static constexpr int bars = stage + 2 * kStageBytes;
+  // q_full, q_empty, slot_full[kSlots], slot_empty[kSlots], s_full[2], p_full[2], o_final[2]
+  static constexpr int n_bars = 2 + 2 * kSlots + 6;
   static constexpr int tmem_slot = bars + 8 * n_bars;
   static constexpr int abort_flag = tmem_slot + 4;
   static constexpr int total = abort_flag + 4;
 };
 constexpr int kSmemBytes = SmemLayout::total + 1024;   // + slack for the 1024-byte alignment
 
+#ifdef DAM_PROFILE
+#define PROF_DECL(n) long long prof_acc[n] = {0}; long long prof_t = clock64();
+#define PROF_LAP(k) { long long now_ = clock64(); prof_acc[k] += now_ - prof_t; prof_t = now_; }
+#define PROF_FLUSH(base, n) if (blockIdx.x == 0) { for (int q_ = 0; q_ < n; ++q_) prm.prof[(base) + q_] = (unsigned long long)prof_acc[q_]; }
+#else
+#define PROF_DECL(n)
+#define PROF_LAP(k)
+#define PROF_FLUSH(base, n)
+#endif
+
 struct AttnParams {
+  unsigned long long* prof;
   const unsigned char* blob;
   __nv_bfloat16* O;
   float* lse;
@@ -56,31 +72,177 @@ struct AttnParams {
 
 __device__ __forceinline__ float ex2(float x) {
   float y;
-  asm volatile("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
 
+// One work item: a pair of query blocks of one (sequence, head) and the tile-list ranges of both.
 struct Item {
-  int head, seq_tok0, qb, S;
-  uint32_t t0, nt;
+  int head, tok0, qb0, S, hasB, seq;
+  uint32_t a0, a1, b0, b1;      // tile list [a0, a1) of block 2p, [b0, b1) of block 2p+1
 };
 
-__device__ __forceinline__ Item load_item(const unsigned char* blob, const DamHeader* H, int w, DamSeq* sq_out) {
-  const uint32_t row = __ldg(reinterpret_cast<const uint32_t*>(blob + H->off_work) + w);
-  const int h = row / H->total_qblocks, gqb = row % H->total_qblocks;
-  const int b = __ldg(reinterpret_cast<const int32_t*>(blob + H->off_qbseq) + gqb);
-  const DamSeq sq = reinterpret_cast<const DamSeq*>(blob + H->off_seq)[b];
-  const uint32_t* tp = reinterpret_cast<const uint32_t*>(blob + H->off_tile_ptr);
+__device__ __forceinline__ Item load_item(const unsigned char* blob, const DamHeader* H, int w) {
+  const uint4* src = reinterpret_cast<const uint4*>(blob + H->off_work) + 2 * (size_t)w;
+  const uint4 u = __ldg(src), v = __ldg(src + 1);
   Item it;
-  it.head = h; it.seq_tok0 = sq.tok_start; it.qb = gqb - sq.first_qblock; it.S = sq.S;
-  it.t0 = __ldg(tp + row); it.nt = __ldg(tp + row + 1) - it.t0;
-  if (sq_out) *sq_out = sq;
+  it.head = (int)u.x; it.tok0 = (int)u.y; it.qb0 = (int)u.z; it.S = (int)u.w;
+  it.a0 = v.x; it.a1 = v.y; it.b0 = v.y; it.b1 = v.z;
+  it.hasB = (int)(v.w >> 31); it.seq = (int)(v.w & 0x7FFFFFFFu);
   return it;
+}
+
+// Merge of the two ascending tile lists: every step is one kv tile with the kinds it has in A and in B.
+struct Walker {
+  const uint32_t* tiles;
+  uint32_t ia, ea, ib, eb, ca, cb;
+  __device__ __forceinline__ void init(const uint32_t* t, const Item& it) {
+    tiles = t; ia = it.a0; ea = it.a1; ib = it.b0; eb = it.b1;
+    ca = ia < ea ? __ldg(tiles + ia) : kNone;
+    cb = ib < eb ? __ldg(tiles + ib) : kNone;
+  }
+  __device__ __forceinline__ bool next(int& kb, uint32_t& kindA, uint32_t& kindB) {
+    const uint32_t ja = ca == kNone ? kNone : (ca & 0x0FFFFFFFu);
+    const uint32_t jb = cb == kNone ? kNone : (cb & 0x0FFFFFFFu);
+    const uint32_t k = ja < jb ? ja : jb;
+    if (k == kNone) return false;
+    kb = (int)k;
+    kindA = (ja == k) ? (ca >> 28) : 0u;
+    kindB = (jb == k) ? (cb >> 28) : 0u;
+    if (ja == k) { ++ia; ca = ia < ea ? __ldg(tiles + ia) : kNone; }
+    if (jb == k) { ++ib; cb = ib < eb ? __ldg(tiles + ib) : kNone; }
+    return true;
+  }
+  __device__ __forceinline__ bool a_done() const { return ia >= ea; }
+  __device__ __forceinline__ bool b_done() const { return ib >= eb; }
+};
+
+__device__ __forceinline__ uint32_t pick_word(const uint4& b, int c) {
+  return c == 0 ? b.x : (c == 1 ? b.y : (c == 2 ? b.z : b.w));
+}
+
+
+// ---- packed fp32x2 arithmetic (one instruction for two lanes of a register pair) -----------------------
+__device__ __forceinline__ void fma2(float& d0, float& d1, float a0, float a1, float b0, float b1, float c0, float c1) {
+  asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
+      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%6, %7};\n\t"
+      "fma.rn.f32x2 rd, ra, rb, rc;\n\t"
+      "mov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1), "f"(c0), "f"(c1));
+}
+__device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1, float b0, float b1) {
+  asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+      "add.rn.f32x2 rd, ra, rb;\n\t"
+      "mov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+
+// 2^y for a pair of values on the FMA / ALU pipes instead of the special-function unit: split y into its
+// nearest integer (added to the exponent field) and a remainder in [-0.5, 0.5] (degree-3 minimax polynomial,
+// relative error 7.6e-5, far below the bf16 rounding of P).  y is clamped at -125 so that the exponent stays
+// in range; that turns an underflowing probability into 2^-125 instead of 0.
+__device__ __forceinline__ void ex2_poly2(float y0, float y1, float& p0, float& p1) {
+  const float kMagic = 12582912.f;    // 1.5 * 2^23: adding it leaves round(y) in the low mantissa bits
+  y0 = fmaxf(y0, -125.f); y1 = fmaxf(y1, -125.f);
+  float r0, r1, i0, i1, f0, f1, q0, q1;
+  add2(r0, r1, y0, y1, kMagic, kMagic);
+  add2(i0, i1, r0, r1, -kMagic, -kMagic);
+  add2(f0, f1, y0, y1, -i0, -i1);
+  fma2(q0, q1, f0, f1, 0.05520550534129143f, 0.05520550534129143f, 0.24261397123336792f, 0.24261397123336792f);
+  fma2(q0, q1, q0, q1, f0, f1, 0.6932547688484192f, 0.6932547688484192f);
+  fma2(q0, q1, q0, q1, f0, f1, 0.9999276995658875f, 0.9999276995658875f);
+  p0 = __int_as_float(__float_as_int(q0) + (__float_as_int(r0) << 23));
+  p1 = __int_as_float(__float_as_int(q1) + (__float_as_int(r1) << 23));
+}
+
+// Sweep 1 over one S row held in TMEM (4 chunks of 32 columns, next chunk in flight while one is reduced).
+template <bool MASKED>
+__device__ __forceinline__ float sweep_max(uint32_t tS, const uint4& bits) {
+  uint32_t ra[32], rb[32];
+  float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F, mx2 = -CUDART_INF_F, mx3 = -CUDART_INF_F;
+  tmem_ld32(tS, ra);
+  tc_wait_ld();
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    uint32_t* cur = (c & 1) ? rb : ra;
+    uint32_t* nxt = (c & 1) ? ra : rb;
+    if (c < 3) tmem_ld32(tS + (c + 1) * 32, nxt);
+    const uint32_t word = pick_word(bits, c);
+#pragma unroll
+    for (int q = 0; q < 32; q += 4) {
+      float v0 = __uint_as_float(cur[q]), v1 = __uint_as_float(cur[q + 1]);
+      float v2 = __uint_as_float(cur[q + 2]), v3 = __uint_as_float(cur[q + 3]);
+      if (MASKED) {
+        v0 = ((word >> q) & 1u) ? v0 : -CUDART_INF_F;
+        v1 = ((word >> (q + 1)) & 1u) ? v1 : -CUDART_INF_F;
+        v2 = ((word >> (q + 2)) & 1u) ? v2 : -CUDART_INF_F;
+        v3 = ((word >> (q + 3)) & 1u) ? v3 : -CUDART_INF_F;
+      }
+      mx0 = fmaxf(mx0, v0); mx1 = fmaxf(mx1, v1); mx2 = fmaxf(mx2, v2); mx3 = fmaxf(mx3, v3);
+    }
+    if (c < 3) tc_wait_ld();
+  }
+  return fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+}
+
+// Sweep 2: p = 2^(s * scale + neg_m) for the row, packed to bf16 and stored over the first 64 columns of the
+// row's S (chunk c+1 is in registers before chunk c's columns are overwritten).  Of every 8 probabilities, 6
+// go through the special-function unit and 2 through the polynomial.  Returns the row sum (fp32, before the
+// bf16 rounding).  A masked tile skips the arithmetic of a 32-column chunk that is inactive for every row of
+// the warp.
+template <bool MASKED>
+__device__ __forceinline__ float sweep_exp(uint32_t tS, const uint4& bits, float scale, float neg_m) {
+  uint32_t ra[32], rb[32];
+  float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+  tmem_ld32(tS, ra);
+  tc_wait_ld();
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    uint32_t* cur = (c & 1) ? rb : ra;
+    uint32_t* nxt = (c & 1) ? ra : rb;
+    if (c < 3) tmem_ld32(tS + (c + 1) * 32, nxt);
+    const uint32_t word = pick_word(bits, c);
+    uint32_t pk[16];
+    const bool live = !MASKED || __any_sync(0xFFFFFFFFu, word != 0u);
+    if (live) {
+#pragma unroll
+      for (int q = 0; q < 32; q += 8) {
+        float y[8], p[8];
+#pragma unroll
+        for (int u = 0; u < 8; u += 2)
+          fma2(y[u], y[u + 1], __uint_as_float(cur[q + u]), __uint_as_float(cur[q + u + 1]), scale, scale, neg_m, neg_m);
+#pragma unroll
+        for (int u = 0; u < 6; ++u) p[u] = ex2(y[u]);
+        ex2_poly2(y[6], y[7], p[6], p[7]);
+        if (MASKED) {
+#pragma unroll
+          for (int u = 0; u < 8; ++u) p[u] = ((word >> (q + u)) & 1u) ? p[u] : 0.f;
+        }
+        add2(s0, s1, s0, s1, p[0], p[1]);
+        add2(s2, s3, s2, s3, p[2], p[3]);
+        add2(s0, s1, s0, s1, p[4], p[5]);
+        add2(s2, s3, s2, s3, p[6], p[7]);
+#pragma unroll
+        for (int u = 0; u < 8; u += 2) {
+          __nv_bfloat162 h = __floats2bfloat162_rn(p[u], p[u + 1]);
+          pk[(q + u) >> 1] = *reinterpret_cast<uint32_t*>(&h);
+        }
+      }
+    } else {
+#pragma unroll
+      for (int q = 0; q < 16; ++q) pk[q] = 0u;
+    }
+    if (c < 3) tc_wait_ld();
+    tmem_st16(tS + c * 16, pk);
+  }
+  return (s0 + s1) + (s2 + s3);
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
 attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                  const __grid_constant__ CUtensorMap tmV, const AttnParams prm) {
+                  const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
+                  const AttnParams prm) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t sbase = smem_u32(smem);
@@ -89,24 +251,23 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   const uint32_t bar0 = sbase + SmemLayout::bars;
   const uint32_t bQFull = bar0, bQEmpty = bar0 + 8;
   const uint32_t bSlotFull = bar0 + 16, bSlotEmpty = bSlotFull + 8 * kSlots;
-  const uint32_t bSFull = bSlotEmpty + 8 * kSlots, bPFull = bSFull + 16, bPvDone = bPFull + 16;
+  const uint32_t bSFull = bSlotEmpty + 8 * kSlots, bPFull = bSFull + 16, bOFinal = bPFull + 16;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + SmemLayout::tmem_slot);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + SmemLayout::abort_flag);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const unsigned char* blob = prm.blob;
   const DamHeader* H = reinterpret_cast<const DamHeader*>(blob);
-  const int nrows = H->rows;
+  const int nitems = H->prows;
   const uint32_t* tiles = reinterpret_cast<const uint32_t*>(blob + H->off_tiles);
 
   if (tid == 0) {
     mbar_init(bQFull, 1); mbar_init(bQEmpty, 1);
     for (int s = 0; s < kSlots; ++s) { mbar_init(bSlotFull + 8 * s, 1); mbar_init(bSlotEmpty + 8 * s, 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(bSFull + 8 * s, 1); mbar_init(bPFull + 8 * s, 128); }
-    mbar_init(bPvDone, 1);
+    for (int s = 0; s < 2; ++s) { mbar_init(bSFull + 8 * s, 1); mbar_init(bPFull + 8 * s, 4); mbar_init(bOFinal + 8 * s, 1); }
     *abort_flag = 0u;
     mbar_fence_init();
-    tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
+    tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); tma_prefetch_desc(&tmO);
   }
   if (warp == 0) { tmem_alloc(smem_u32(tmem_slot), kTmemCols); tmem_relinquish(); }
   tc_fence_before();
@@ -122,9 +283,12 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 #pragma unroll
       for (int s = 0; s < kSlots; ++s) armed[s] = 2u;      // 2 = never armed
       bool ok = true;
+      PROF_DECL(4)
       auto load_tile = [&](const CUtensorMap* tm, int head, int tok) -> bool {
         const uint32_t s = sc % kSlots, ph = (sc / kSlots) & 1u;
+        PROF_LAP(0)
         if (!mbar_wait(bSlotEmpty + 8 * s, ph ^ 1u, abort_flag)) return false;
+        PROF_LAP(1)
         const uint32_t dst = sSlots + s * kSlotBytes, bar = bSlotFull + 8 * s;
         mbar_arrive_expect_tx(bar, kSlotBytes);
         tma_load_3d(dst, tm, bar, 0, head, tok);
@@ -133,27 +297,25 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         ++sc;
         return true;
       };
-      for (int w = blockIdx.x; w < nrows && ok; w += gridDim.x) {
-        const Item it = load_item(blob, H, w, nullptr);
-        if (it.nt == 0) continue;
+      for (int w = blockIdx.x; w < nitems && ok; w += gridDim.x) {
+        const Item it = load_item(blob, H, w);
+        if (it.a0 == it.b1) continue;                        // no tile in either list
         if (!(ok = mbar_wait(bQEmpty, (ic & 1u) ^ 1u, abort_flag))) break;
-        mbar_arrive_expect_tx(bQFull, kSlotBytes);
-        tma_load_3d(sQ, &tmQ, bQFull, 0, it.head, it.seq_tok0 + it.qb * DAM_TILE);
-        tma_load_3d(sQ + 16384, &tmQ, bQFull, 64, it.head, it.seq_tok0 + it.qb * DAM_TILE);
+        const int tokq = it.tok0 + it.qb0 * DAM_TILE;
+        mbar_arrive_expect_tx(bQFull, it.hasB ? 2 * kSlotBytes : kSlotBytes);
+        tma_load_3d(sQ, &tmQ, bQFull, 0, it.head, tokq);
+        tma_load_3d(sQ + 16384, &tmQ, bQFull, 64, it.head, tokq);
+        if (it.hasB) {
+          tma_load_3d(sQ + 32768, &tmQ, bQFull, 0, it.head, tokq + DAM_TILE);
+          tma_load_3d(sQ + 49152, &tmQ, bQFull, 64, it.head, tokq + DAM_TILE);
+        }
         ++ic;
         const int kvh = it.head / prm.group;
-        // ring order = order in which the MMA warp consumes: K0, K1, V0, K2, V1, ..., V(n-1)
-        for (uint32_t t = 0; t < it.nt && ok; ++t) {
-          const int kb = (int)(__ldg(tiles + it.t0 + t) & 0x0FFFFFFFu);
-          ok = load_tile(&tmK, kvh, it.seq_tok0 + kb * DAM_TILE);
-          if (ok && t >= 1) {
-            const int kbp = (int)(__ldg(tiles + it.t0 + t - 1) & 0x0FFFFFFFu);
-            ok = load_tile(&tmV, kvh, it.seq_tok0 + kbp * DAM_TILE);
-          }
-        }
-        if (ok) {
-          const int kbl = (int)(__ldg(tiles + it.t0 + it.nt - 1) & 0x0FFFFFFFu);
-          ok = load_tile(&tmV, kvh, it.seq_tok0 + kbl * DAM_TILE);
+        Walker wk; wk.init(tiles, it);
+        int kb; uint32_t kA, kB;
+        while (ok && wk.next(kb, kA, kB)) {
+          ok = load_tile(&tmK, kvh, it.tok0 + kb * DAM_TILE);
+          if (ok) ok = load_tile(&tmV, kvh, it.tok0 + kb * DAM_TILE);
         }
       }
       if (!ok) {
@@ -163,75 +325,132 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           if (armed[s] != 2u) mbar_wait(bSlotFull + 8 * s, armed[s], &dummy, 20000000ull);
         mbar_wait(bQFull, (ic + 1u) & 1u, &dummy, 20000000ull);
       }
+      PROF_LAP(0)
+      PROF_FLUSH(0, 4)
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       const uint32_t idesc_qk = idesc_bf16_f32(128, 128, 0);
       const uint32_t idesc_pv = idesc_bf16_f32(128, 128, 1);
-      uint32_t sc = 0, ic = 0, g = 0;
+      uint32_t sc = 0, ic = 0;
+      uint32_t cP[2] = {0u, 0u};           // P tiles consumed per stream (phase of p_full)
       bool ok = true;
-      for (int w = blockIdx.x; w < nrows && ok; w += gridDim.x) {
-        const Item it = load_item(blob, H, w, nullptr);
-        if (it.nt == 0) continue;
-        if (!(ok = mbar_wait(bQFull, ic & 1u, abort_flag))) break;
-        ++ic;
-        tc_fence_after();
-        auto do_pv = [&](uint32_t u) -> bool {
-          const uint32_t gt = g + u, buf = gt & 1u;
-          if (!mbar_wait(bPFull + 8 * buf, (gt >> 1) & 1u, abort_flag)) return false;
-          const uint32_t s = sc % kSlots;
-          if (!mbar_wait(bSlotFull + 8 * s, (sc / kSlots) & 1u, abort_flag)) return false;
-          tc_fence_after();
-          const uint32_t vaddr = sSlots + s * kSlotBytes;
+      PROF_DECL(6)
+      // descriptors: the high words are invariant, the low words step by (byte offset >> 4)
+      const uint64_t dQ = smem_desc_sw128(sQ, 16, 1024);
+      const uint64_t dK = smem_desc_sw128(sSlots, 16, 1024);
+      const uint64_t dV = smem_desc_sw128(sSlots, 16384, 1024);
+      const uint32_t dQ_lo = (uint32_t)dQ, dQ_hi = (uint32_t)(dQ >> 32);
+      const uint32_t dK_lo = (uint32_t)dK, dK_hi = (uint32_t)(dK >> 32);
+      const uint32_t dV_lo = (uint32_t)dV, dV_hi = (uint32_t)(dV >> 32);
+      auto issue_s = [&](int X, uint32_t slot) {
+        const uint32_t a0 = dQ_lo + X * (kSlotBytes >> 4), b0 = dK_lo + slot * (kSlotBytes >> 4);
+        const uint32_t d = tmem + kColS + X * 128;
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {
-            // V is MN-major: 16 keys per step = 2048 bytes; 64-column halves 16384 bytes apart
-            const uint64_t bdesc = smem_desc_sw128(vaddr + ks * 2048, 16384, 1024);
-            mma_ts(tmem + kColO, tmem + kColP + buf * 64 + ks * 8, bdesc, idesc_pv, (u > 0 || ks > 0) ? 1u : 0u);
-          }
-          tc_commit(bSlotEmpty + 8 * s);
-          tc_commit(bPvDone);
-          ++sc;
-          return true;
-        };
-        for (uint32_t t = 0; t < it.nt && ok; ++t) {
-          const uint32_t gt = g + t, buf = gt & 1u;
+        for (int ks = 0; ks < 8; ++ks) {
+          const uint32_t off = ((ks >> 2) * 16384 + (ks & 3) * 32) >> 4;
+          mma_ss_lh(d, a0 + off, dQ_hi, b0 + off, dK_hi, idesc_qk, ks > 0 ? 1u : 0u);
+        }
+        tc_commit(bSFull + 8 * X);
+      };
+      auto issue_pv = [&](int X, uint32_t slot, bool accumulate) -> bool {
+        PROF_LAP(0)
+        if (!mbar_wait(bPFull + 8 * X, cP[X] & 1u, abort_flag)) return false;
+        PROF_LAP(1 + X)
+        ++cP[X];
+        tc_fence_after();
+        const uint32_t b0 = dV_lo + slot * (kSlotBytes >> 4);
+        const uint32_t d = tmem + kColO + X * 128, a = tmem + kColS + X * 128;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          // V is MN-major: 16 keys per step = 2048 bytes; 64-column halves 16384 bytes apart
+          mma_ts_lh(d, a + ks * 8, b0 + ks * (2048 >> 4), dV_hi, idesc_pv, (accumulate || ks > 0) ? 1u : 0u);
+        }
+        return true;
+      };
+      for (int w = blockIdx.x; w < nitems && ok; w += gridDim.x) {
+        const Item it = load_item(blob, H, w);
+        if (it.a0 == it.b1) continue;
+        Walker wk; wk.init(tiles, it);
+        int kb; uint32_t curA, curB;
+        wk.next(kb, curA, curB);                               // at least one step exists
+        PROF_LAP(0)
+        if (!(ok = mbar_wait(bQFull, ic & 1u, abort_flag))) break;
+        PROF_LAP(3)
+        ++ic;
+        // S of the first step
+        {
           const uint32_t s = sc % kSlots;
           if (!(ok = mbar_wait(bSlotFull + 8 * s, (sc / kSlots) & 1u, abort_flag))) break;
+          PROF_LAP(4)
           tc_fence_after();
-          const uint32_t kaddr = sSlots + s * kSlotBytes;
-#pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {
-            const uint32_t off = (ks >> 2) * 16384 + (ks & 3) * 32;
-            const uint64_t adesc = smem_desc_sw128(sQ + off, 16, 1024);
-            const uint64_t bdesc = smem_desc_sw128(kaddr + off, 16, 1024);
-            mma_ss(tmem + kColS + buf * 128, adesc, bdesc, idesc_qk, ks > 0 ? 1u : 0u);
-          }
+          if (curA) issue_s(0, s);
+          if (curB) issue_s(1, s);
           tc_commit(bSlotEmpty + 8 * s);
-          tc_commit(bSFull + 8 * buf);
-          if (t + 1 == it.nt) tc_commit(bQEmpty);
           ++sc;
-          if (t >= 1) ok = do_pv(t - 1);
         }
-        if (ok) ok = do_pv(it.nt - 1);
-        g += it.nt;
+        bool accA = false, accB = false;
+        while (ok) {
+          uint32_t nxtA = 0, nxtB = 0;
+          const bool have_nxt = wk.next(kb, nxtA, nxtB);
+          if (!have_nxt) tc_commit(bQEmpty);                   // every S of this item has been issued
+          const uint32_t sv = sc % kSlots;                     // V of the current step
+          PROF_LAP(0)
+          if (!(ok = mbar_wait(bSlotFull + 8 * sv, (sc / kSlots) & 1u, abort_flag))) break;
+          PROF_LAP(4)
+          ++sc;
+          uint32_t sk = 0;
+          // a stream's output is final right after the P V of its last listed tile
+          const bool lastA = curA && nxtA == 0u && wk.a_done();
+          const bool lastB = curB && nxtB == 0u && wk.b_done();
+          if (curA) { if (!(ok = issue_pv(0, sv, accA))) break; accA = true; if (lastA) tc_commit(bOFinal); }
+          if (have_nxt) {                                      // K of the next step
+            sk = sc % kSlots;
+            PROF_LAP(0)
+            if (!(ok = mbar_wait(bSlotFull + 8 * sk, (sc / kSlots) & 1u, abort_flag))) break;
+            PROF_LAP(4)
+            ++sc;
+            tc_fence_after();
+            if (nxtA) issue_s(0, sk);
+          }
+          if (curB) { if (!(ok = issue_pv(1, sv, accB))) break; accB = true; if (lastB) tc_commit(bOFinal + 8); }
+          tc_commit(bSlotEmpty + 8 * sv);
+          if (have_nxt) {
+            if (nxtB) issue_s(1, sk);
+            tc_commit(bSlotEmpty + 8 * sk);
+          } else {
+            break;
+          }
+          curA = nxtA; curB = nxtB;
+        }
       }
+      PROF_LAP(0)
+      PROF_FLUSH(4, 6)
     }
   } else {
     // ------------------------------------------------------------------ softmax / epilogue warps
+    const int X = (warp - 2) >> 2;                           // stream: 0 = block 2p, 1 = block 2p+1
     const int r = (warp & 3) * 32 + lane;                    // row of the tile = TMEM lane
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-    uint32_t g = 0;
+    const uint32_t tS = tmem + lane_addr + kColS + X * 128;
+    const uint32_t tO = tmem + lane_addr + kColO + X * 128;
+    const uint32_t bS = bSFull + 8 * X, bP = bPFull + 8 * X, bO = bOFinal + 8 * X;
+    const uint32_t stage_addr = sbase + SmemLayout::stage + X * kStageBytes;
+    const bool stage_leader = (warp & 3) == 0 && lane == 0;   // issues this stream's TMA stores
+    uint32_t cS = 0, cO = 0;
     bool ok = true;
-    for (int w = blockIdx.x; w < nrows && ok; w += gridDim.x) {
-      DamSeq sq;
-      const Item it = load_item(blob, H, w, &sq);
-      const int i = it.qb * DAM_TILE + r;
+    PROF_DECL(8)
+    for (int w = blockIdx.x; w < nitems && ok; w += gridDim.x) {
+      const Item it = load_item(blob, H, w);
+      if (X == 1 && !it.hasB) continue;
+      const int qb = it.qb0 + X;
+      const uint32_t t0 = X ? it.b0 : it.a0, t1 = X ? it.b1 : it.a1;
+      const int i = qb * DAM_TILE + r;
       const bool row_valid = i < it.S;
-      __nv_bfloat16* orow = prm.O + (int64_t)(it.seq_tok0 + i) * prm.o_stride_tok + (int64_t)it.head * prm.o_stride_head;
-      float* lse_p = prm.lse + (int64_t)it.head * prm.total_tokens + it.seq_tok0 + i;
-      if (it.nt == 0) {
+      __nv_bfloat16* orow = prm.O + (int64_t)(it.tok0 + i) * prm.o_stride_tok + (int64_t)it.head * prm.o_stride_head;
+      float* lse_p = prm.lse + (int64_t)it.head * prm.total_tokens + it.tok0 + i;
+      if (t0 == t1) {
         if (row_valid) {
           const uint4 z = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
@@ -240,40 +459,38 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
         continue;
       }
+      const DamSeq sq = reinterpret_cast<const DamSeq*>(blob + H->off_seq)[it.seq];
       const DamHeadBits hb = dam_head_bits(blob, H, sq, it.head);
       float m_ref = -CUDART_INF_F;   // reference max (scaled, log2 domain) that P and O are expressed against
       float l = 0.f;
-      for (uint32_t t = 0; t < it.nt; ++t) {
-        const uint32_t e = __ldg(tiles + it.t0 + t);
+      // the mask words of a tile come from global memory: they are fetched one tile ahead
+      auto tile_bits = [&](uint32_t e, bool& need) -> uint4 {
         const int kb = (int)(e & 0x0FFFFFFFu);
         const uint32_t kind = e >> 28;
-        const bool need_mask = (kind != DAM_KIND_FULL) || (prm.causal && kb >= it.qb) || ((kb + 1) * DAM_TILE > it.S);
-        uint4 bits = make_uint4(~0u, ~0u, ~0u, ~0u);
-        if (need_mask) bits = dam_apply_bits(hb, kind, i, kb, prm.causal);
-        const uint32_t gt = g + t, buf = gt & 1u;
-        if (!(ok = mbar_wait(bSFull + 8 * buf, (gt >> 1) & 1u, abort_flag))) break;
-        tc_fence_after();
-        // ---- S row -> registers (raw dot products), masked entries -> -inf
-        float x[128];
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t rr[32];
-          tmem_ld32(tmem + lane_addr + kColS + buf * 128 + c * 32, rr);
-          tc_wait_ld();
-          const uint32_t word = c == 0 ? bits.x : (c == 1 ? bits.y : (c == 2 ? bits.z : bits.w));
-#pragma unroll
-          for (int q = 0; q < 32; ++q) {
-            float v = __uint_as_float(rr[q]);
-            if (need_mask) v = ((word >> q) & 1u) ? v : -CUDART_INF_F;
-            x[c * 32 + q] = v;
-          }
+        need = (kind != DAM_KIND_FULL) || (prm.causal && kb >= qb) || ((kb + 1) * DAM_TILE > it.S);
+        return need ? dam_apply_bits(hb, kind, i, kb, prm.causal) : make_uint4(~0u, ~0u, ~0u, ~0u);
+      };
+      uint32_t e_next = t0 + 1 < t1 ? __ldg(tiles + t0 + 1) : 0u;
+      bool need_nx = false;
+      uint4 bits_nx = tile_bits(__ldg(tiles + t0), need_nx);
+      for (uint32_t t = t0; t < t1; ++t) {
+        const bool need_mask = need_nx;
+        const uint4 bits = bits_nx;
+        if (t + 1 < t1) {
+          bits_nx = tile_bits(e_next, need_nx);
+          if (t + 2 < t1) e_next = __ldg(tiles + t + 2);
         }
-        float mx = -CUDART_INF_F;
-#pragma unroll
-        for (int q = 0; q < 128; ++q) mx = fmaxf(mx, x[q]);
+        PROF_LAP(0)
+        if (!(ok = mbar_wait(bS, cS & 1u, abort_flag))) break;
+        PROF_LAP(1)
+        ++cS;
+        tc_fence_after();
+        // ---- sweep 1: row maximum of the raw dot products (masked entries excluded)
+        const float mx = need_mask ? sweep_max<true>(tS, bits) : sweep_max<false>(tS, bits);
+        PROF_LAP(2)
         const float m_new = fmaxf(m_ref, mx * prm.scale_log2);
-        // move the reference only when it is the first tile or the max grew by more than the threshold
-        bool move = (t == 0) || (m_new - m_ref > kRescaleThreshold);   // -inf reference: inf > 8 is true
+        // move the reference only on the first tile or when the max grew by more than the threshold
+        bool move = (t == t0) || (m_new - m_ref > kRescaleThreshold);   // -inf reference: inf > 8 is true
         if (m_new == -CUDART_INF_F) move = false;
         float alpha = 1.f;
         if (move) {
@@ -281,70 +498,103 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           m_ref = m_new;
         }
         const float mm = (m_ref == -CUDART_INF_F) ? 0.f : m_ref;
-        float sum = 0.f;
-        uint32_t pk[64];
-#pragma unroll
-        for (int q = 0; q < 64; ++q) {
-          const float p0 = ex2(fmaf(x[2 * q], prm.scale_log2, -mm));
-          const float p1 = ex2(fmaf(x[2 * q + 1], prm.scale_log2, -mm));
-          sum += p0 + p1;
-          __nv_bfloat162 hpair = __floats2bfloat162_rn(p0, p1);
-          pk[q] = *reinterpret_cast<uint32_t*>(&hpair);
-        }
-        l = l * alpha + sum;
-        tmem_st32(tmem + lane_addr + kColP + buf * 64, pk);
-        tmem_st32(tmem + lane_addr + kColP + buf * 64 + 32, pk + 32);
-        // ---- O must be complete up to the previous tile before it is rescaled / before P(t) is consumed
-        if (t > 0) {
-          if (!(ok = mbar_wait(bPvDone, (gt - 1u) & 1u, abort_flag))) break;
-          tc_fence_after();
+        // ---- sweep 2: probabilities against the reference max, packed to bf16 into the first half of S
+        const float tsum = need_mask ? sweep_exp<true>(tS, bits, prm.scale_log2, -mm)
+                                     : sweep_exp<false>(tS, bits, prm.scale_log2, -mm);
+        PROF_LAP(3)
+        l = l * alpha + tsum;
+        // ---- O is complete up to the previous tile of this stream (its MMAs precede S of this tile)
+        if (t > t0) {
           const bool resc = alpha != 1.f;
           if (__any_sync(0xFFFFFFFFu, resc)) {
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
               uint32_t rr[32];
-              tmem_ld32(tmem + lane_addr + kColO + c * 32, rr);
+              tmem_ld32(tO + c * 32, rr);
               tc_wait_ld();
 #pragma unroll
               for (int q = 0; q < 32; ++q) rr[q] = __float_as_uint(__uint_as_float(rr[q]) * alpha);
-              tmem_st32(tmem + lane_addr + kColO + c * 32, rr);
+              tmem_st32(tO + c * 32, rr);
             }
           }
         }
+        PROF_LAP(4)
         tc_wait_st();
         tc_fence_before();
-        mbar_arrive(bPFull + 8 * buf);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bP);
+        PROF_LAP(5)
       }
       if (!ok) break;
       // ---- epilogue: O / l and the log-sum-exp
-      const uint32_t glast = g + it.nt - 1u;
-      if (!(ok = mbar_wait(bPvDone, glast & 1u, abort_flag))) break;
+      PROF_LAP(0)
+      if (!(ok = mbar_wait(bO, cO & 1u, abort_flag))) break;
+      PROF_LAP(6)
+      ++cO;
       tc_fence_after();
       const float inv = l > 0.f ? 1.0f / l : 0.f;
+      if ((qb + 1) * DAM_TILE <= it.S) {
+        // whole tile inside the sequence: through shared memory (128-byte swizzle) and two TMA stores
+        const int tok = it.tok0 + qb * DAM_TILE;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t rr[32];
-        tmem_ld32(tmem + lane_addr + kColO + c * 32, rr);
-        tc_wait_ld();
-        if (row_valid) {
+        for (int half = 0; half < 2; ++half) {
+          uint32_t pk[32];
 #pragma unroll
-          for (int v4 = 0; v4 < 4; ++v4) {
-            uint32_t o[4];
+          for (int c = 0; c < 2; ++c) {
+            uint32_t rr[32];
+            tmem_ld32(tO + (half * 2 + c) * 32, rr);
+            tc_wait_ld();
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              float a = l > 0.f ? __uint_as_float(rr[v4 * 8 + 2 * q]) * inv : 0.f;
-              float b = l > 0.f ? __uint_as_float(rr[v4 * 8 + 2 * q + 1]) * inv : 0.f;
-              __nv_bfloat162 hpair = __floats2bfloat162_rn(a, b);
-              o[q] = *reinterpret_cast<uint32_t*>(&hpair);
+            for (int q = 0; q < 16; ++q) {
+              __nv_bfloat162 hpair = __floats2bfloat162_rn(__uint_as_float(rr[2 * q]) * inv, __uint_as_float(rr[2 * q + 1]) * inv);
+              pk[c * 16 + q] = *reinterpret_cast<uint32_t*>(&hpair);
             }
-            reinterpret_cast<uint4*>(orow)[c * 4 + v4] = make_uint4(o[0], o[1], o[2], o[3]);
+          }
+          // the staging buffer is free once the previous store has been read out of it
+          if (stage_leader) tma_store_wait_read();
+          named_barrier(1 + X, 128);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const uint32_t dst = stage_addr + r * 128 + ((j ^ (r & 7)) << 4);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pk[4 * j]), "r"(pk[4 * j + 1]),
+                         "r"(pk[4 * j + 2]), "r"(pk[4 * j + 3]) : "memory");
+          }
+          fence_proxy_async();
+          named_barrier(1 + X, 128);
+          if (stage_leader) {
+            tma_store_3d(&tmO, stage_addr, half * 64, it.head, tok);
+            tma_store_commit();
+          }
+        }
+      } else {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t rr[32];
+          tmem_ld32(tO + c * 32, rr);
+          tc_wait_ld();
+          if (row_valid) {
+#pragma unroll
+            for (int v4 = 0; v4 < 4; ++v4) {
+              uint32_t o[4];
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                __nv_bfloat162 hpair = __floats2bfloat162_rn(__uint_as_float(rr[v4 * 8 + 2 * q]) * inv,
+                                                             __uint_as_float(rr[v4 * 8 + 2 * q + 1]) * inv);
+                o[q] = *reinterpret_cast<uint32_t*>(&hpair);
+              }
+              reinterpret_cast<uint4*>(orow)[c * 4 + v4] = make_uint4(o[0], o[1], o[2], o[3]);
+            }
           }
         }
       }
       if (row_valid) *lse_p = l > 0.f ? (m_ref + log2f(l)) * 0.6931471805599453f : -CUDART_INF_F;
       tc_fence_before();
-      g += it.nt;
+      PROF_LAP(7)
     }
+    if (stage_leader) tma_store_wait_all();                 // outstanding O stores complete before the CTA exits
+#ifdef DAM_PROFILE
+    if (tid == 64 || tid == 192) { PROF_FLUSH(10 + 8 * X, 8) }
+#endif
   }
 
   if (*abort_flag && tid == 64) atomicMax(prm.status, (uint32_t)DAM_ERR_DEVICE_TIMEOUT);
@@ -374,26 +624,30 @@ cudaError_t dam_launch_attn_sm100(const void* Q, const void* K, const void* V, c
       return e;
     cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
   }
-  CUtensorMap tq, tk, tv;
-  if (!dam_make_tmap_bf16(&tq, Q, 128, s->num_q_heads, s->total_tokens, s->q_stride_tok, s->q_stride_head) ||
+  CUtensorMap tq, tk, tv, to;
+  if (!dam_make_tmap_bf16(&to, O, 128, s->num_q_heads, s->total_tokens, s->o_stride_tok, s->o_stride_head) ||
+      !dam_make_tmap_bf16(&tq, Q, 128, s->num_q_heads, s->total_tokens, s->q_stride_tok, s->q_stride_head) ||
       !dam_make_tmap_bf16(&tk, K, 128, s->num_kv_heads, s->total_tokens, s->k_stride_tok, s->k_stride_head) ||
       !dam_make_tmap_bf16(&tv, V, 128, s->num_kv_heads, s->total_tokens, s->v_stride_tok, s->v_stride_head))
     return cudaErrorInvalidValue;
-  int rows = 0;
-  for (int b = 0; b < s->num_seqs; ++b)
-    rows += (s->cu_seqlens_host[b + 1] - s->cu_seqlens_host[b] + DAM_TILE - 1) / DAM_TILE;
-  rows *= s->num_q_heads;
-  if (rows == 0) return cudaSuccess;
+  int pairs = 0;
+  for (int b = 0; b < s->num_seqs; ++b) {
+    int nq = (s->cu_seqlens_host[b + 1] - s->cu_seqlens_host[b] + DAM_TILE - 1) / DAM_TILE;
+    pairs += (nq + 1) / 2;
+  }
+  pairs *= s->num_q_heads;
+  if (pairs == 0) return cudaSuccess;
   AttnParams p;
   p.blob = reinterpret_cast<const unsigned char*>(blob);
   p.O = reinterpret_cast<__nv_bfloat16*>(O);
   p.lse = lse;
   p.status = reinterpret_cast<uint32_t*>(scratch) + 1;
+  p.prof = reinterpret_cast<unsigned long long*>(reinterpret_cast<unsigned char*>(scratch) + 256);
   p.Hq = s->num_q_heads; p.group = s->num_q_heads / s->num_kv_heads; p.total_tokens = s->total_tokens;
   p.causal = causal;
   p.o_stride_tok = s->o_stride_tok; p.o_stride_head = s->o_stride_head;
   p.scale_log2 = scale * 1.4426950408889634f;
-  const int grid = rows < sm_count ? rows : sm_count;
-  attn_sm100_kernel<<<grid, kThreads, kSmemBytes, st>>>(tq, tk, tv, p);
+  const int grid = pairs < sm_count ? pairs : sm_count;
+  attn_sm100_kernel<<<grid, kThreads, kSmemBytes, st>>>(tq, tk, tv, to, p);
   return cudaGetLastError();
 }

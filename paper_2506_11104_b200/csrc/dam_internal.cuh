@@ -10,8 +10,12 @@
 //                                bit x = D[L-1-x]), V (matched columns c); W = ceil(L/32) rounded
 //                                up to a multiple of 4 words
 //   per (seq, head) true mask    L rows x W words, bit (j % 32) of word (j / 32) = M[i][j]
+//   pair_tab[total_pairs]        first global q-block of every pair of adjacent q-blocks (2p, 2p+1) of a
+//                                sequence; bit 31 set when the second block exists
 //   tile_ptr[rows + 1]           CSR over rows = head * total_qblocks + global q-block
-//   work_order[rows]             row ids, longest tile list first
+//   items[prows]                 work list of the attention kernel (DamItem, 32 B): one entry per
+//                                (head, pair), the pair with the most listed tiles (both blocks
+//                                together) first, with everything a CTA needs to start on it
 //   tiles[...]                   one u32 per listed tile: kv tile index | kind << 28
 //
 // A PARTIAL tile stores no bits of its own: inside the window they are the true-mask words of the
@@ -47,13 +51,23 @@ struct DamHeader {
   uint64_t off_seq, off_qbseq, off_dv, off_true, off_tile_ptr, off_work, off_tiles;
   uint64_t bytes_used;
   uint64_t causal_tiles;    // sum over heads and sequences of nq (nq + 1) / 2
-  uint64_t reserved[17];
+  uint64_t off_pairtab;
+  int32_t total_pairs;      // sum over sequences of ceil(nq / 2)
+  int32_t prows;            // num_q_heads * total_pairs
+  uint64_t reserved[15];
 };
 static_assert(sizeof(DamHeader) == 256, "DamHeader must be 256 bytes");
 
+struct DamItem {            // one unit of attention work: query blocks (2p, 2p+1) of one (sequence, head)
+  int32_t head, tok0, qb0, S;      // tok0 = first token of the sequence, qb0 = 2p, S = sequence length
+  uint32_t a0, a1, b1;             // tile list [a0, a1) of block 2p and [a1, b1) of block 2p+1
+  uint32_t seq_hasB;               // sequence index | (second block exists) << 31
+};
+static_assert(sizeof(DamItem) == 32, "DamItem must be 32 bytes");
+
 struct DamSeq {
   int32_t tok_start, S, L, nq;
-  int32_t first_qblock, W, nL, pad;
+  int32_t first_qblock, W, nL, first_pair;
   uint64_t dv_off;     // u32 words from off_dv: head h at dv_off + h * 3 * W
   uint64_t true_off;   // u32 words from off_true: head h at true_off + h * L * W
   uint64_t p_off;      // fp32 elements into a score tensor: head h at p_off + h * L * L
@@ -160,7 +174,7 @@ struct DamBuildCtx {
   unsigned char* blob;
   unsigned char* scratch;
   int num_seqs, Hq, Hkv, d, dtype;
-  int total_qblocks, rows;
+  int total_qblocks, rows, prows;
   int max_L, max_W, max_nL, max_nq;
   float pstar;       // single-compare threshold on p equivalent to the Box-Cox chain
   float mu;

@@ -20,10 +20,11 @@ __global__ void init_blob_kernel(unsigned char* blob, DamHeader hdr, const int32
   DamHeader* H = reinterpret_cast<DamHeader*>(blob);
   DamSeq* seqs = reinterpret_cast<DamSeq*>(blob + hdr.off_seq);
   int32_t* qbseq = reinterpret_cast<int32_t*>(blob + hdr.off_qbseq);
+  uint32_t* pairtab = reinterpret_cast<uint32_t*>(blob + hdr.off_pairtab);
   if (threadIdx.x == 0) {
     *H = hdr;
     uint64_t dv = 0, tr = 0, po = 0, co = 0;
-    int fq = 0;
+    int fq = 0, fp = 0;
     for (int b = 0; b < hdr.num_seqs; ++b) {
       int t0 = cu[b], S = cu[b + 1] - t0;
       int L = S < pcl_max ? S : pcl_max;
@@ -33,7 +34,7 @@ __global__ void init_blob_kernel(unsigned char* blob, DamHeader hdr, const int32
       int nq = (S + DAM_TILE - 1) / DAM_TILE;
       DamSeq s;
       s.tok_start = t0; s.S = S; s.L = L; s.nq = nq;
-      s.first_qblock = fq; s.W = W; s.nL = nL; s.pad = 0;
+      s.first_qblock = fq; s.W = W; s.nL = nL; s.first_pair = fp;
       s.dv_off = dv; s.true_off = tr; s.p_off = po; s.cnt_off = co;
       seqs[b] = s;
       dv += (uint64_t)Hq * 3 * W;
@@ -42,12 +43,15 @@ __global__ void init_blob_kernel(unsigned char* blob, DamHeader hdr, const int32
       if (all_ones_causal < 0) co += (uint64_t)Hq * dam_cnt_stride(L, W, nL);
       else co += all_ones_causal ? (uint64_t)nq * (nq + 1) / 2 : (uint64_t)nq * nq;   // tile base per head
       fq += nq;
+      fp += (nq + 1) / 2;
     }
   }
   __syncthreads();
   for (int b = 0; b < hdr.num_seqs; ++b) {
-    int fq = seqs[b].first_qblock, nq = seqs[b].nq;
+    int fq = seqs[b].first_qblock, nq = seqs[b].nq, fp = seqs[b].first_pair;
     for (int q = threadIdx.x; q < nq; q += blockDim.x) qbseq[fq + q] = b;
+    for (int p = threadIdx.x; p < (nq + 1) / 2; p += blockDim.x)
+      pairtab[fp + p] = (uint32_t)(fq + 2 * p) | ((2 * p + 1 < nq) ? 0x80000000u : 0u);
   }
 }
 
@@ -247,12 +251,13 @@ __global__ void classify_kernel(unsigned char* blob, unsigned char* scratch, uin
                                 uint64_t off_hist, uint64_t off_cursor) {
   DamHeader* H = reinterpret_cast<DamHeader*>(blob);
   const int lane = threadIdx.x & 31;
-  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (row >= H->rows) return;
-  const int h = row / H->total_qblocks, gqb = row % H->total_qblocks;
-  const int b = reinterpret_cast<const int32_t*>(blob + H->off_qbseq)[gqb];
+  const int prow = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);   // one warp per (head, q-block pair)
+  if (prow >= H->prows) return;
+  const int h = prow / H->total_pairs, gp = prow % H->total_pairs;
+  const uint32_t pt = reinterpret_cast<const uint32_t*>(blob + H->off_pairtab)[gp];
+  const int gqb0 = (int)(pt & 0x7FFFFFFFu), nblk = (pt >> 31) ? 2 : 1;
+  const int b = reinterpret_cast<const int32_t*>(blob + H->off_qbseq)[gqb0];
   const DamSeq sq = blob_seqs(blob, H)[b];
-  const int qb = gqb - sq.first_qblock;
   HeadView v;
   const uint32_t* dv = reinterpret_cast<const uint32_t*>(blob + H->off_dv) + sq.dv_off + (uint64_t)h * 3 * sq.W;
   const int32_t* cnt = reinterpret_cast<const int32_t*>(scratch + off_cnt) + sq.cnt_off +
@@ -260,43 +265,57 @@ __global__ void classify_kernel(unsigned char* blob, unsigned char* scratch, uin
   v.Dw = dv; v.Vw = dv + 2 * sq.W;
   v.prefD = cnt + 2 * sq.L; v.prefV = v.prefD + (sq.W + 1); v.tile_pop = v.prefV + (sq.W + 1);
   v.L = sq.L; v.W = sq.W; v.nL = sq.nL; v.S = sq.S;
-
-  // candidates, ascending: [0, min(qb, nL-1)] then [max(that + 1, qb - nL), qb]
-  const int n1 = min(qb, sq.nL - 1) + 1;
-  const int lo2 = max(n1, qb - sq.nL);
-  const int n2 = max(0, qb - lo2 + 1);
   uint32_t* rowcnt = reinterpret_cast<uint32_t*>(scratch + off_rowcnt);
   uint32_t* tile_ptr = reinterpret_cast<uint32_t*>(blob + H->off_tile_ptr);
   uint32_t* tiles = reinterpret_cast<uint32_t*>(blob + H->off_tiles);
-  uint32_t base = 0;
-  if (PASS == 1) {
-    base = tile_ptr[row];
-    if (base + rowcnt[row] > H->tile_capacity) return;   // overflow already flagged by the scan
-  }
-  int total = 0, nfull = 0;
-  for (int c0 = 0; c0 < n1 + n2; c0 += 32) {
-    int idx = c0 + lane;
-    uint32_t kind = 0;
-    int kb = 0;
-    if (idx < n1 + n2) {
-      kb = idx < n1 ? idx : lo2 + (idx - n1);
-      kind = classify_tile(v, qb, kb);
+  int pair_total = 0, nfull = 0;
+  for (int x = 0; x < nblk; ++x) {
+    const int gqb = gqb0 + x;
+    const int row = h * H->total_qblocks + gqb;
+    const int qb = gqb - sq.first_qblock;
+    // candidates, ascending: [0, min(qb, nL-1)] then [max(that + 1, qb - nL), qb]
+    const int n1 = min(qb, sq.nL - 1) + 1;
+    const int lo2 = max(n1, qb - sq.nL);
+    const int n2 = max(0, qb - lo2 + 1);
+    uint32_t base = 0;
+    bool write = PASS == 1;
+    if (PASS == 1) {
+      base = tile_ptr[row];
+      if (base + rowcnt[row] > H->tile_capacity) write = false;   // overflow already flagged by the scan
     }
-    uint32_t m = __ballot_sync(0xFFFFFFFFu, kind != 0);
-    if (PASS == 1 && kind) {
-      int rank = __popc(m & ((1u << lane) - 1u));
-      tiles[base + total + rank] = (uint32_t)kb | (kind << 28);
+    int total = 0;
+    for (int c0 = 0; c0 < n1 + n2; c0 += 32) {
+      int idx = c0 + lane;
+      uint32_t kind = 0;
+      int kb = 0;
+      if (idx < n1 + n2) {
+        kb = idx < n1 ? idx : lo2 + (idx - n1);
+        kind = classify_tile(v, qb, kb);
+      }
+      uint32_t m = __ballot_sync(0xFFFFFFFFu, kind != 0);
+      if (write && kind) {
+        int rank = __popc(m & ((1u << lane) - 1u));
+        tiles[base + total + rank] = (uint32_t)kb | (kind << 28);
+      }
+      if (PASS == 1) nfull += __popc(__ballot_sync(0xFFFFFFFFu, kind == DAM_KIND_FULL));
+      total += __popc(m);
     }
-    if (PASS == 1) nfull += __popc(__ballot_sync(0xFFFFFFFFu, kind == DAM_KIND_FULL));
-    total += __popc(m);
+    if (PASS == 0 && lane == 0) rowcnt[row] = total;
+    pair_total += total;
   }
   if (lane == 0) {
+    const int key = min(pair_total, DAM_HIST - 1);
     if (PASS == 0) {
-      rowcnt[row] = total;
-      atomicAdd(reinterpret_cast<uint32_t*>(scratch + off_hist) + min(total, DAM_HIST - 1), 1u);
+      atomicAdd(reinterpret_cast<uint32_t*>(scratch + off_hist) + key, 1u);
     } else {
-      uint32_t pos = atomicAdd(reinterpret_cast<uint32_t*>(scratch + off_cursor) + min(total, DAM_HIST - 1), 1u);
-      reinterpret_cast<uint32_t*>(blob + H->off_work)[pos] = row;
+      uint32_t pos = atomicAdd(reinterpret_cast<uint32_t*>(scratch + off_cursor) + key, 1u);
+      const int rowA = h * H->total_qblocks + gqb0;
+      DamItem it;
+      it.head = h; it.tok0 = sq.tok_start; it.qb0 = gqb0 - sq.first_qblock; it.S = sq.S;
+      it.a0 = tile_ptr[rowA]; it.a1 = it.a0 + rowcnt[rowA];
+      it.b1 = it.a1 + (nblk == 2 ? rowcnt[rowA + 1] : 0u);
+      it.seq_hasB = (uint32_t)b | (nblk == 2 ? 0x80000000u : 0u);
+      reinterpret_cast<DamItem*>(blob + H->off_work)[pos] = it;
       if (nfull) atomicAdd(&H->full_tiles, (uint32_t)nfull);
     }
   }
@@ -392,8 +411,17 @@ __global__ void all_ones_kernel(unsigned char* blob, int causal) {
   for (int k = lane; k < n; k += 32) tiles[base + k] = (uint32_t)k | (DAM_KIND_FULL << 28);
   if (lane == 0) {
     tile_ptr[row] = (uint32_t)base;
-    // heaviest q-blocks first (exact longest-first for one sequence)
-    reinterpret_cast<uint32_t*>(blob + H->off_work)[(uint64_t)h * H->total_qblocks + (H->total_qblocks - 1 - gqb)] = row;
+    // pair order: heaviest q-blocks first (exact longest-first for one sequence)
+    if (((qb & 1) == 0)) {
+      const int gp = sq.first_pair + (qb >> 1);
+      const bool hasB = qb + 1 < sq.nq;
+      DamItem it;
+      it.head = h; it.tok0 = sq.tok_start; it.qb0 = qb; it.S = sq.S;
+      it.a0 = (uint32_t)base; it.a1 = it.a0 + n;
+      it.b1 = it.a1 + (hasB ? (causal ? qb + 2 : sq.nq) : 0);
+      it.seq_hasB = (uint32_t)b | (hasB ? 0x80000000u : 0u);
+      reinterpret_cast<DamItem*>(blob + H->off_work)[(uint64_t)h * H->total_pairs + (H->total_pairs - 1 - gp)] = it;
+    }
     if (row == H->rows - 1) {
       uint32_t tot = (uint32_t)(base + n);
       tile_ptr[H->rows] = tot;
@@ -465,7 +493,7 @@ cudaError_t dam_launch_rule(const DamBuildCtx& c, cudaStream_t st) {
     match_kernel<<<c.num_seqs * c.Hq, 256, 0, st>>>(c.blob, c.scratch, c.off_cnt, c.mu, c.min_support);
   }
   if (c.rows > 0) {
-    int blocks = (c.rows + 7) / 8;
+    int blocks = (c.prows + 7) / 8;
     classify_kernel<0><<<blocks, 256, 0, st>>>(c.blob, c.scratch, c.off_cnt, c.off_rowcnt, c.off_hist, c.off_cursor);
     scan_kernel<<<1, 1024, 0, st>>>(c.blob, c.scratch, c.off_rowcnt, c.off_hist, c.off_cursor);
     classify_kernel<1><<<blocks, 256, 0, st>>>(c.blob, c.scratch, c.off_cnt, c.off_rowcnt, c.off_hist, c.off_cursor);

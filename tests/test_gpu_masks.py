@@ -118,7 +118,21 @@ def _build_and_check(w, qblocks=None):
         for h in range(0, w.num_q_heads, max(1, w.num_q_heads // 4)):
             assert all(np.array_equal(x, y) for x, y in zip(mb1.pattern_bits(b, h), mb2.pattern_bits(b, h)))
             assert np.array_equal(mb1.true_mask(b, h), mb2.true_mask(b, h))
-    assert sorted(mb1.work.tolist()) == list(range(int(mb1.hdr["rows"])))
+    # work list: one item per (head, pair of adjacent query blocks), most listed tiles first
+    tq = int(mb1.hdr["total_qblocks"])
+    seen, keys = set(), []
+    for it in mb1.items:
+        b, has2 = int(it["seq_hasB"] & 0x7FFFFFFF), int(it["seq_hasB"] >> 31)
+        sq = mb1.seqs[b]
+        row = int(it["head"]) * tq + int(sq["first_qblock"]) + int(it["qb0"])
+        assert int(it["qb0"]) % 2 == 0 and int(it["tok0"]) == int(sq["tok_start"]) and int(it["S"]) == int(sq["S"])
+        assert has2 == (int(it["qb0"]) + 1 < int(sq["nq"]))
+        assert int(it["a0"]) == int(mb1.tile_ptr[row]) and int(it["a1"]) == int(mb1.tile_ptr[row + 1])
+        assert int(it["b1"]) == int(mb1.tile_ptr[row + 1 + has2])
+        seen.add((int(it["head"]), b, int(it["qb0"])))
+        keys.append(int(it["b1"]) - int(it["a0"]))
+    assert len(seen) == int(mb1.hdr["prows"]) == len(mb1.items)
+    assert all(a >= c for a, c in zip(keys[:-1], keys[1:]))
     return blob, shape, masks, dump
 
 
