@@ -201,6 +201,31 @@ dam_status_t dam_prefill_host(const void* Q_host, const void* K_host, const void
                               void* O_host, float* lse_host, void* workspace,
                               size_t* workspace_bytes, void* stream);
 
+/*
+ * Stage 1 for callers that cannot allocate device memory (the paper has no counterpart: this is a
+ * packaging variant of dam_build_masks, not a step of the method).  A serving process that gave the
+ * whole GPU to its own memory pool, or a loop that must never call cudaMalloc, has no scratch buffer
+ * to pass; this call uses a fixed scratch array inside the library instead and allocates nothing
+ * (no cudaMalloc, cudaFree or allocating library routine on any path).
+ *   - Arguments, layouts, outputs and errors are those of dam_build_masks without `scratch`,
+ *     `scratch_bytes` and `scores_dump`; the mask blob written is identical to dam_build_masks'.
+ *   - The built-in scratch holds dam_static_scratch_bytes() bytes (8 MiB, enough for 131072 tokens x
+ *     32 heads at PCL 4096).  A shape whose build scratch (dam_mask_sizes) is larger is rejected
+ *     with DAM_ERR_BUFFER_TOO_SMALL before anything is enqueued.
+ *   - Every GPU that loads the library keeps that array until the process exits.
+ *   - The first call on a device looks up the array's device address (once per device, with that
+ *     device current); make that first call before starting any stream capture.
+ *   - All calls on a device share the one array.  Each call clears the counters it needs, so the
+ *     previous call's contents are harmless, but two calls whose GPU work overlaps (different
+ *     streams, or threads) race on it: serialise them, or use dam_build_masks with own buffers.
+ */
+dam_status_t dam_build_masks_static(const void* Q, const void* K, const dam_shape_t* shape,
+                                    const dam_rule_t* rule, void* mask, size_t mask_capacity,
+                                    void* stream);
+
+/* Size in bytes of the scratch array behind dam_build_masks_static. Host only. */
+size_t dam_static_scratch_bytes(void);
+
 #ifdef __cplusplus
 }
 #endif

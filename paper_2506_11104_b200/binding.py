@@ -23,7 +23,7 @@ STATUS = {0: "DAM_OK", 1: "DAM_ERR_INVALID_ARGUMENT", 2: "DAM_ERR_UNSUPPORTED", 
 
 EXPORTS = ["dam_version", "dam_status_string", "dam_mask_sizes", "dam_build_masks", "dam_build_masks_from_scores",
            "dam_mask_all_ones", "dam_sparse_attention", "dam_mask_stats", "dam_mask_expand_rows", "dam_poll_status",
-           "dam_prefill_host"]
+           "dam_prefill_host", "dam_build_masks_static", "dam_static_scratch_bytes"]
 
 
 class DamError(RuntimeError):
@@ -66,6 +66,7 @@ def lib():
         _lib.dam_status_string.argtypes = [ctypes.c_int]
         for name in EXPORTS[2:]:
             getattr(_lib, name).restype = ctypes.c_int
+        _lib.dam_static_scratch_bytes.restype = ctypes.c_size_t
     return _lib
 
 
@@ -161,6 +162,19 @@ def dam_build_masks(Q: torch.Tensor, K: torch.Tensor, shape: Shape, rule: dam_ru
                                _ptr(scores_dump), _stream(Q.device))
     _check(rc, "dam_build_masks")
     return mask, scratch
+
+
+def dam_build_masks_static(Q: torch.Tensor, K: torch.Tensor, shape: Shape, rule: dam_rule_t, mask: torch.Tensor):
+    """Stage 1 with the library's built-in scratch: for callers that cannot allocate device memory.
+    `mask` must already exist (size from dam_mask_sizes); nothing is allocated here or in the library."""
+    rc = lib().dam_build_masks_static(_ptr(Q), _ptr(K), shape.ref, ctypes.byref(rule), _ptr(mask),
+                                      ctypes.c_size_t(mask.numel()), _stream(Q.device))
+    _check(rc, "dam_build_masks_static")
+    return mask
+
+
+def dam_static_scratch_bytes() -> int:
+    return int(lib().dam_static_scratch_bytes())
 
 
 def dam_build_masks_from_scores(P: torch.Tensor, shape: Shape, rule: dam_rule_t, mask: Optional[torch.Tensor] = None,
