@@ -61,6 +61,32 @@ def make_layer(cfg, layer, device):
     return w
 
 
+def layer_ids_for_rank(rank, n_layers):
+    """Each rank owns its own layers (independent problems, no data-path collective): seeds differ per rank."""
+    return [rank * 1000 + l for l in range(n_layers)]
+
+
+def aggregate_over_ranks(total_ms, flops, world, device):
+    """Whole-job figures: time = MAX over ranks, work = SUM over ranks.  Returns (ms, flops)."""
+    if world <= 1:
+        return float(total_ms), float(flops)
+    import torch.distributed as dist
+    t = torch.tensor([total_ms], dtype=torch.float64, device=device)
+    f = torch.tensor([flops], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(f, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(f.item())
+
+
+def measured_traffic(kernel, cfg):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu capture (profiles/traffic.json)."""
+    p = os.path.join(ROOT, "profiles", "traffic.json")
+    try:
+        return json.load(open(p)).get(kernel, {}).get(f"C{cfg}")
+    except Exception:
+        return None
+
+
 class ClockSampler(threading.Thread):
     """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
 
@@ -160,7 +186,7 @@ def main():
     n_distinct = {1: 32, 2: 32, 3: 2, 4: 1}[cfg]
     n_layers = min(n_distinct, args.steps + args.warmup)
     # each rank owns its own layers (independent problems: no data-path collective)
-    layers = [make_layer(cfg, rank * 1000 + l, dev) for l in range(n_layers)]
+    layers = [make_layer(cfg, l, dev) for l in layer_ids_for_rank(rank, n_layers)]
     w0 = layers[0]
     shape = B.make_shape(w0.cu_seqlens, w0.num_q_heads, w0.num_kv_heads, w0.head_dim, w0.Q.dtype, dev)
     rule = B.make_rule(w0.pcl_max, w0.tau, w0.mu, w0.lam, w0.eps)
@@ -192,13 +218,21 @@ def main():
         step(i)
     torch.cuda.synchronize()
     assert B.dam_poll_status(mask) == 0 and B.dam_poll_status(ascr) == 0
+    # a longer loaded stretch before the timed region so that the clock sampler sees the GPU under this load
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    t_end = time.perf_counter() + 1.0
+    i = 0
+    while time.perf_counter() < t_end:
+        step(i)
+        i += 1
+        if i % 8 == 0:
+            torch.cuda.synchronize()
 
     # ---- timed region: exactly K steps, device-timed, per-stage events inside
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler = ClockSampler(local_rank)
     barrier()
-    sampler.start()
     start.record()
     for i in range(args.steps):
         step(args.warmup + i, evs[i])
@@ -219,12 +253,7 @@ def main():
     step_tiles = [per_layer_stats[(args.warmup + i) % n_layers]["tiles"] for i in range(args.steps)]
     total_flops = flops_tile * sum(step_tiles)
     causal_tiles = per_layer_stats[next(iter(per_layer_stats))]["causal_tiles"]
-    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    fl = torch.tensor([total_flops], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dist.all_reduce(fl, op=dist.ReduceOp.SUM)
-    total_ms_max, flops_all = float(t.item()), float(fl.item())
+    total_ms_max, flops_all = aggregate_over_ranks(total_ms, total_flops, world, dev)
     value = flops_all / (total_ms_max * 1e-3) / 1e12
 
     # ---- roofline of the dominant kernel (sparse attention), from the per-launch events
@@ -233,7 +262,7 @@ def main():
     peak = pk["bf16_sustained"] or pk["bf16"]
     roof = {"bound": "tensor", "kernel": "attn_sm100_kernel", "achieved": round(attn_tflops, 2), "peak": peak,
             "peak_kind": f"sustained cuBLAS bf16, {pk['which']}", "unit": "TFLOP/s", "frac": round(attn_tflops / peak, 4),
-            "frac_of_burst": round(attn_tflops / pk["bf16"], 4), "traffic": None,
+            "frac_of_burst": round(attn_tflops / pk["bf16"], 4), "traffic": measured_traffic("attn_sm100_kernel", cfg),
             "avg_launch_ms": round(attn_ms, 4)}
 
     out = {"metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -304,7 +333,7 @@ def main():
         del ws, hosts
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        layer_s, info = oracle_sample(layers[args.warmup % n_layers], n_rows=2048, heads=(0, 7, 13, 22, 29))
+        layer_s, info = oracle_sample(layers[args.warmup % n_layers], n_rows=6144, heads=tuple(range(w0.num_q_heads)))
         l = args.warmup % n_layers
         info["value"] = round(flops_tile * per_layer_stats.get(l, next(iter(per_layer_stats.values())))["tiles"] / layer_s / 1e12, 6)
         info["unit"] = UNIT

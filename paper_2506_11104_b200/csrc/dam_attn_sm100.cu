@@ -436,8 +436,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const uint32_t tS = tmem + lane_addr + kColS + X * 128;
     const uint32_t tO = tmem + lane_addr + kColO + X * 128;
     const uint32_t bS = bSFull + 8 * X, bP = bPFull + 8 * X, bO = bOFinal + 8 * X;
-    const uint32_t stage_addr = sbase + SmemLayout::stage + X * kStageBytes;
-    const bool stage_leader = (warp & 3) == 0 && lane == 0;   // issues this stream's TMA stores
+    const uint32_t stage_addr = sbase + SmemLayout::stage + X * kStageBytes + (warp & 3) * 4096;   // 32 rows x 128 B
     uint32_t cS = 0, cO = 0;
     bool ok = true;
     PROF_DECL(8)
@@ -534,7 +533,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       tc_fence_after();
       const float inv = l > 0.f ? 1.0f / l : 0.f;
       if ((qb + 1) * DAM_TILE <= it.S) {
-        // whole tile inside the sequence: through shared memory (128-byte swizzle) and two TMA stores
+        // whole tile inside the sequence: through shared memory (128-byte swizzle) and TMA stores
         const int tok = it.tok0 + qb * DAM_TILE;
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
@@ -550,19 +549,20 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
               pk[c * 16 + q] = *reinterpret_cast<uint32_t*>(&hpair);
             }
           }
-          // the staging buffer is free once the previous store has been read out of it
-          if (stage_leader) tma_store_wait_read();
-          named_barrier(1 + X, 128);
+          // every warp stages and stores its own 32 rows: no synchronisation beyond the warp.  The warp's
+          // staging block is free once its previous store has been read out of shared memory.
+          if (lane == 0) tma_store_wait_read();
+          __syncwarp();
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
-            const uint32_t dst = stage_addr + r * 128 + ((j ^ (r & 7)) << 4);
+            const uint32_t dst = stage_addr + lane * 128 + ((j ^ (lane & 7)) << 4);
             asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pk[4 * j]), "r"(pk[4 * j + 1]),
                          "r"(pk[4 * j + 2]), "r"(pk[4 * j + 3]) : "memory");
           }
           fence_proxy_async();
-          named_barrier(1 + X, 128);
-          if (stage_leader) {
-            tma_store_3d(&tmO, stage_addr, half * 64, it.head, tok);
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_3d(&tmO, stage_addr, half * 64, it.head, tok + (warp & 3) * 32);
             tma_store_commit();
           }
         }
@@ -591,7 +591,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       tc_fence_before();
       PROF_LAP(7)
     }
-    if (stage_leader) tma_store_wait_all();                 // outstanding O stores complete before the CTA exits
+    if (lane == 0) tma_store_wait_all();                    // outstanding O stores complete before the CTA exits
 #ifdef DAM_PROFILE
     if (tid == 64 || tid == 192) { PROF_FLUSH(10 + 8 * X, 8) }
 #endif
@@ -625,7 +625,7 @@ cudaError_t dam_launch_attn_sm100(const void* Q, const void* K, const void* V, c
     cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
   }
   CUtensorMap tq, tk, tv, to;
-  if (!dam_make_tmap_bf16(&to, O, 128, s->num_q_heads, s->total_tokens, s->o_stride_tok, s->o_stride_head) ||
+  if (!dam_make_tmap_bf16(&to, O, 128, s->num_q_heads, s->total_tokens, s->o_stride_tok, s->o_stride_head, 32) ||
       !dam_make_tmap_bf16(&tq, Q, 128, s->num_q_heads, s->total_tokens, s->q_stride_tok, s->q_stride_head) ||
       !dam_make_tmap_bf16(&tk, K, 128, s->num_kv_heads, s->total_tokens, s->k_stride_tok, s->k_stride_head) ||
       !dam_make_tmap_bf16(&tv, V, 128, s->num_kv_heads, s->total_tokens, s->v_stride_tok, s->v_stride_head))

@@ -185,13 +185,23 @@ __global__ void match_kernel(unsigned char* blob, unsigned char* scratch, uint64
     uint32_t rw = __ballot_sync(0xFFFFFFFFu, bit);
     if (lane == 0) Rw[w] = rw;
   }
-  if (threadIdx.x == 0) {
-    int a = 0, c = 0;
-    for (int w = 0; w < W; ++w) {
-      prefD[w] = a; prefV[w] = c;
-      a += __popc(Dw[w]); c += __popc(Vw[w]);
+  if (warp == 0) {
+    // prefix popcounts per word (exclusive), 32 words at a time
+    int runD = 0, runV = 0;
+    for (int w0 = 0; w0 < W; w0 += 32) {
+      const int w = w0 + lane;
+      int pd = w < W ? __popc(Dw[w]) : 0, pv = w < W ? __popc(Vw[w]) : 0;
+      int id = pd, iv = pv;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        int yd = __shfl_up_sync(0xFFFFFFFFu, id, o), yv = __shfl_up_sync(0xFFFFFFFFu, iv, o);
+        if (lane >= o) { id += yd; iv += yv; }
+      }
+      if (w < W) { prefD[w] = runD + id - pd; prefV[w] = runV + iv - pv; }
+      runD += __shfl_sync(0xFFFFFFFFu, id, 31);
+      runV += __shfl_sync(0xFFFFFFFFu, iv, 31);
     }
-    prefD[W] = a; prefV[W] = c;
+    if (lane == 0) { prefD[W] = runD; prefV[W] = runV; }
   }
 }
 
@@ -360,32 +370,33 @@ __global__ void scan_kernel(unsigned char* blob, unsigned char* scratch, uint64_
   const uint32_t* rowcnt = reinterpret_cast<const uint32_t*>(scratch + off_rowcnt);
   uint32_t* tile_ptr = reinterpret_cast<uint32_t*>(blob + H->off_tile_ptr);
   const int rows = H->rows;
-  uint32_t run = 0;
-  for (int base = 0; base < rows; base += blockDim.x) {
-    int r = base + threadIdx.x;
-    uint32_t x = r < rows ? rowcnt[r] : 0u;
-    uint32_t e = block_excl_scan(x, &tot, sm);
-    if (r < rows) tile_ptr[r] = run + e;
-    run += tot;
+  // every thread owns a run of consecutive rows: one block-wide scan over the per-thread sums
+  {
+    const int per = (rows + blockDim.x - 1) / blockDim.x;
+    const int r0 = threadIdx.x * per, r1 = min(rows, r0 + per);
+    uint32_t local = 0;
+    for (int r = r0; r < r1; ++r) local += rowcnt[r];
+    uint32_t e = block_excl_scan(local, &tot, sm);
+    for (int r = r0; r < r1; ++r) { tile_ptr[r] = e; e += rowcnt[r]; }
+    if (threadIdx.x == 0) {
+      const uint32_t run = tot;
+      tile_ptr[rows] = run;
+      H->total_tiles = run;
+      H->bytes_used = H->off_tiles + 4ull * run;
+      if (run > H->tile_capacity) H->status = DAM_ERR_BUFFER_TOO_SMALL;
+    }
     __syncthreads();
   }
-  if (threadIdx.x == 0) {
-    tile_ptr[rows] = run;
-    H->total_tiles = run;
-    H->bytes_used = H->off_tiles + 4ull * run;
-    if (run > H->tile_capacity) H->status = DAM_ERR_BUFFER_TOO_SMALL;
-  }
-  // cursors: bucket c starts after all buckets with more tiles
-  const uint32_t* hist = reinterpret_cast<const uint32_t*>(scratch + off_hist);
-  uint32_t* cursor = reinterpret_cast<uint32_t*>(scratch + off_cursor);
-  run = 0;
-  for (int base = 0; base < DAM_HIST; base += blockDim.x) {
-    int c = DAM_HIST - 1 - (base + threadIdx.x);
-    uint32_t x = hist[c];
-    uint32_t e = block_excl_scan(x, &tot, sm);
-    cursor[c] = run + e;
-    run += tot;
-    __syncthreads();
+  // cursors: bucket c starts after all buckets with more tiles (descending order of the key)
+  {
+    const uint32_t* hist = reinterpret_cast<const uint32_t*>(scratch + off_hist);
+    uint32_t* cursor = reinterpret_cast<uint32_t*>(scratch + off_cursor);
+    const int per = (DAM_HIST + blockDim.x - 1) / blockDim.x;
+    const int k0 = threadIdx.x * per, k1 = min(DAM_HIST, k0 + per);     // positions in descending-key order
+    uint32_t local = 0;
+    for (int k = k0; k < k1; ++k) local += hist[DAM_HIST - 1 - k];
+    uint32_t e = block_excl_scan(local, &tot, sm);
+    for (int k = k0; k < k1; ++k) { cursor[DAM_HIST - 1 - k] = e; e += hist[DAM_HIST - 1 - k]; }
   }
 }
 

@@ -7,8 +7,9 @@
 //   sweep A  S = Q K^T (tcgen05, accumulator in TMEM) -> per-row running max and sum;
 //   sweep B  S again -> p = exp2(x - max) / sum in fp32 -> bit = [p >= p*] -> one 16-byte store of the
 //            row's 128 bits per tile (and the optional dump of p).
-// Warp roles as in the attention kernel: warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 one thread
-// per query row.  Every wait is bounded.
+// Warp roles: warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 and 6-9 two groups of one thread per query
+// row; group G owns TMEM buffer G, i.e. every other kv tile, and the two groups merge their row statistics
+// through shared memory between the sweeps.  Every wait is bounded.
 #include <cuda_bf16.h>
 #include <math_constants.h>
 
@@ -21,16 +22,17 @@ namespace {
 
 constexpr int kSlots = 5;
 constexpr int kSlotBytes = 32768;
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;
 constexpr uint32_t kTmemCols = 256;
 
 struct SmemLayout {
   static constexpr int q = 0;
   static constexpr int slots = kSlotBytes;
   static constexpr int bars = kSlotBytes * (1 + kSlots);
-  // q_full, q_empty, slot_full[kSlots], slot_empty[kSlots], s_full[2], s_empty[2]
-  static constexpr int n_bars = 2 + 2 * kSlots + 4;
-  static constexpr int tmem_slot = bars + 8 * n_bars;
+  // q_full, q_empty, slot_full[kSlots], slot_empty[kSlots], s_full[2], s_empty[2], stat_ready
+  static constexpr int n_bars = 2 + 2 * kSlots + 5;
+  static constexpr int stat = bars + 8 * n_bars;            // float2 [2][2][128]
+  static constexpr int tmem_slot = stat + 2 * 2 * 128 * 8;
   static constexpr int abort_flag = tmem_slot + 4;
   static constexpr int total = abort_flag + 4;
 };
@@ -46,8 +48,18 @@ struct ScoreParams {
 
 __device__ __forceinline__ float ex2(float x) {
   float y;
-  asm volatile("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+__device__ __forceinline__ void mul2(float& d0, float& d1, float a0, float a1, float b0, float b1) {
+  asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+      "mul.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+__device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1, float b0, float b1) {
+  asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+      "add.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
 }
 
 struct Item { int b, h, qb, valid; DamSeq sq; };
@@ -74,7 +86,7 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   const uint32_t bar0 = sbase + SmemLayout::bars;
   const uint32_t bQFull = bar0, bQEmpty = bar0 + 8;
   const uint32_t bSlotFull = bar0 + 16, bSlotEmpty = bSlotFull + 8 * kSlots;
-  const uint32_t bSFull = bSlotEmpty + 8 * kSlots, bSEmpty = bSFull + 16;
+  const uint32_t bSFull = bSlotEmpty + 8 * kSlots, bSEmpty = bSFull + 16, bStat = bSEmpty + 16;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + SmemLayout::tmem_slot);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + SmemLayout::abort_flag);
 
@@ -86,7 +98,8 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   if (tid == 0) {
     mbar_init(bQFull, 1); mbar_init(bQEmpty, 1);
     for (int s = 0; s < kSlots; ++s) { mbar_init(bSlotFull + 8 * s, 1); mbar_init(bSlotEmpty + 8 * s, 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(bSFull + 8 * s, 1); mbar_init(bSEmpty + 8 * s, 128); }
+    for (int s = 0; s < 2; ++s) { mbar_init(bSFull + 8 * s, 1); mbar_init(bSEmpty + 8 * s, 4); }
+    mbar_init(bStat, 8);
     *abort_flag = 0u;
     mbar_fence_init();
     tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK);
@@ -164,9 +177,14 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       }
     }
   } else {
+    // ---------------------------------------------------------------- row statistics and thresholding
+    // Two groups of four warps; group G owns the S buffer G, i.e. every other kv tile of the item.
+    const int G = (warp - 2) >> 2;
     const int r = (warp & 3) * 32 + lane;
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-    uint32_t g = 0;
+    const uint32_t tS = tmem + lane_addr + G * 128;
+    float2* stat = reinterpret_cast<float2*>(smem + SmemLayout::stat);      // [2 item parities][2 groups][128 rows]
+    uint32_t g = 0, cG = 0, nitem = 0;      // g: tiles issued so far (all groups); cG: tiles this group consumed
     bool ok = true;
     for (int w = blockIdx.x; w < nitems && ok; w += gridDim.x) {
       const Item it = decode_item(blob, H, prm, w);
@@ -176,48 +194,76 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       const bool row_valid = i < L;
       uint32_t* Mrow = reinterpret_cast<uint32_t*>(blob + H->off_true) + it.sq.true_off + (uint64_t)it.h * L * W + (size_t)i * W;
       float* Prow = prm.dump ? prm.dump + it.sq.p_off + (uint64_t)it.h * L * L + (size_t)i * L : nullptr;
-      float m = -CUDART_INF_F, l = 0.f, inv_l = 0.f;
       const int nk = it.qb + 1;
+      float m = -CUDART_INF_F, l = 0.f, inv_l = 0.f;
       for (int t = 0; t < 2 * nk; ++t, ++g) {
+        if (t == nk) {
+          // both groups have finished sweep A: merge their (max, sum) per row through shared memory
+          float2* mine = stat + ((nitem & 1u) * 2 + G) * DAM_TILE;
+          const float2* other = stat + ((nitem & 1u) * 2 + (G ^ 1)) * DAM_TILE;
+          mine[r] = make_float2(m, l);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bStat);                       // release: the warp's 32 rows are written
+          if (!(ok = mbar_wait(bStat, nitem & 1u, abort_flag))) break;
+          const float2 o = other[r];
+          const float mn = fmaxf(m, o.x);
+          l = (m == -CUDART_INF_F ? 0.f : l * ex2(m - mn)) + (o.x == -CUDART_INF_F ? 0.f : o.y * ex2(o.x - mn));
+          m = mn;
+          inv_l = l > 0.f ? 1.0f / l : 0.f;
+        }
+        if ((g & 1u) != (uint32_t)G) continue;
         const int kb = t % nk;
         const bool sweepB = t >= nk;
-        const uint32_t buf = g & 1u;
-        if (!(ok = mbar_wait(bSFull + 8 * buf, (g >> 1) & 1u, abort_flag))) break;
+        if (!(ok = mbar_wait(bSFull + 8 * G, cG & 1u, abort_flag))) break;
+        ++cG;
         tc_fence_after();
         // keys beyond the causal limit (and beyond the window, which the limit implies) do not exist
-        const int nvalid = min(DAM_TILE, i - kb * DAM_TILE + 1);
-        if (t == nk) inv_l = l > 0.f ? 1.0f / l : 0.f;
+        const int nvalid = kb == it.qb ? r + 1 : DAM_TILE;
+        const bool diag = kb == it.qb;
         uint4 words = make_uint4(0u, 0u, 0u, 0u);
         float tmax = -CUDART_INF_F, tsum = 0.f;
+        uint32_t ra[32], rb[32];
+        tmem_ld32(tS, ra);
+        tc_wait_ld();
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-          uint32_t rr[32];
-          tmem_ld32(tmem + lane_addr + buf * 128 + c * 32, rr);
-          tc_wait_ld();
+          uint32_t* cur = (c & 1) ? rb : ra;
+          uint32_t* nxt = (c & 1) ? ra : rb;
+          if (c < 3) tmem_ld32(tS + (c + 1) * 32, nxt);
+          float x[32];
+#pragma unroll
+          for (int q = 0; q < 32; q += 2)
+            mul2(x[q], x[q + 1], __uint_as_float(cur[q]), __uint_as_float(cur[q + 1]), prm.scale_log2, prm.scale_log2);
+          if (diag) {
+#pragma unroll
+            for (int q = 0; q < 32; ++q) x[q] = (c * 32 + q < nvalid) ? x[q] : -CUDART_INF_F;
+          }
           if (!sweepB) {
-            float cm = -CUDART_INF_F;
+            float c0 = -CUDART_INF_F, c1 = -CUDART_INF_F, c2 = -CUDART_INF_F, c3 = -CUDART_INF_F;
 #pragma unroll
-            for (int q = 0; q < 32; ++q) {
-              float x = __uint_as_float(rr[q]) * prm.scale_log2;
-              x = (c * 32 + q < nvalid) ? x : -CUDART_INF_F;
-              rr[q] = __float_as_uint(x);
-              cm = fmaxf(cm, x);
+            for (int q = 0; q < 32; q += 4) {
+              c0 = fmaxf(c0, x[q]); c1 = fmaxf(c1, x[q + 1]); c2 = fmaxf(c2, x[q + 2]); c3 = fmaxf(c3, x[q + 3]);
             }
-            const float mn = fmaxf(tmax, cm);
+            const float mn = fmaxf(tmax, fmaxf(fmaxf(c0, c1), fmaxf(c2, c3)));
             if (mn > -CUDART_INF_F) {
-              float cs = 0.f;
+              float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
-              for (int q = 0; q < 32; ++q) cs += ex2(__uint_as_float(rr[q]) - mn);
-              tsum = tsum * ex2(tmax - mn) + cs;     // tmax = -inf gives a factor 0
+              for (int q = 0; q < 32; q += 4) {
+                float y0, y1, y2, y3;
+                add2(y0, y1, x[q], x[q + 1], -mn, -mn);
+                add2(y2, y3, x[q + 2], x[q + 3], -mn, -mn);
+                add2(a0, a1, a0, a1, ex2(y0), ex2(y1));
+                add2(a2, a3, a2, a3, ex2(y2), ex2(y3));
+              }
+              tsum = tsum * ex2(tmax - mn) + ((a0 + a1) + (a2 + a3));     // tmax = -inf gives a factor 0
               tmax = mn;
             }
           } else {
             uint32_t word = 0u;
 #pragma unroll
             for (int q = 0; q < 32; ++q) {
-              float x = __uint_as_float(rr[q]) * prm.scale_log2;
-              float p = (c * 32 + q < nvalid) ? ex2(x - m) * inv_l : 0.f;
-              rr[q] = __float_as_uint(p);
+              const float p = ex2(x[q] - m) * inv_l;       // x = -inf beyond the causal limit gives 0
+              x[q] = p;
               word |= (p >= prm.pstar ? 1u : 0u) << q;
             }
             if (c == 0) words.x = word; else if (c == 1) words.y = word; else if (c == 2) words.z = word; else words.w = word;
@@ -225,12 +271,14 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
               const int j0 = kb * DAM_TILE + c * 32;
 #pragma unroll
               for (int q = 0; q < 32; ++q)
-                if (j0 + q < L) Prow[j0 + q] = __uint_as_float(rr[q]);
+                if (j0 + q < L) Prow[j0 + q] = x[q];
             }
           }
+          if (c < 3) tc_wait_ld();
         }
         tc_fence_before();
-        mbar_arrive(bSEmpty + 8 * buf);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bSEmpty + 8 * G);
         if (!sweepB) {
           if (tmax > -CUDART_INF_F) {
             const float mn = fmaxf(m, tmax);
@@ -242,8 +290,9 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         }
       }
       if (!ok) break;
+      ++nitem;
       // dump: zeros above the diagonal for the tiles this item does not visit
-      if (Prow && row_valid)
+      if (Prow && row_valid && G == 0)
         for (int j = (it.qb + 1) * DAM_TILE; j < L; ++j) Prow[j] = 0.f;
     }
   }
