@@ -260,6 +260,12 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   const DamHeader* H = reinterpret_cast<const DamHeader*>(blob);
   const int nitems = H->prows;
   const uint32_t* tiles = reinterpret_cast<const uint32_t*>(blob + H->off_tiles);
+  // The work list is sorted by length; CTAs take it in boustrophedon order (forward on even rounds, backward
+  // on odd rounds) so that no CTA gets the longest item of every round.
+  auto item_of_round = [&](int rnd) -> int {
+    const int G = (int)gridDim.x, c = (int)blockIdx.x;
+    return rnd * G + ((rnd & 1) ? (G - 1 - c) : c);
+  };
 
   if (tid == 0) {
     mbar_init(bQFull, 1); mbar_init(bQEmpty, 1);
@@ -297,7 +303,9 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         ++sc;
         return true;
       };
-      for (int w = blockIdx.x; w < nitems && ok; w += gridDim.x) {
+      for (int rnd = 0; ok; ++rnd) {
+        const int w = item_of_round(rnd);
+        if (w >= nitems) { if (rnd * (int)gridDim.x >= nitems) break; continue; }
         const Item it = load_item(blob, H, w);
         if (it.a0 == it.b1) continue;                        // no tile in either list
         if (!(ok = mbar_wait(bQEmpty, (ic & 1u) ^ 1u, abort_flag))) break;
@@ -369,7 +377,9 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
         return true;
       };
-      for (int w = blockIdx.x; w < nitems && ok; w += gridDim.x) {
+      for (int rnd = 0; ok; ++rnd) {
+        const int w = item_of_round(rnd);
+        if (w >= nitems) { if (rnd * (int)gridDim.x >= nitems) break; continue; }
         const Item it = load_item(blob, H, w);
         if (it.a0 == it.b1) continue;
         Walker wk; wk.init(tiles, it);
@@ -427,6 +437,10 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       }
       PROF_LAP(0)
       PROF_FLUSH(4, 6)
+#ifdef DAM_PROFILE
+      { long long tot_ = 0; for (int q_ = 0; q_ < 6; ++q_) tot_ += prof_acc[q_];
+        prm.prof[128 + 2 * blockIdx.x] = (unsigned long long)tot_; prm.prof[128 + 2 * blockIdx.x + 1] = (unsigned long long)prof_acc[0]; }
+#endif
     }
   } else {
     // ------------------------------------------------------------------ softmax / epilogue warps
@@ -440,7 +454,9 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     uint32_t cS = 0, cO = 0;
     bool ok = true;
     PROF_DECL(8)
-    for (int w = blockIdx.x; w < nitems && ok; w += gridDim.x) {
+    for (int rnd = 0; ok; ++rnd) {
+        const int w = item_of_round(rnd);
+        if (w >= nitems) { if (rnd * (int)gridDim.x >= nitems) break; continue; }
       const Item it = load_item(blob, H, w);
       if (X == 1 && !it.hasB) continue;
       const int qb = it.qb0 + X;

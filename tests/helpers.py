@@ -13,6 +13,13 @@ def to_f32_numpy(t: torch.Tensor) -> np.ndarray:
     return t.detach().float().cpu().numpy()
 
 
+def host_qkv(w):
+    """float32 numpy copies of a workload's Q, K, V, converted once and kept on the workload object."""
+    if not hasattr(w, "_host_qkv"):
+        w._host_qkv = tuple(to_f32_numpy(x) for x in (w.Q, w.K, w.V))
+    return w._host_qkv
+
+
 def split_dump(dump: np.ndarray, lengths, Hq: int, pcl: int):
     """Flat fp32 score dump -> P[seq][head] arrays of shape [L, L]."""
     out, off = [], 0
@@ -26,13 +33,13 @@ def split_dump(dump: np.ndarray, lengths, Hq: int, pcl: int):
     return out
 
 
-def oracle_masks_from_dump(w, dump: np.ndarray, min_support: int = 1):
+def oracle_masks_from_dump(w, dump: np.ndarray, min_support: int = 1, heads=None):
     lengths = [b - a for a, b in zip(w.cu_seqlens[:-1], w.cu_seqlens[1:])]
     P = split_dump(dump, lengths, w.num_q_heads, w.pcl_max)
     out = []
     for b, S in enumerate(lengths):
         out.append([orc.head_mask_from_probs(np.ascontiguousarray(P[b][h]), S, w.tau, w.mu, w.lam, w.eps, min_support)
-                    for h in range(w.num_q_heads)])
+                    if (heads is None or h in heads) else None for h in range(w.num_q_heads)])
     return out
 
 
@@ -99,7 +106,7 @@ def check_blob_against_oracle(blob, shape, masks, qblocks_per_head=None, rng=Non
 def attention_errors(O_gpu: torch.Tensor, lse_gpu: torch.Tensor, w, masks, seq: int, head: int, rows, causal=True,
                      all_ones=False):
     """Max / mean abs error of O and max abs error of LSE on the given rows of (seq, head) vs the oracle."""
-    Q, K, V = to_f32_numpy(w.Q), to_f32_numpy(w.K), to_f32_numpy(w.V)
+    Q, K, V = host_qkv(w)
     hm = None if all_ones else masks[seq][head]
     O_ref, lse_ref = orc.attention(Q, K, V, w.cu_seqlens, seq, head, rows, hm, causal=causal)
     t0 = w.cu_seqlens[seq]

@@ -74,7 +74,7 @@ def _masked_case(w, rows_for, heads=None):
     dump = torch.zeros(n, dtype=torch.float32, device=DEV)
     blob, _ = B.dam_build_masks(w.Q.to(DEV), w.K.to(DEV), shape, rule, scores_dump=dump)
     assert B.dam_poll_status(blob) == 0
-    masks = H.oracle_masks_from_dump(w, dump.cpu().numpy())      # identical mask on both sides
+    masks = H.oracle_masks_from_dump(w, dump.cpu().numpy(), heads=heads)      # identical mask on both sides
     O, lse = _run(w, blob, shape)
     worst = _check(w, O, lse, masks, rows_for, heads=heads)
     return blob, shape, masks, O, lse, worst
@@ -122,3 +122,17 @@ def test_config1_dense_causal_sampled_rows():
 def test_config4_varlen_sampled_rows():
     w = synth.config4()
     _masked_case(w, _sample_rows(1024), heads=[2, 17])
+
+
+def test_config2_layer_sampled_rows():
+    """One layer of the 32-layer stack (32768 tokens, PCL 2048), in the launch configuration the benchmark times."""
+    w = synth.config2_layer(5, DEV)
+    blob, shape, masks, O, lse, worst = _masked_case(w, _sample_rows(2048), heads=[1, 12, 27])
+    st = B.dam_mask_stats(blob, shape)
+    assert 0.01 <= st["tiles"] / st["causal_tiles"] <= 0.30
+
+
+def test_config3_sampled_rows():
+    """131072 tokens, PCL 4096: sampled rows of a few heads against the oracle over all 131072 keys."""
+    w = synth.config3(DEV)
+    _masked_case(w, _sample_rows(4096), heads=[4, 19])

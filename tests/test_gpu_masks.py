@@ -138,7 +138,7 @@ def _build_and_check(w, qblocks=None):
 
 def _score_closeness(w, dump, masks, heads):
     """GPU fp32 map vs the float64 map; every cell whose decision differs must sit within 2 % of p*."""
-    Q, K = H.to_f32_numpy(w.Q), H.to_f32_numpy(w.K)
+    Q, K, _ = H.host_qkv(w)
     P = H.split_dump(dump.cpu().numpy(), [b - a for a, b in zip(w.cu_seqlens[:-1], w.cu_seqlens[1:])],
                      w.num_q_heads, w.pcl_max)
     g = w.num_q_heads // w.num_kv_heads
@@ -191,6 +191,14 @@ def test_config1_full_size_masks():
     assert 0.03 <= st["tiles"] / st["causal_tiles"] <= 0.45
 
 
+def test_config2_layer_masks():
+    """A layer of the 32-layer stack: 32768 tokens, PCL 2048."""
+    w = synth.config2_layer(3, DEV)
+    blob, shape, masks, dump = _build_and_check(w, qblocks=10)
+    st = B.dam_mask_stats(blob, shape)
+    assert 0.01 <= st["tiles"] / st["causal_tiles"] <= 0.30
+
+
 def test_config4_varlen_masks():
     w = synth.config4(lengths=(4096, 16384, 32768, 65536))
     _build_and_check(w, qblocks=8)
@@ -199,7 +207,6 @@ def test_config4_varlen_masks():
 def test_config3_shape_masks():
     """131072 tokens, PCL 4096 (config 3): all heads' pattern bits and true masks, sampled q-blocks."""
     w = synth.config3(device=DEV)
-    w.Q, w.K, w.V = w.Q.cpu(), w.K.cpu(), w.V.cpu()
     blob, shape, masks, dump = _build_and_check(w, qblocks=8)
     st = B.dam_mask_stats(blob, shape)
     assert 0.005 <= st["tiles"] / st["causal_tiles"] <= 0.08
