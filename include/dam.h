@@ -80,8 +80,18 @@ typedef struct dam_rule_t {
   float eps;            /* clamp constant, > 0 (Sec. 4.2.2)                                        */
   float softmax_scale;  /* 0 selects 1 / sqrt(head_dim) (Sec. 3)                                   */
   int32_t min_support;  /* ignore patterns with fewer cells; 1 = the paper's rule                  */
-  uint32_t flags;       /* reserved, 0                                                             */
+  uint32_t flags;       /* 0 or DAM_RULE_GATHER_COLUMNS                                            */
 } dam_rule_t;
+
+/*
+ * dam_rule_t.flags bit: below row 2L - 1 of a sequence the matched columns (all < L) and the matched
+ * diagonals (keys > i - L >= L - 1) never meet (Sec. 4.3, Case 2), so the K / V rows of the matched columns
+ * can be copied once per (sequence, head) into dense tiles of 128 keys that every such query block
+ * visits as fully active tiles, instead of one mostly-empty tile per stripe. The mask content is
+ * unchanged; only the tile lists differ, and dam_sparse_attention needs the larger scratch that
+ * dam_mask_sizes then reports. Honoured for the tensor-core shapes (bf16, head_dim 128); ignored otherwise.
+ */
+#define DAM_RULE_GATHER_COLUMNS 1u
 
 /* Library version (major * 1000 + minor). No arguments, no device work. */
 int32_t dam_version(void);

@@ -121,12 +121,15 @@ def make_shape(cu_seqlens: Sequence[int], Hq: int, Hkv: int, d: int, dtype: torc
     return Shape(c=s, cu_host=cu_host, cu_dev=cu_dev, lengths=lengths)
 
 
+DAM_RULE_GATHER_COLUMNS = 1
+
+
 def make_rule(pcl_max: int, tau: float, mu: float, lam: float = 0.5, eps: float = 1e-8,
-              softmax_scale: float = 0.0, min_support: int = 1) -> dam_rule_t:
+              softmax_scale: float = 0.0, min_support: int = 1, gather_columns: bool = False) -> dam_rule_t:
     r = dam_rule_t()
     r.struct_size = ctypes.sizeof(dam_rule_t)
     r.pcl_max, r.tau, r.mu, r.lambda_, r.eps = pcl_max, tau, mu, lam, eps
-    r.softmax_scale, r.min_support, r.flags = softmax_scale, min_support, 0
+    r.softmax_scale, r.min_support, r.flags = softmax_scale, min_support, (DAM_RULE_GATHER_COLUMNS if gather_columns else 0)
     return r
 
 
@@ -208,7 +211,10 @@ def dam_sparse_attention(Q, K, V, mask, shape: Shape, causal: bool = True, softm
     if lse is None:
         lse = torch.empty(shape.c.num_q_heads, shape.c.total_tokens, dtype=torch.float32, device=Q.device)
     if scratch is None:
-        scratch = _alloc(256, Q.device)
+        # a blob with gathered-column tiles records the scratch size it needs in its header
+        off = _HDR.fields["attn_scratch_bytes"][1]
+        need = int(mask[off: off + 8].cpu().numpy().view(np.uint64)[0]) if mask.numel() >= 256 else 256
+        scratch = _alloc(max(256, need), Q.device)
     rc = lib().dam_sparse_attention(_ptr(Q), _ptr(K), _ptr(V), _ptr(mask), shape.ref, int(causal),
                                     shape.c.num_q_heads // shape.c.num_kv_heads, ctypes.c_float(softmax_scale),
                                     _ptr(O), _ptr(lse), _ptr(scratch), ctypes.c_size_t(scratch.numel()),
@@ -259,10 +265,10 @@ _HDR = np.dtype([("magic", "<u4"), ("status", "<u4"), ("version", "<u4"), ("flag
                  ("off_seq", "<u8"), ("off_qbseq", "<u8"), ("off_dv", "<u8"), ("off_true", "<u8"),
                  ("off_tile_ptr", "<u8"), ("off_work", "<u8"), ("off_tiles", "<u8"), ("bytes_used", "<u8"),
                  ("causal_tiles", "<u8"), ("off_pairtab", "<u8"), ("total_pairs", "<i4"), ("prows", "<i4"),
-                 ("reserved", "<u8", (15,))])
+                 ("gath_tiles", "<u8"), ("attn_scratch_bytes", "<u8"), ("reserved", "<u8", (13,))])
 _SEQ = np.dtype([("tok_start", "<i4"), ("S", "<i4"), ("L", "<i4"), ("nq", "<i4"), ("first_qblock", "<i4"),
                  ("W", "<i4"), ("nL", "<i4"), ("first_pair", "<i4"), ("dv_off", "<u8"), ("true_off", "<u8"),
-                 ("p_off", "<u8"), ("cnt_off", "<u8")])
+                 ("p_off", "<u8"), ("cnt_off", "<u8"), ("gath_off", "<u8"), ("reserved", "<u8")])
 
 
 _ITEM = np.dtype([("head", "<i4"), ("tok0", "<i4"), ("qb0", "<i4"), ("S", "<i4"), ("a0", "<u4"), ("a1", "<u4"),
@@ -315,4 +321,10 @@ class MaskBlob:
         """(kv tile indices, kinds) of query block qb of (seq, head)."""
         row = head * int(self.hdr["total_qblocks"]) + int(self.seqs[seq]["first_qblock"]) + qb
         e = self.tiles[self.tile_ptr[row]: self.tile_ptr[row + 1]]
-        return (e & 0x0FFFFFFF).astype(np.int64), (e >> 28).astype(np.int64)
+        kinds = (e >> 28).astype(np.int64)
+        idx = np.where(kinds == 3, e & 0xFFFF, e & 0x0FFFFFFF).astype(np.int64)
+        return idx, kinds
+
+    def row_entries(self, seq: int, head: int, qb: int) -> np.ndarray:
+        row = head * int(self.hdr["total_qblocks"]) + int(self.seqs[seq]["first_qblock"]) + qb
+        return self.tiles[self.tile_ptr[row]: self.tile_ptr[row + 1]]

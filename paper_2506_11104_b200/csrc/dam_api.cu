@@ -44,20 +44,28 @@ dam_status_t check_rule(const dam_rule_t* r) {
   if (!r || r->struct_size != sizeof(dam_rule_t)) return DAM_ERR_INVALID_ARGUMENT;
   if (r->pcl_max < 1) return DAM_ERR_INVALID_ARGUMENT;
   if (!(r->tau > 0.f) || !(r->eps > 0.f) || !(r->mu == r->mu)) return DAM_ERR_INVALID_ARGUMENT;
-  if (r->min_support < 1 || r->flags != 0 || r->softmax_scale < 0.f) return DAM_ERR_INVALID_ARGUMENT;
+  if (r->min_support < 1 || (r->flags & ~DAM_RULE_GATHER_COLUMNS) != 0 || r->softmax_scale < 0.f)
+    return DAM_ERR_INVALID_ARGUMENT;
   if (r->lambda != 0.5f) return DAM_ERR_UNSUPPORTED;
   return DAM_OK;
+}
+
+bool sm100_shape(const dam_shape_t* s) { return s->dtype == DAM_BF16 && s->head_dim == 128; }
+
+// Gathered-column tiles: asked for by the rule, tensor-core shape, window small enough for the gather kernel.
+bool gather_enabled(const dam_shape_t* s, const dam_rule_t* r) {
+  return r && (r->flags & DAM_RULE_GATHER_COLUMNS) && sm100_shape(s) && r->pcl_max <= 32768;
 }
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 // Layout of the blob and of the scratch buffers, from the host copy of cu_seqlens.
 // pcl_max == 0 selects the all-ones blob (no window sections).
-void compute_layout(const dam_shape_t* s, int pcl_max, int all_ones_causal, Layout* out) {
+void compute_layout(const dam_shape_t* s, int pcl_max, int all_ones_causal, int gather, Layout* out) {
   Layout& y = *out;
   memset(&y, 0, sizeof(y));
   const int Hq = s->num_q_heads;
-  uint64_t dv = 0, tr = 0, cnt = 0, cap = 0, causal_tiles = 0, lrows = 0, po = 0;
+  uint64_t dv = 0, tr = 0, cnt = 0, cap = 0, causal_tiles = 0, lrows = 0, po = 0, gath = 0;
   int total_qb = 0, total_pairs = 0;
   for (int b = 0; b < s->num_seqs; ++b) {
     int S = s->cu_seqlens_host[b + 1] - s->cu_seqlens_host[b];
@@ -70,6 +78,7 @@ void compute_layout(const dam_shape_t* s, int pcl_max, int all_ones_causal, Layo
     po += (uint64_t)Hq * L * L;
     cnt += (uint64_t)Hq * dam_cnt_stride(L, W, nL);
     lrows += (uint64_t)Hq * L;
+    gath += (uint64_t)Hq * nL;
     causal_tiles += (uint64_t)Hq * nq * (nq + 1) / 2;
     if (pcl_max > 0) {
       for (int qb = 0; qb < nq; ++qb) cap += (uint64_t)Hq * dam_row_tile_bound(qb, nL);
@@ -87,7 +96,8 @@ void compute_layout(const dam_shape_t* s, int pcl_max, int all_ones_causal, Layo
   h.magic = DAM_MAGIC;
   h.status = 0;
   h.version = 1;
-  h.flags = pcl_max > 0 ? DAM_FLAG_CAUSAL_LIST : (DAM_FLAG_ALL_ONES | (all_ones_causal ? DAM_FLAG_CAUSAL_LIST : 0u));
+  h.flags = pcl_max > 0 ? (DAM_FLAG_CAUSAL_LIST | (gather ? DAM_FLAG_GATHER : 0u))
+                        : (DAM_FLAG_ALL_ONES | (all_ones_causal ? DAM_FLAG_CAUSAL_LIST : 0u));
   h.num_seqs = s->num_seqs;
   h.num_q_heads = Hq;
   h.total_qblocks = total_qb;
@@ -113,7 +123,11 @@ void compute_layout(const dam_shape_t* s, int pcl_max, int all_ones_causal, Layo
   y.off_hist = dam_align(y.off_rowcnt + 4ull * h.rows, 256);
   y.off_cursor = y.off_hist + 4ull * DAM_HIST;
   y.build_scratch_bytes = dam_align(y.off_cursor + 4ull * DAM_HIST, 256);
-  y.attn_scratch_bytes = 256;
+  // attention scratch: 256-byte status block, then (gathered columns only) one K tile and one V tile of
+  // 128 keys per gathered-column tile
+  h.gath_tiles = (pcl_max > 0 && gather) ? gath : 0;
+  y.attn_scratch_bytes = 256 + h.gath_tiles * 2ull * DAM_TILE * s->head_dim * 2ull;
+  h.attn_scratch_bytes = y.attn_scratch_bytes;
   y.score_elems = po;
 }
 
@@ -159,7 +173,8 @@ dam_status_t fill_ctx(const dam_shape_t* s, const dam_rule_t* r, void* mask, siz
   if ((st = check_shape(s)) != DAM_OK) return st;
   if ((st = check_rule(r)) != DAM_OK) return st;
   if (!mask || !scratch || !aligned(mask, 256) || !aligned(scratch, 256)) return DAM_ERR_INVALID_ARGUMENT;
-  compute_layout(s, r->pcl_max, 1, y);
+  const int gather = gather_enabled(s, r);
+  compute_layout(s, r->pcl_max, 1, gather, y);
   if (cap < y->mask_bytes || scratch_bytes < y->build_scratch_bytes) return DAM_ERR_BUFFER_TOO_SMALL;
   c->blob = reinterpret_cast<unsigned char*>(mask);
   c->scratch = reinterpret_cast<unsigned char*>(scratch);
@@ -171,12 +186,9 @@ dam_status_t fill_ctx(const dam_shape_t* s, const dam_rule_t* r, void* mask, siz
   c->scale = r->softmax_scale > 0.f ? r->softmax_scale : 1.0f / sqrtf((float)s->head_dim);
   c->off_cnt = y->off_cnt; c->off_rowstat = y->off_rowstat; c->off_rowcnt = y->off_rowcnt;
   c->off_hist = y->off_hist; c->off_cursor = y->off_cursor;
+  c->gather = gather;
   c->off_true = y->hdr.off_true; c->true_bytes = y->hdr.off_tile_ptr - y->hdr.off_true;
   return DAM_OK;
-}
-
-bool sm100_shape(const dam_shape_t* s) {
-  return s->dtype == DAM_BF16 && s->head_dim == 128;
 }
 
 }  // namespace
@@ -204,7 +216,8 @@ dam_status_t dam_mask_sizes(const dam_shape_t* shape, const dam_rule_t* rule, in
   if ((st = check_shape(shape)) != DAM_OK) return st;
   if (rule && (st = check_rule(rule)) != DAM_OK) return st;
   Layout y;
-  compute_layout(shape, rule ? rule->pcl_max : 0, causal != 0, &y);
+  compute_layout(shape, rule ? rule->pcl_max : 0, causal != 0,
+                 gather_enabled(shape, rule), &y);
   if (mask_bytes) *mask_bytes = y.mask_bytes;
   if (build_scratch_bytes) *build_scratch_bytes = rule ? y.build_scratch_bytes : 0;
   if (attn_scratch_bytes) *attn_scratch_bytes = y.attn_scratch_bytes;
@@ -251,7 +264,7 @@ dam_status_t dam_mask_all_ones(const dam_shape_t* shape, int32_t causal, void* m
   if ((st = check_shape(shape)) != DAM_OK) return st;
   if (!mask || !aligned(mask, 256)) return DAM_ERR_INVALID_ARGUMENT;
   Layout y;
-  compute_layout(shape, 0, causal != 0, &y);
+  compute_layout(shape, 0, causal != 0, 0, &y);
   if (mask_capacity < y.mask_bytes) return DAM_ERR_BUFFER_TOO_SMALL;
   cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
   if (dam_launch_init_blob(shape, 0, y.hdr.flags, mask, y.hdr.tile_capacity, y.hdr, cs) != cudaSuccess)
@@ -276,7 +289,8 @@ dam_status_t dam_sparse_attention(const void* Q, const void* K, const void* V, c
   // status word and work counter start at zero
   if (cudaMemsetAsync(scratch, 0, 256, cs) != cudaSuccess) return DAM_ERR_CUDA;
   cudaError_t e = cudaErrorNotSupported;
-  if (sm100_shape(shape)) e = dam_launch_attn_sm100(Q, K, V, mask, shape, causal != 0, scale, O, lse, scratch, cs);
+  if (sm100_shape(shape))
+    e = dam_launch_attn_sm100(Q, K, V, mask, shape, causal != 0, scale, O, lse, scratch, scratch_bytes, cs);
   if (e == cudaErrorNotSupported) e = dam_launch_attn_ref(Q, K, V, mask, shape, causal != 0, scale, O, lse, scratch, cs);
   return e == cudaSuccess ? DAM_OK : DAM_ERR_CUDA;
 }
@@ -334,7 +348,7 @@ dam_status_t dam_prefill_host(const void* Qh, const void* Kh, const void* Vh, co
       shape->o_stride_head != d || shape->o_stride_tok != Hq * d)
     return DAM_ERR_UNSUPPORTED;
   Layout y;
-  compute_layout(shape, rule->pcl_max, 1, &y);
+  compute_layout(shape, rule->pcl_max, 1, gather_enabled(shape, rule), &y);
   const size_t qb = dam_align((size_t)T * Hq * d * es, 256), kb = dam_align((size_t)T * Hkv * d * es, 256);
   const size_t lb = dam_align((size_t)Hq * T * 4, 256);
   size_t off_q = 0, off_k = off_q + qb, off_v = off_k + kb, off_o = off_v + kb, off_l = off_o + qb;

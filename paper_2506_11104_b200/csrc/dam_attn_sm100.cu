@@ -41,9 +41,11 @@ struct SmemLayout {
   static constexpr int slots = 2 * kSlotBytes;
   static constexpr int stage = kSlotBytes * (2 + kSlots);           // two staging buffers (stream A, B)
   static constexpr int bars = stage + 2 * kStageBytes;
-  // q_full, q_empty, slot_full[kSlots], slot_empty[kSlots], s_full[2], p_full[2], o_final[2]
-  static constexpr int n_bars = 2 + 2 * kSlots + 6;
-  static constexpr int tmem_slot = bars + 8 * n_bars;
+  // q_full, q_empty, slot_full[kSlots], slot_empty[kSlots], s_full[2], p_full[2], o_final[2],
+  // sched_full[2], sched_empty[2]
+  static constexpr int n_bars = 2 + 2 * kSlots + 10;
+  static constexpr int sched_items = bars + 8 * n_bars;     // int[2]: work-list positions handed to the consumers
+  static constexpr int tmem_slot = sched_items + 8;
   static constexpr int abort_flag = tmem_slot + 4;
   static constexpr int total = abort_flag + 4;
 };
@@ -65,6 +67,8 @@ struct AttnParams {
   __nv_bfloat16* O;
   float* lse;
   uint32_t* status;         // scratch status word
+  uint32_t* work_counter;   // scratch word 2, zero at launch
+  unsigned long long scratch_bytes;
   int Hq, group, total_tokens, causal;
   int64_t o_stride_tok, o_stride_head;
   float scale_log2;         // softmax scale * log2(e)
@@ -101,12 +105,17 @@ struct Walker {
     ca = ia < ea ? __ldg(tiles + ia) : kNone;
     cb = ib < eb ? __ldg(tiles + ib) : kNone;
   }
+  // Order inside a row list: gathered-column tiles first (ascending index), then kv tiles (ascending).
+  static __device__ __forceinline__ uint32_t key(uint32_t e) {
+    if (e == kNone) return kNone;
+    return (e >> 28) == DAM_KIND_GATHERED ? (e & 0xFFFFu) : ((e & 0x0FFFFFFFu) | 0x10000000u);
+  }
+  // One step: kb = kv tile index, or gathered tile index when the kinds are DAM_KIND_GATHERED.
   __device__ __forceinline__ bool next(int& kb, uint32_t& kindA, uint32_t& kindB) {
-    const uint32_t ja = ca == kNone ? kNone : (ca & 0x0FFFFFFFu);
-    const uint32_t jb = cb == kNone ? kNone : (cb & 0x0FFFFFFFu);
+    const uint32_t ja = key(ca), jb = key(cb);
     const uint32_t k = ja < jb ? ja : jb;
     if (k == kNone) return false;
-    kb = (int)k;
+    kb = (int)(k & 0x0FFFFFFFu);
     kindA = (ja == k) ? (ca >> 28) : 0u;
     kindB = (jb == k) ? (cb >> 28) : 0u;
     if (ja == k) { ++ia; ca = ia < ea ? __ldg(tiles + ia) : kNone; }
@@ -242,7 +251,7 @@ __device__ __forceinline__ float sweep_exp(uint32_t tS, const uint4& bits, float
 __global__ void __launch_bounds__(kThreads, 1)
 attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                   const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
-                  const AttnParams prm) {
+                  const __grid_constant__ CUtensorMap tmG, const AttnParams prm) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t sbase = smem_u32(smem);
@@ -252,6 +261,8 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   const uint32_t bQFull = bar0, bQEmpty = bar0 + 8;
   const uint32_t bSlotFull = bar0 + 16, bSlotEmpty = bSlotFull + 8 * kSlots;
   const uint32_t bSFull = bSlotEmpty + 8 * kSlots, bPFull = bSFull + 16, bOFinal = bPFull + 16;
+  const uint32_t bSchedFull = bOFinal + 16, bSchedEmpty = bSchedFull + 16;
+  volatile int* sched_items = reinterpret_cast<volatile int*>(smem + SmemLayout::sched_items);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + SmemLayout::tmem_slot);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + SmemLayout::abort_flag);
 
@@ -260,20 +271,27 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   const DamHeader* H = reinterpret_cast<const DamHeader*>(blob);
   const int nitems = H->prows;
   const uint32_t* tiles = reinterpret_cast<const uint32_t*>(blob + H->off_tiles);
-  // The work list is sorted by length; CTAs take it in boustrophedon order (forward on even rounds, backward
-  // on odd rounds) so that no CTA gets the longest item of every round.
-  auto item_of_round = [&](int rnd) -> int {
-    const int G = (int)gridDim.x, c = (int)blockIdx.x;
-    return rnd * G + ((rnd & 1) ? (G - 1 - c) : c);
+  // a blob with gathered-column tiles needs the larger scratch; the gather kernel has recorded the error
+  if ((H->flags & DAM_FLAG_GATHER) && H->attn_scratch_bytes > prm.scratch_bytes) return;
+  // Dynamic scheduling: the work list is sorted longest first; the producer thread takes positions from a
+  // global counter (the first one is the CTA index) and hands each to the other roles through a two-entry
+  // ring in shared memory.  A negative position ends the loop.
+  auto next_item_consumer = [&](uint32_t n, bool arrive) -> int {
+    const uint32_t slot = n & 1u;
+    if (!mbar_wait(bSchedFull + 8 * slot, (n >> 1) & 1u, abort_flag)) return -2;
+    const int w = sched_items[slot];
+    if (arrive) mbar_arrive(bSchedEmpty + 8 * slot);
+    return w;
   };
 
   if (tid == 0) {
     mbar_init(bQFull, 1); mbar_init(bQEmpty, 1);
     for (int s = 0; s < kSlots; ++s) { mbar_init(bSlotFull + 8 * s, 1); mbar_init(bSlotEmpty + 8 * s, 1); }
     for (int s = 0; s < 2; ++s) { mbar_init(bSFull + 8 * s, 1); mbar_init(bPFull + 8 * s, 4); mbar_init(bOFinal + 8 * s, 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(bSchedFull + 8 * s, 1); mbar_init(bSchedEmpty + 8 * s, 9); }   // MMA thread + 8 softmax warps
     *abort_flag = 0u;
     mbar_fence_init();
-    tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); tma_prefetch_desc(&tmO);
+    tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); tma_prefetch_desc(&tmO); tma_prefetch_desc(&tmG);
   }
   if (warp == 0) { tmem_alloc(smem_u32(tmem_slot), kTmemCols); tmem_relinquish(); }
   tc_fence_before();
@@ -303,9 +321,15 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         ++sc;
         return true;
       };
-      for (int rnd = 0; ok; ++rnd) {
-        const int w = item_of_round(rnd);
-        if (w >= nitems) { if (rnd * (int)gridDim.x >= nitems) break; continue; }
+      for (uint32_t n = 0; ok; ++n) {
+        // claim the next position of the work list and publish it to the other roles
+        const uint32_t slot = n & 1u;
+        if (!(ok = mbar_wait(bSchedEmpty + 8 * slot, ((n >> 1) & 1u) ^ 1u, abort_flag))) break;
+        int w = n == 0 ? (int)blockIdx.x : (int)(gridDim.x + atomicAdd(prm.work_counter, 1u));
+        if (w >= nitems) w = -1;
+        sched_items[slot] = w;
+        mbar_arrive(bSchedFull + 8 * slot);
+        if (w < 0) break;
         const Item it = load_item(blob, H, w);
         if (it.a0 == it.b1) continue;                        // no tile in either list
         if (!(ok = mbar_wait(bQEmpty, (ic & 1u) ^ 1u, abort_flag))) break;
@@ -319,11 +343,23 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
         ++ic;
         const int kvh = it.head / prm.group;
+        // gathered-column tiles of this (sequence, head): K tile at rows (2T) * 128, V tile at (2T + 1) * 128
+        long long gtile0 = 0;
+        if (H->flags & DAM_FLAG_GATHER) {
+          const DamSeq* sqp = reinterpret_cast<const DamSeq*>(blob + H->off_seq) + it.seq;
+          gtile0 = (long long)sqp->gath_off + (long long)it.head * sqp->nL;
+        }
         Walker wk; wk.init(tiles, it);
         int kb; uint32_t kA, kB;
         while (ok && wk.next(kb, kA, kB)) {
-          ok = load_tile(&tmK, kvh, it.tok0 + kb * DAM_TILE);
-          if (ok) ok = load_tile(&tmV, kvh, it.tok0 + kb * DAM_TILE);
+          if (kA == DAM_KIND_GATHERED || kB == DAM_KIND_GATHERED) {
+            const int row = (int)((gtile0 + kb) * 2 * DAM_TILE);
+            ok = load_tile(&tmG, 0, row);
+            if (ok) ok = load_tile(&tmG, 0, row + DAM_TILE);
+          } else {
+            ok = load_tile(&tmK, kvh, it.tok0 + kb * DAM_TILE);
+            if (ok) ok = load_tile(&tmV, kvh, it.tok0 + kb * DAM_TILE);
+          }
         }
       }
       if (!ok) {
@@ -377,9 +413,9 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
         return true;
       };
-      for (int rnd = 0; ok; ++rnd) {
-        const int w = item_of_round(rnd);
-        if (w >= nitems) { if (rnd * (int)gridDim.x >= nitems) break; continue; }
+      for (uint32_t n = 0; ok; ++n) {
+        const int w = next_item_consumer(n, true);
+        if (w < 0) { ok = (w == -1); break; }
         const Item it = load_item(blob, H, w);
         if (it.a0 == it.b1) continue;
         Walker wk; wk.init(tiles, it);
@@ -454,9 +490,11 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     uint32_t cS = 0, cO = 0;
     bool ok = true;
     PROF_DECL(8)
-    for (int rnd = 0; ok; ++rnd) {
-        const int w = item_of_round(rnd);
-        if (w >= nitems) { if (rnd * (int)gridDim.x >= nitems) break; continue; }
+    for (uint32_t n = 0; ok; ++n) {
+      const int w = next_item_consumer(n, false);
+      __syncwarp();
+      if (lane == 0 && w != -2) mbar_arrive(bSchedEmpty + 8 * (n & 1u));    // the whole warp has read the entry
+      if (w < 0) { ok = (w == -1); break; }
       const Item it = load_item(blob, H, w);
       if (X == 1 && !it.hasB) continue;
       const int qb = it.qb0 + X;
@@ -480,8 +518,13 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       float l = 0.f;
       // the mask words of a tile come from global memory: they are fetched one tile ahead
       auto tile_bits = [&](uint32_t e, bool& need) -> uint4 {
-        const int kb = (int)(e & 0x0FFFFFFFu);
         const uint32_t kind = e >> 28;
+        if (kind == DAM_KIND_GATHERED) {       // all rows see the same columns: the first n of the tile
+          const int n = (int)((e >> 16) & 0xFFu) + 1;
+          need = n < DAM_TILE;
+          return row_valid ? dam_low_ones128(n) : make_uint4(0u, 0u, 0u, 0u);
+        }
+        const int kb = (int)(e & 0x0FFFFFFFu);
         need = (kind != DAM_KIND_FULL) || (prm.causal && kb >= qb) || ((kb + 1) * DAM_TILE > it.S);
         return need ? dam_apply_bits(hb, kind, i, kb, prm.causal) : make_uint4(~0u, ~0u, ~0u, ~0u);
       };
@@ -619,11 +662,75 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   if (warp == 0) tmem_dealloc(tmem, kTmemCols);
 }
 
+// Copies the K and V rows of the matched columns of every (sequence, head) into dense tiles of 128 keys in
+// the scratch buffer (K tile at rows (2T) * 128, V tile at rows (2T + 1) * 128 of a [rows][128] bf16 array;
+// T = gath_off + head * nL + g).  Rows past the last matched column are zero.  One block per tile, grid-stride.
+__global__ void __launch_bounds__(128)
+gather_columns_kernel(const unsigned char* __restrict__ blob, const __nv_bfloat16* __restrict__ K,
+                      const __nv_bfloat16* __restrict__ V, int Hq, int group, int64_t kst, int64_t ksh, int64_t vst,
+                      int64_t vsh, unsigned char* scratch, unsigned long long scratch_bytes) {
+  const DamHeader* H = reinterpret_cast<const DamHeader*>(blob);
+  if (!(H->flags & DAM_FLAG_GATHER)) return;
+  if (H->attn_scratch_bytes > scratch_bytes) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) atomicMax(reinterpret_cast<uint32_t*>(scratch) + 1, (uint32_t)DAM_ERR_BUFFER_TOO_SMALL);
+    return;
+  }
+  __shared__ int pref[1025];
+  __shared__ int col[DAM_TILE];
+  uint4* out = reinterpret_cast<uint4*>(scratch + 256);
+  const DamSeq* seqs = reinterpret_cast<const DamSeq*>(blob + H->off_seq);
+  const int tid = threadIdx.x;
+  for (long long T = blockIdx.x; T < (long long)H->gath_tiles; T += gridDim.x) {
+    int b = 0;
+    while (b + 1 < H->num_seqs && (long long)seqs[b + 1].gath_off <= T) ++b;
+    const DamSeq sq = seqs[b];
+    if (sq.nL == 0) continue;
+    const int h = (int)((T - (long long)sq.gath_off) / sq.nL), g = (int)((T - (long long)sq.gath_off) % sq.nL);
+    if (h >= Hq) continue;
+    const uint32_t* Vw = reinterpret_cast<const uint32_t*>(blob + H->off_dv) + sq.dv_off + (uint64_t)h * 3 * sq.W + 2 * sq.W;
+    // exclusive prefix popcounts of the V words (W <= 1024 words, i.e. windows up to 32768 tokens)
+    const int W = min(sq.W, 1024);
+    __syncthreads();
+    if (tid == 0) {
+      int a = 0;
+      for (int w = 0; w < W; ++w) { pref[w] = a; a += __popc(Vw[w]); }
+      pref[W] = a;
+    }
+    __syncthreads();
+    const int nV = pref[W];
+    if (g * DAM_TILE >= nV) continue;                         // capacity tile that no row list refers to
+    {
+      const int rank = g * DAM_TILE + tid;
+      int c = -1;
+      if (rank < nV) {
+        int lo = 0, hi = W;                                     // last word with pref <= rank
+        while (hi - lo > 1) { int mid = (lo + hi) >> 1; if (pref[mid] <= rank) lo = mid; else hi = mid; }
+        c = lo * 32 + (int)__fns(Vw[lo], 0, rank - pref[lo] + 1);
+      }
+      col[tid] = c;
+    }
+    __syncthreads();
+    const __nv_bfloat16* Kh = K + (int64_t)sq.tok_start * kst + (int64_t)(h / group) * ksh;
+    const __nv_bfloat16* Vh = V + (int64_t)sq.tok_start * vst + (int64_t)(h / group) * vsh;
+    const int part = tid & 15, r0 = tid >> 4;                   // 16 threads x 16 bytes per 256-byte row
+    for (int r = r0; r < DAM_TILE; r += 8) {
+      const int c = col[r];
+      uint4 kv = make_uint4(0u, 0u, 0u, 0u), vv = kv;
+      if (c >= 0) {
+        kv = __ldg(reinterpret_cast<const uint4*>(Kh + (int64_t)c * kst) + part);
+        vv = __ldg(reinterpret_cast<const uint4*>(Vh + (int64_t)c * vst) + part);
+      }
+      out[((size_t)(2 * T) * DAM_TILE + r) * 16 + part] = kv;
+      out[((size_t)(2 * T + 1) * DAM_TILE + r) * 16 + part] = vv;
+    }
+  }
+}
+
 }  // namespace
 
 cudaError_t dam_launch_attn_sm100(const void* Q, const void* K, const void* V, const void* blob,
                                   const dam_shape_t* s, int causal, float scale, void* O, float* lse, void* scratch,
-                                  cudaStream_t st) {
+                                  size_t scratch_bytes, cudaStream_t st) {
   if (s->dtype != DAM_BF16 || s->head_dim != 128) return cudaErrorNotSupported;
   if (s->total_tokens == 0) return cudaSuccess;
   static int sm_count = 0, smem_optin = 0;
@@ -640,7 +747,20 @@ cudaError_t dam_launch_attn_sm100(const void* Q, const void* K, const void* V, c
       return e;
     cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
   }
-  CUtensorMap tq, tk, tv, to;
+  // gathered-column tiles (if the blob has any) live after the 256-byte status block of the scratch buffer
+  const size_t grows = scratch_bytes > 256 ? (scratch_bytes - 256) / 256 : 0;      // rows of 128 bf16
+  CUtensorMap tq, tk, tv, to, tg;
+  const bool has_g = grows >= 2 * DAM_TILE;
+  if (!dam_make_tmap_bf16(&tg, has_g ? reinterpret_cast<const unsigned char*>(scratch) + 256 : Q, 128, 1,
+                          has_g ? (int64_t)grows : DAM_TILE, 128, 128))
+    return cudaErrorInvalidValue;
+  if (has_g) {
+    gather_columns_kernel<<<sm_count * 4, 128, 0, st>>>(
+        reinterpret_cast<const unsigned char*>(blob), reinterpret_cast<const __nv_bfloat16*>(K),
+        reinterpret_cast<const __nv_bfloat16*>(V), s->num_q_heads, s->num_q_heads / s->num_kv_heads, s->k_stride_tok,
+        s->k_stride_head, s->v_stride_tok, s->v_stride_head, reinterpret_cast<unsigned char*>(scratch),
+        (unsigned long long)scratch_bytes);
+  }
   if (!dam_make_tmap_bf16(&to, O, 128, s->num_q_heads, s->total_tokens, s->o_stride_tok, s->o_stride_head, 32) ||
       !dam_make_tmap_bf16(&tq, Q, 128, s->num_q_heads, s->total_tokens, s->q_stride_tok, s->q_stride_head) ||
       !dam_make_tmap_bf16(&tk, K, 128, s->num_kv_heads, s->total_tokens, s->k_stride_tok, s->k_stride_head) ||
@@ -658,12 +778,15 @@ cudaError_t dam_launch_attn_sm100(const void* Q, const void* K, const void* V, c
   p.O = reinterpret_cast<__nv_bfloat16*>(O);
   p.lse = lse;
   p.status = reinterpret_cast<uint32_t*>(scratch) + 1;
-  p.prof = reinterpret_cast<unsigned long long*>(reinterpret_cast<unsigned char*>(scratch) + 256);
+  p.work_counter = reinterpret_cast<uint32_t*>(scratch) + 2;
+  p.scratch_bytes = scratch_bytes;
+  // profile builds keep their cycle counters in the last 8 KiB of the scratch buffer
+  p.prof = reinterpret_cast<unsigned long long*>(reinterpret_cast<unsigned char*>(scratch) + (scratch_bytes >= 16384 ? scratch_bytes - 8192 : 256));
   p.Hq = s->num_q_heads; p.group = s->num_q_heads / s->num_kv_heads; p.total_tokens = s->total_tokens;
   p.causal = causal;
   p.o_stride_tok = s->o_stride_tok; p.o_stride_head = s->o_stride_head;
   p.scale_log2 = scale * 1.4426950408889634f;
   const int grid = pairs < sm_count ? pairs : sm_count;
-  attn_sm100_kernel<<<grid, kThreads, kSmemBytes, st>>>(tq, tk, tv, to, p);
+  attn_sm100_kernel<<<grid, kThreads, kSmemBytes, st>>>(tq, tk, tv, to, tg, p);
   return cudaGetLastError();
 }

@@ -31,8 +31,10 @@
 #define DAM_SCRATCH_MAGIC 0x534D4144u /* "DAMS" */
 #define DAM_KIND_FULL 1u
 #define DAM_KIND_PARTIAL 2u
+#define DAM_KIND_GATHERED 3u    /* entry = gathered tile index | (columns in it - 1) << 16 | kind << 28 */
 #define DAM_FLAG_ALL_ONES 1u
 #define DAM_FLAG_CAUSAL_LIST 2u    /* tile lists hold only kb <= qb */
+#define DAM_FLAG_GATHER 4u         /* rows from 2L-1 on list gathered-column tiles instead of vertical tiles */
 #define DAM_HIST 4096
 
 struct DamHeader {
@@ -54,7 +56,9 @@ struct DamHeader {
   uint64_t off_pairtab;
   int32_t total_pairs;      // sum over sequences of ceil(nq / 2)
   int32_t prows;            // num_q_heads * total_pairs
-  uint64_t reserved[15];
+  uint64_t gath_tiles;      // gathered-column tiles over all (seq, head): sum Hq * nL (capacity, 128 keys each)
+  uint64_t attn_scratch_bytes;   // scratch dam_sparse_attention needs for this blob
+  uint64_t reserved[13];
 };
 static_assert(sizeof(DamHeader) == 256, "DamHeader must be 256 bytes");
 
@@ -72,8 +76,10 @@ struct DamSeq {
   uint64_t true_off;   // u32 words from off_true: head h at true_off + h * L * W
   uint64_t p_off;      // fp32 elements into a score tensor: head h at p_off + h * L * L
   uint64_t cnt_off;    // int32 elements into the build scratch count area: head h at cnt_off + h * cnt_stride
+  uint64_t gath_off;   // gathered-column tiles: head h owns tiles [gath_off + h * nL, +nL)
+  uint64_t reserved;
 };
-static_assert(sizeof(DamSeq) == 64, "DamSeq must be 64 bytes");
+static_assert(sizeof(DamSeq) == 80, "DamSeq must be 80 bytes");
 
 // Per-(seq, head) words in the build scratch count area:
 //   cntD[L], cntV[L], prefD[W + 1], prefV[W + 1], tile_pop[nL * nL], padded to a multiple of 4.
@@ -90,12 +96,17 @@ __host__ __device__ inline int dam_row_tile_bound(int qb, int nL) {
   return a < b ? a : b;
 }
 
+// Gathered-column tiles serve the query blocks that start at or after row 2L - 1 (first multiple of 128).
+__host__ __device__ inline int dam_gather_first_qblock(int L) { return (2 * L - 1 + DAM_TILE - 1) / DAM_TILE; }
+__host__ __device__ inline int dam_gather_first_row(int L) { return dam_gather_first_qblock(L) * DAM_TILE; }
+
 struct DamHeadBits {
   const uint32_t* D;
   const uint32_t* Drev;
   const uint32_t* V;
   const uint32_t* M;
   int L, W, S;
+  int gather_from;     // first row whose matched columns are served by gathered tiles (INT_MAX: none)
 };
 
 __device__ __forceinline__ DamHeadBits dam_head_bits(const unsigned char* blob, const DamHeader* hdr,
@@ -109,6 +120,7 @@ __device__ __forceinline__ DamHeadBits dam_head_bits(const unsigned char* blob, 
   hb.L = sq.L;
   hb.W = sq.W;
   hb.S = sq.S;
+  hb.gather_from = (hdr->flags & DAM_FLAG_GATHER) ? dam_gather_first_row(sq.L) : 0x7FFFFFFF;
   return hb;
 }
 
@@ -132,7 +144,7 @@ __device__ __forceinline__ uint4 dam_tile_row_bits(const DamHeadBits& hb, int i,
   if (i < hb.L) {
     if (j0 < hb.L) r = __ldg(reinterpret_cast<const uint4*>(hb.M + (size_t)i * hb.W + kb * 4));
   } else {
-    if (j0 < hb.L) r = __ldg(reinterpret_cast<const uint4*>(hb.V + kb * 4));
+    if (j0 < hb.L && i < hb.gather_from) r = __ldg(reinterpret_cast<const uint4*>(hb.V + kb * 4));
     const int x0 = hb.L - 1 - i + j0;
     if (x0 + DAM_TILE > 0 && x0 < hb.L) {
       r.x |= dam_window32(hb.Drev, hb.W, x0);
@@ -180,6 +192,7 @@ struct DamBuildCtx {
   float mu;
   int min_support;
   float scale;
+  int gather;        // list gathered-column tiles
   uint64_t off_cnt, off_rowstat, off_rowcnt, off_hist, off_cursor;   // scratch sections
   uint64_t off_true, true_bytes;                                     // true-mask section of the blob
 };
@@ -199,6 +212,6 @@ cudaError_t dam_launch_attn_ref(const void* Q, const void* K, const void* V, con
 // tensor-core paths (bf16, d = 128); return cudaErrorNotSupported when the shape does not qualify
 cudaError_t dam_launch_attn_sm100(const void* Q, const void* K, const void* V, const void* blob,
                                   const dam_shape_t* shape, int causal, float scale, void* O, float* lse,
-                                  void* scratch, cudaStream_t st);
+                                  void* scratch, size_t scratch_bytes, cudaStream_t st);
 cudaError_t dam_launch_scores_sm100(const void* Q, const void* K, const dam_shape_t* shape, const DamBuildCtx& c,
                                     float* scores_dump, cudaStream_t st);

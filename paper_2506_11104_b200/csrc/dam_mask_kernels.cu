@@ -23,7 +23,7 @@ __global__ void init_blob_kernel(unsigned char* blob, DamHeader hdr, const int32
   uint32_t* pairtab = reinterpret_cast<uint32_t*>(blob + hdr.off_pairtab);
   if (threadIdx.x == 0) {
     *H = hdr;
-    uint64_t dv = 0, tr = 0, po = 0, co = 0;
+    uint64_t dv = 0, tr = 0, po = 0, co = 0, go = 0;
     int fq = 0, fp = 0;
     for (int b = 0; b < hdr.num_seqs; ++b) {
       int t0 = cu[b], S = cu[b + 1] - t0;
@@ -35,13 +35,14 @@ __global__ void init_blob_kernel(unsigned char* blob, DamHeader hdr, const int32
       DamSeq s;
       s.tok_start = t0; s.S = S; s.L = L; s.nq = nq;
       s.first_qblock = fq; s.W = W; s.nL = nL; s.first_pair = fp;
-      s.dv_off = dv; s.true_off = tr; s.p_off = po; s.cnt_off = co;
+      s.dv_off = dv; s.true_off = tr; s.p_off = po; s.cnt_off = co; s.gath_off = go; s.reserved = 0;
       seqs[b] = s;
       dv += (uint64_t)Hq * 3 * W;
       tr += (uint64_t)Hq * L * W;
       po += (uint64_t)Hq * L * L;
       if (all_ones_causal < 0) co += (uint64_t)Hq * dam_cnt_stride(L, W, nL);
       else co += all_ones_causal ? (uint64_t)nq * (nq + 1) / 2 : (uint64_t)nq * nq;   // tile base per head
+      go += (uint64_t)Hq * nL;
       fq += nq;
       fp += (nq + 1) / 2;
     }
@@ -256,6 +257,21 @@ __device__ __forceinline__ uint32_t classify_tile(const HeadView& v, int qb, int
   return act ? (full ? DAM_KIND_FULL : DAM_KIND_PARTIAL) : 0u;
 }
 
+// Rows from 2L - 1 on with gathered columns: only the matched diagonals count (their keys are all >= L - 1
+// while every matched column is < L and served by the gathered tiles).
+__device__ __forceinline__ uint32_t classify_band(const HeadView& v, int qb, int kb) {
+  const int i0 = qb * DAM_TILE;
+  const int i1 = min(i0 + DAM_TILE, v.S);
+  const int j0 = kb * DAM_TILE;
+  const int rlo = i0 - (j0 + DAM_TILE - 1), rhi = (i1 - 1) - j0;
+  const int clo = max(rlo, 0), chi = min(rhi, v.L - 1);
+  if (clo > chi) return 0u;
+  const int n = cnt_range(v.Dw, v.prefD, clo, chi);
+  if (n == 0) return 0u;
+  const bool whole = (i1 - i0 == DAM_TILE) && (kb < qb) && clo == rlo && chi == rhi;
+  return (whole && n == 2 * DAM_TILE - 1) ? DAM_KIND_FULL : DAM_KIND_PARTIAL;
+}
+
 template <int PASS>
 __global__ void classify_kernel(unsigned char* blob, unsigned char* scratch, uint64_t off_cnt, uint64_t off_rowcnt,
                                 uint64_t off_hist, uint64_t off_cursor) {
@@ -283,9 +299,13 @@ __global__ void classify_kernel(unsigned char* blob, unsigned char* scratch, uin
     const int gqb = gqb0 + x;
     const int row = h * H->total_qblocks + gqb;
     const int qb = gqb - sq.first_qblock;
-    // candidates, ascending: [0, min(qb, nL-1)] then [max(that + 1, qb - nL), qb]
-    const int n1 = min(qb, sq.nL - 1) + 1;
-    const int lo2 = max(n1, qb - sq.nL);
+    // candidates, ascending: [0, min(qb, nL-1)] then [max(that + 1, qb - nL), qb].  From row 2L - 1 on
+    // (gathered columns enabled) the first range is replaced by the gathered tiles and the second range
+    // is classified on the matched diagonals alone.
+    const bool gathered = (H->flags & DAM_FLAG_GATHER) && sq.L > 0 && qb >= dam_gather_first_qblock(sq.L);
+    const int nV = gathered ? v.prefV[sq.W] : 0;
+    const int n1 = gathered ? (nV + DAM_TILE - 1) / DAM_TILE : min(qb, sq.nL - 1) + 1;
+    const int lo2 = gathered ? max(0, qb - sq.nL) : max(n1, qb - sq.nL);
     const int n2 = max(0, qb - lo2 + 1);
     uint32_t base = 0;
     bool write = PASS == 1;
@@ -296,18 +316,23 @@ __global__ void classify_kernel(unsigned char* blob, unsigned char* scratch, uin
     int total = 0;
     for (int c0 = 0; c0 < n1 + n2; c0 += 32) {
       int idx = c0 + lane;
-      uint32_t kind = 0;
-      int kb = 0;
+      uint32_t kind = 0, entry = 0;
       if (idx < n1 + n2) {
-        kb = idx < n1 ? idx : lo2 + (idx - n1);
-        kind = classify_tile(v, qb, kb);
+        if (gathered && idx < n1) {
+          kind = DAM_KIND_GATHERED;
+          entry = (uint32_t)idx | ((uint32_t)(min(DAM_TILE, nV - idx * DAM_TILE) - 1) << 16) | (kind << 28);
+        } else {
+          const int kb = idx < n1 ? idx : lo2 + (idx - n1);
+          kind = gathered ? classify_band(v, qb, kb) : classify_tile(v, qb, kb);
+          entry = (uint32_t)kb | (kind << 28);
+        }
       }
       uint32_t m = __ballot_sync(0xFFFFFFFFu, kind != 0);
       if (write && kind) {
         int rank = __popc(m & ((1u << lane) - 1u));
-        tiles[base + total + rank] = (uint32_t)kb | (kind << 28);
+        tiles[base + total + rank] = entry;
       }
-      if (PASS == 1) nfull += __popc(__ballot_sync(0xFFFFFFFFu, kind == DAM_KIND_FULL));
+      if (PASS == 1) nfull += __popc(__ballot_sync(0xFFFFFFFFu, kind == DAM_KIND_FULL || (kind == DAM_KIND_GATHERED && ((entry >> 16) & 0xFFu) == DAM_TILE - 1)));
       total += __popc(m);
     }
     if (PASS == 0 && lane == 0) rowcnt[row] = total;
@@ -464,10 +489,37 @@ __global__ void expand_rows_kernel(const unsigned char* blob, int seq, int head,
   DamHeadBits hb = dam_head_bits(blob, H, sq, head);
   for (uint32_t t = tile_ptr[row] + threadIdx.x; t < tile_ptr[row + 1]; t += blockDim.x) {
     uint32_t e = tiles[t];
+    if ((e >> 28) == DAM_KIND_GATHERED) continue;          // handled below
     int kb = (int)(e & 0x0FFFFFFFu);
     uint4 bits = dam_apply_bits(hb, e >> 28, i, kb, causal);
     if (kb * 4 + 3 < words) {
-      o[kb * 4 + 0] = bits.x; o[kb * 4 + 1] = bits.y; o[kb * 4 + 2] = bits.z; o[kb * 4 + 3] = bits.w;
+      atomicOr(&o[kb * 4 + 0], bits.x); atomicOr(&o[kb * 4 + 1], bits.y);
+      atomicOr(&o[kb * 4 + 2], bits.z); atomicOr(&o[kb * 4 + 3], bits.w);
+    }
+  }
+  // gathered tiles: together they hold exactly the matched columns, in ascending order, 128 per tile
+  const uint32_t r0 = tile_ptr[row], r1 = tile_ptr[row + 1];
+  int ngath = 0, ncols = 0;
+  for (uint32_t t = r0; t < r1; ++t) {
+    uint32_t e = tiles[t];
+    if ((e >> 28) != DAM_KIND_GATHERED) break;
+    ++ngath;
+    ncols += (int)((e >> 16) & 0xFFu) + 1;
+  }
+  if (ngath) {
+    // the first `ncols` set bits of V, as words
+    int seen = 0;
+    for (int w = 0; w < sq.W && w < words; ++w) {
+      uint32_t vw = hb.V[w];
+      int pc = __popc(vw);
+      if (seen + pc > ncols) {              // keep only the lowest (ncols - seen) set bits
+        uint32_t keep = 0u;
+        for (int k = 0; k < ncols - seen; ++k) { uint32_t low = vw & (0u - vw); keep |= low; vw ^= low; }
+        vw = keep; pc = ncols - seen;
+      }
+      if (threadIdx.x == 0 && vw) atomicOr(&o[w], vw);
+      seen += pc;
+      if (seen >= ncols) break;
     }
   }
 }

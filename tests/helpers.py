@@ -86,11 +86,26 @@ def check_blob_against_oracle(blob, shape, masks, qblocks_per_head=None, rng=Non
                            min(nq - 1, (2 * L - 1) // TILE + 1)}
                 extra = rng.choice(nq, size=max(0, qblocks_per_head - len(special)), replace=False)
                 qbs = sorted(special | set(int(x) for x in extra))
+            gather = bool(int(mb.hdr["flags"]) & 4)
+            L = hm.L
+            g_first = (2 * L - 1 + TILE - 1) // TILE if (gather and L > 0) else 1 << 30
+            nV = int(hm.V.sum())
             for qb in qbs:
                 i0, i1 = qb * TILE, min(S, qb * TILE + TILE)
                 rows = hm.rows(list(range(i0, i1)))
-                want, full = nonempty_tiles(rows, S)
                 kbs, kinds = mb.row_tiles(b, h, qb)
+                if qb >= g_first:
+                    # gathered-column tiles first: ceil(nV / 128) of them, holding the matched columns in order
+                    ng = (nV + TILE - 1) // TILE
+                    ent = mb.row_entries(b, h, qb)
+                    assert np.array_equal(kinds[:ng], np.full(ng, 3)) and np.array_equal(kbs[:ng], np.arange(ng))
+                    assert all(int((e >> 16) & 0xFF) + 1 == min(TILE, nV - g * TILE) for g, e in enumerate(ent[:ng]))
+                    band = rows.copy()
+                    band[:, :L][:, hm.V.astype(bool)] = 0          # columns served by the gathered tiles
+                    want, full = nonempty_tiles(band, S)
+                    kbs, kinds = kbs[ng:], kinds[ng:]
+                else:
+                    want, full = nonempty_tiles(rows, S)
                 assert np.array_equal(kbs, want), f"tile list differs seq {b} head {h} qb {qb}: {kbs} vs {want}"
                 for kb, kind in zip(kbs, kinds):
                     assert kind in (1, 2)

@@ -67,9 +67,9 @@ def test_all_ones_mask_is_dense_attention(lengths, Hq, Hkv, d, dtype, causal):
     _check(w, O, lse, None, _all_rows, causal=causal, all_ones=True)
 
 
-def _masked_case(w, rows_for, heads=None):
+def _masked_case(w, rows_for, heads=None, gather=False):
     shape = _shape(w)
-    rule = B.make_rule(w.pcl_max, w.tau, w.mu, w.lam, w.eps)
+    rule = B.make_rule(w.pcl_max, w.tau, w.mu, w.lam, w.eps, gather_columns=gather)
     n = sum(w.num_q_heads * min(S, w.pcl_max) ** 2 for S in shape.lengths)
     dump = torch.zeros(n, dtype=torch.float32, device=DEV)
     blob, _ = B.dam_build_masks(w.Q.to(DEV), w.K.to(DEV), shape, rule, scores_dump=dump)
@@ -93,9 +93,10 @@ def test_config0_every_row():
     ([1500, 130], 256, 8, 2, 128, torch.bfloat16),
     ([513], 300, 2, 2, 32, torch.float32),
 ])
-def test_masked_small_cases_every_row(lengths, pcl, Hq, Hkv, d, dtype):
+@pytest.mark.parametrize("gather", [False, True])
+def test_masked_small_cases_every_row(lengths, pcl, Hq, Hkv, d, dtype, gather):
     w = synth.small_case(0, Hq, Hkv, d, pcl, seed=11, dtype=dtype, lengths=lengths)
-    _masked_case(w, _all_rows)
+    _masked_case(w, _all_rows, gather=gather)
 
 
 def test_empty_rows_and_no_patterns():
@@ -106,9 +107,10 @@ def test_empty_rows_and_no_patterns():
     assert torch.isneginf(lse[:, 128:]).all() and (O[128:] == 0).all()
 
 
-def test_config1_sampled_rows():
+@pytest.mark.parametrize("gather", [False, True])
+def test_config1_sampled_rows(gather):
     w = synth.config1()
-    _masked_case(w, _sample_rows(1024), heads=[0, 5, 13, 22, 31])
+    _masked_case(w, _sample_rows(1024), heads=[0, 5, 13, 22, 31], gather=gather)
 
 
 def test_config1_dense_causal_sampled_rows():
@@ -119,15 +121,16 @@ def test_config1_dense_causal_sampled_rows():
     _check(w, O, lse, None, lambda S: [0, 1, 127, 128, 4095, 8191], heads=[3, 30], all_ones=True)
 
 
-def test_config4_varlen_sampled_rows():
+@pytest.mark.parametrize("gather", [False, True])
+def test_config4_varlen_sampled_rows(gather):
     w = synth.config4()
-    _masked_case(w, _sample_rows(1024), heads=[2, 17])
+    _masked_case(w, _sample_rows(1024), heads=[2, 17], gather=gather)
 
 
 def test_config2_layer_sampled_rows():
     """One layer of the 32-layer stack (32768 tokens, PCL 2048), in the launch configuration the benchmark times."""
     w = synth.config2_layer(5, DEV)
-    blob, shape, masks, O, lse, worst = _masked_case(w, _sample_rows(2048), heads=[1, 12, 27])
+    blob, shape, masks, O, lse, worst = _masked_case(w, _sample_rows(2048), heads=[1, 12, 27], gather=True)
     st = B.dam_mask_stats(blob, shape)
     assert 0.01 <= st["tiles"] / st["causal_tiles"] <= 0.30
 
@@ -135,4 +138,17 @@ def test_config2_layer_sampled_rows():
 def test_config3_sampled_rows():
     """131072 tokens, PCL 4096: sampled rows of a few heads against the oracle over all 131072 keys."""
     w = synth.config3(DEV)
-    _masked_case(w, _sample_rows(4096), heads=[4, 19])
+    _masked_case(w, _sample_rows(4096), heads=[4, 19], gather=True)
+
+
+def test_gathered_blob_with_small_scratch_reports_error():
+    """A blob with gathered-column tiles needs the larger scratch; a 256-byte scratch is refused on the device."""
+    w = synth.small_case(0, 4, 2, 128, 128, seed=4, lengths=[900])
+    shape = _shape(w)
+    rule = B.make_rule(w.pcl_max, w.tau, w.mu, gather_columns=True)
+    blob, _ = B.dam_build_masks(w.Q.to(DEV), w.K.to(DEV), shape, rule)
+    assert B.dam_mask_sizes(shape, rule)[2] > 256
+    small = torch.zeros(256 + 70000, dtype=torch.uint8, device=DEV)[:256 + 65536]
+    O, lse, scr = B.dam_sparse_attention(w.Q.to(DEV), w.K.to(DEV), w.V.to(DEV), blob, shape, scratch=small)
+    torch.cuda.synchronize()
+    assert B.dam_poll_status(scr) == 3
