@@ -173,10 +173,12 @@ dam_status_t dam_sparse_attention(const void* Q, const void* K, const void* V, c
                                   size_t scratch_bytes, void* stream);
 
 /*
- * Counts taken from a mask blob (DEVICE): out[0] = listed tiles, out[1] = tiles listed as fully
- * active, out[2] = total causal tiles of the shape (for densities), out[3] = bytes of the blob in
- * use. `out` is HOST memory (4 x uint64). Synchronises `stream`. The paper reports no such counts;
- * they feed the density and active-FLOP figures of the benchmark.
+ * Counts taken from a mask blob (DEVICE): out[0] = listed tiles (what the attention kernel executes),
+ * out[1] = of those, fully active ones, out[2] = total causal tiles of the shape (for densities),
+ * out[3] = bytes of the blob in use, out[4] = 128 x 128 tiles of the masks themselves that hold an
+ * active cell (equals out[0] unless gathered-column tiles are listed). `out` is HOST memory
+ * (5 x uint64). Synchronises `stream`. The paper reports no such counts; they feed the density and
+ * active-FLOP figures of the benchmark.
  */
 dam_status_t dam_mask_stats(const void* mask, const dam_shape_t* shape, uint64_t* out,
                             void* stream);

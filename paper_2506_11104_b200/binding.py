@@ -224,10 +224,11 @@ def dam_sparse_attention(Q, K, V, mask, shape: Shape, causal: bool = True, softm
 
 
 def dam_mask_stats(mask: torch.Tensor, shape: Shape) -> dict:
-    out = (ctypes.c_uint64 * 4)()
+    out = (ctypes.c_uint64 * 5)()
     rc = lib().dam_mask_stats(_ptr(mask), shape.ref, out, _stream(mask.device))
     _check(rc, "dam_mask_stats")
-    return {"tiles": int(out[0]), "full_tiles": int(out[1]), "causal_tiles": int(out[2]), "bytes_used": int(out[3])}
+    return {"tiles": int(out[0]), "full_tiles": int(out[1]), "causal_tiles": int(out[2]), "bytes_used": int(out[3]),
+            "mask_tiles": int(out[4])}
 
 
 def dam_mask_expand_rows(mask: torch.Tensor, shape: Shape, seq: int, head: int, row_begin: int, nrows: int,
@@ -265,7 +266,7 @@ _HDR = np.dtype([("magic", "<u4"), ("status", "<u4"), ("version", "<u4"), ("flag
                  ("off_seq", "<u8"), ("off_qbseq", "<u8"), ("off_dv", "<u8"), ("off_true", "<u8"),
                  ("off_tile_ptr", "<u8"), ("off_work", "<u8"), ("off_tiles", "<u8"), ("bytes_used", "<u8"),
                  ("causal_tiles", "<u8"), ("off_pairtab", "<u8"), ("total_pairs", "<i4"), ("prows", "<i4"),
-                 ("gath_tiles", "<u8"), ("attn_scratch_bytes", "<u8"), ("reserved", "<u8", (13,))])
+                 ("gath_tiles", "<u8"), ("attn_scratch_bytes", "<u8"), ("mask_tiles", "<u8"), ("reserved", "<u8", (12,))])
 _SEQ = np.dtype([("tok_start", "<i4"), ("S", "<i4"), ("L", "<i4"), ("nq", "<i4"), ("first_qblock", "<i4"),
                  ("W", "<i4"), ("nL", "<i4"), ("first_pair", "<i4"), ("dv_off", "<u8"), ("true_off", "<u8"),
                  ("p_off", "<u8"), ("cnt_off", "<u8"), ("gath_off", "<u8"), ("reserved", "<u8")])

@@ -303,6 +303,7 @@ dam_status_t dam_mask_stats(const void* mask, const dam_shape_t* shape, uint64_t
   if (cudaStreamSynchronize(cs) != cudaSuccess) return DAM_ERR_CUDA;
   if (h.magic != DAM_MAGIC) return DAM_ERR_INVALID_ARGUMENT;
   out[0] = h.total_tiles; out[1] = h.full_tiles; out[2] = h.causal_tiles; out[3] = h.bytes_used;
+  out[4] = h.mask_tiles;
   return DAM_OK;
 }
 

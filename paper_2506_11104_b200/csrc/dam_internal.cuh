@@ -58,7 +58,8 @@ struct DamHeader {
   int32_t prows;            // num_q_heads * total_pairs
   uint64_t gath_tiles;      // gathered-column tiles over all (seq, head): sum Hq * nL (capacity, 128 keys each)
   uint64_t attn_scratch_bytes;   // scratch dam_sparse_attention needs for this blob
-  uint64_t reserved[13];
+  uint64_t mask_tiles;      // 128 x 128 tiles of the masks that hold an active cell (= total_tiles unless gathered)
+  uint64_t reserved[12];
 };
 static_assert(sizeof(DamHeader) == 256, "DamHeader must be 256 bytes");
 

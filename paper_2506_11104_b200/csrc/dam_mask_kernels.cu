@@ -294,7 +294,7 @@ __global__ void classify_kernel(unsigned char* blob, unsigned char* scratch, uin
   uint32_t* rowcnt = reinterpret_cast<uint32_t*>(scratch + off_rowcnt);
   uint32_t* tile_ptr = reinterpret_cast<uint32_t*>(blob + H->off_tile_ptr);
   uint32_t* tiles = reinterpret_cast<uint32_t*>(blob + H->off_tiles);
-  int pair_total = 0, nfull = 0;
+  int pair_total = 0, nfull = 0, mask_tiles = 0;
   for (int x = 0; x < nblk; ++x) {
     const int gqb = gqb0 + x;
     const int row = h * H->total_qblocks + gqb;
@@ -337,11 +337,26 @@ __global__ void classify_kernel(unsigned char* blob, unsigned char* scratch, uin
     }
     if (PASS == 0 && lane == 0) rowcnt[row] = total;
     pair_total += total;
+    if (PASS == 0) {
+      // tiles of the mask itself (128 x 128 grid) with an active cell: equals `total` unless gathered
+      int nat = total;
+      if (gathered) {
+        nat = 0;
+        const int m1 = min(qb, sq.nL - 1) + 1, l2 = max(m1, qb - sq.nL), m2 = max(0, qb - l2 + 1);
+        for (int c0 = 0; c0 < m1 + m2; c0 += 32) {
+          const int idx = c0 + lane;
+          const bool act = idx < m1 + m2 && classify_tile(v, qb, idx < m1 ? idx : l2 + (idx - m1)) != 0u;
+          nat += __popc(__ballot_sync(0xFFFFFFFFu, act));
+        }
+      }
+      mask_tiles += nat;
+    }
   }
   if (lane == 0) {
     const int key = min(pair_total, DAM_HIST - 1);
     if (PASS == 0) {
       atomicAdd(reinterpret_cast<uint32_t*>(scratch + off_hist) + key, 1u);
+      atomicAdd(reinterpret_cast<unsigned long long*>(&H->mask_tiles), (unsigned long long)mask_tiles);
     } else {
       uint32_t pos = atomicAdd(reinterpret_cast<uint32_t*>(scratch + off_cursor) + key, 1u);
       const int rowA = h * H->total_qblocks + gqb0;
@@ -463,6 +478,7 @@ __global__ void all_ones_kernel(unsigned char* blob, int causal) {
       tile_ptr[H->rows] = tot;
       H->total_tiles = tot;
       H->full_tiles = tot;
+      H->mask_tiles = tot;
       H->bytes_used = H->off_tiles + 4ull * tot;
     }
   }

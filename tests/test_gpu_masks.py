@@ -216,3 +216,16 @@ def test_config3_shape_masks():
     blob, shape, masks, dump = _build_and_check(w, qblocks=8)
     st = B.dam_mask_stats(blob, shape)
     assert 0.005 <= st["tiles"] / st["causal_tiles"] <= 0.08
+
+
+def test_mask_tile_count_is_independent_of_gathering():
+    """The 128 x 128 tiles of the mask with an active cell are counted the same whether matched columns are
+    listed as vertical tiles or served by gathered-column tiles; the executed tile list shrinks."""
+    w = synth.config1()
+    shape = _shape(w)
+    Q, K = w.Q.to(DEV), w.K.to(DEV)
+    plain, _ = B.dam_build_masks(Q, K, shape, _rule(w))
+    gath, _ = B.dam_build_masks(Q, K, shape, _rule(w, gather_columns=True))
+    a, b = B.dam_mask_stats(plain, shape), B.dam_mask_stats(gath, shape)
+    assert a["mask_tiles"] == a["tiles"] == b["mask_tiles"]
+    assert b["tiles"] < a["tiles"]
