@@ -410,20 +410,39 @@ __global__ void scan_kernel(unsigned char* blob, unsigned char* scratch, uint64_
   const uint32_t* rowcnt = reinterpret_cast<const uint32_t*>(scratch + off_rowcnt);
   uint32_t* tile_ptr = reinterpret_cast<uint32_t*>(blob + H->off_tile_ptr);
   const int rows = H->rows;
-  // every thread owns a run of consecutive rows: one block-wide scan over the per-thread sums
+  // every warp owns a contiguous segment of rows and walks it 32 rows at a time (coalesced): first the
+  // segment totals, one block-wide scan over them, then the rows again with the segment's base
   {
-    const int per = (rows + blockDim.x - 1) / blockDim.x;
-    const int r0 = threadIdx.x * per, r1 = min(rows, r0 + per);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    const int seg = ((rows + nw - 1) / nw + 31) & ~31;
+    const int r0 = warp * seg, r1 = min(rows, r0 + seg);
     uint32_t local = 0;
-    for (int r = r0; r < r1; ++r) local += rowcnt[r];
-    uint32_t e = block_excl_scan(local, &tot, sm);
-    for (int r = r0; r < r1; ++r) { tile_ptr[r] = e; e += rowcnt[r]; }
+    for (int r = r0 + lane; r < r1; r += 32) local += rowcnt[r];
+#pragma unroll
+    for (int o = 16; o; o >>= 1) local += __shfl_xor_sync(0xFFFFFFFFu, local, o);
+    __shared__ uint32_t seg_base[32];
+    uint32_t e = block_excl_scan(lane == 0 ? local : 0u, &tot, sm);
+    if (lane == 0) seg_base[warp] = e;
+    __syncthreads();
+    uint32_t run = seg_base[warp];
+    for (int rb = r0; rb < r1; rb += 32) {
+      const int r = rb + lane;
+      const uint32_t x = r < r1 ? rowcnt[r] : 0u;
+      uint32_t inc = x;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+        if (lane >= o) inc += y;
+      }
+      if (r < r1) tile_ptr[r] = run + inc - x;
+      run += __shfl_sync(0xFFFFFFFFu, inc, 31);
+    }
     if (threadIdx.x == 0) {
-      const uint32_t run = tot;
-      tile_ptr[rows] = run;
-      H->total_tiles = run;
-      H->bytes_used = H->off_tiles + 4ull * run;
-      if (run > H->tile_capacity) H->status = DAM_ERR_BUFFER_TOO_SMALL;
+      const uint32_t total = tot;
+      tile_ptr[rows] = total;
+      H->total_tiles = total;
+      H->bytes_used = H->off_tiles + 4ull * total;
+      if (total > H->tile_capacity) H->status = DAM_ERR_BUFFER_TOO_SMALL;
     }
     __syncthreads();
   }

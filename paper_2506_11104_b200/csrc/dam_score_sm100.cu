@@ -2,7 +2,8 @@
 //
 // For every (sequence, query head) the causal softmax map over the first L tokens is computed tile by
 // tile and thresholded straight into the bit-packed true mask (paper Sec. 4.2.1 - 4.2.3); the map itself
-// is never stored unless the caller asks for the fp32 dump.  A work item is one 128-row query block of
+// is never stored unless the caller asks for the fp32 dump.  Four S buffers in TMEM let the MMA warp run two
+// tiles ahead of each softmax group.  A work item is one 128-row query block of
 // one (sequence, head).  Two sweeps over its kv tiles kb = 0 .. qb:
 //   sweep A  S = Q K^T (tcgen05, accumulator in TMEM) -> per-row running max and sum;
 //   sweep B  S again -> p = exp2(x - max) / sum in fp32 -> bit = [p >= p*] -> one 16-byte store of the
@@ -23,15 +24,17 @@ namespace {
 constexpr int kSlots = 5;
 constexpr int kSlotBytes = 32768;
 constexpr int kThreads = 320;
-constexpr uint32_t kTmemCols = 256;
+constexpr uint32_t kTmemCols = 512;       // four S buffers: tile g uses buffer g & 3, group g & 1 owns buffers {G, G + 2}
 
 struct SmemLayout {
   static constexpr int q = 0;
   static constexpr int slots = kSlotBytes;
   static constexpr int bars = kSlotBytes * (1 + kSlots);
-  // q_full, q_empty, slot_full[kSlots], slot_empty[kSlots], s_full[2], s_empty[2], stat_ready
-  static constexpr int n_bars = 2 + 2 * kSlots + 5;
-  static constexpr int stat = bars + 8 * n_bars;            // float2 [2][2][128]
+  // q_full, q_empty, slot_full[kSlots], slot_empty[kSlots], s_full[4], s_empty[4], stat_ready,
+  // sched_full[2], sched_empty[2]
+  static constexpr int n_bars = 2 + 2 * kSlots + 13;
+  static constexpr int sched_items = bars + 8 * n_bars;     // int[2]
+  static constexpr int stat = sched_items + 8;              // float2 [2][2][128]
   static constexpr int tmem_slot = stat + 2 * 2 * 128 * 8;
   static constexpr int abort_flag = tmem_slot + 4;
   static constexpr int total = abort_flag + 4;
@@ -42,6 +45,7 @@ struct ScoreParams {
   unsigned char* blob;
   float* dump;
   uint32_t* status;
+  uint32_t* work_counter;     // zero at launch
   int num_seqs, Hq, group, max_nL;
   float scale_log2, pstar;
 };
@@ -86,7 +90,9 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   const uint32_t bar0 = sbase + SmemLayout::bars;
   const uint32_t bQFull = bar0, bQEmpty = bar0 + 8;
   const uint32_t bSlotFull = bar0 + 16, bSlotEmpty = bSlotFull + 8 * kSlots;
-  const uint32_t bSFull = bSlotEmpty + 8 * kSlots, bSEmpty = bSFull + 16, bStat = bSEmpty + 16;
+  const uint32_t bSFull = bSlotEmpty + 8 * kSlots, bSEmpty = bSFull + 32, bStat = bSEmpty + 32;
+  const uint32_t bSchedFull = bStat + 8, bSchedEmpty = bSchedFull + 16;
+  volatile int* sched_items = reinterpret_cast<volatile int*>(smem + SmemLayout::sched_items);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + SmemLayout::tmem_slot);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + SmemLayout::abort_flag);
 
@@ -94,12 +100,20 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   unsigned char* blob = prm.blob;
   const DamHeader* H = reinterpret_cast<const DamHeader*>(blob);
   const int nitems = prm.max_nL * prm.num_seqs * prm.Hq;
+  // Items (heaviest query blocks first) are claimed from a global counter by the producer thread and handed
+  // to the MMA thread and the eight softmax warps through a two-entry ring; a negative entry ends the loop.
+  auto next_item_consumer = [&](uint32_t n) -> int {
+    const uint32_t slot = n & 1u;
+    if (!mbar_wait(bSchedFull + 8 * slot, (n >> 1) & 1u, abort_flag)) return -2;
+    return sched_items[slot];
+  };
 
   if (tid == 0) {
     mbar_init(bQFull, 1); mbar_init(bQEmpty, 1);
     for (int s = 0; s < kSlots; ++s) { mbar_init(bSlotFull + 8 * s, 1); mbar_init(bSlotEmpty + 8 * s, 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(bSFull + 8 * s, 1); mbar_init(bSEmpty + 8 * s, 4); }
+    for (int s = 0; s < 4; ++s) { mbar_init(bSFull + 8 * s, 1); mbar_init(bSEmpty + 8 * s, 4); }
     mbar_init(bStat, 8);
+    for (int s = 0; s < 2; ++s) { mbar_init(bSchedFull + 8 * s, 1); mbar_init(bSchedEmpty + 8 * s, 9); }
     *abort_flag = 0u;
     mbar_fence_init();
     tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK);
@@ -117,7 +131,14 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
       for (int s = 0; s < kSlots; ++s) armed[s] = 2u;
       bool ok = true;
-      for (int w = blockIdx.x; w < nitems && ok; w += gridDim.x) {
+      for (uint32_t n = 0; ok; ++n) {
+        const uint32_t sl = n & 1u;
+        if (!(ok = mbar_wait(bSchedEmpty + 8 * sl, ((n >> 1) & 1u) ^ 1u, abort_flag))) break;
+        int w = n == 0 ? (int)blockIdx.x : (int)(gridDim.x + atomicAdd(prm.work_counter, 1u));
+        if (w >= nitems) w = -1;
+        sched_items[sl] = w;
+        mbar_arrive(bSchedFull + 8 * sl);
+        if (w < 0) break;
         const Item it = decode_item(blob, H, prm, w);
         if (!it.valid) continue;
         if (!(ok = mbar_wait(bQEmpty, (ic & 1u) ^ 1u, abort_flag))) break;
@@ -127,8 +148,8 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         tma_load_3d(sQ + 16384, &tmQ, bQFull, 64, it.h, tokq);
         ++ic;
         const int kvh = it.h / prm.group;
-        const int n = 2 * (it.qb + 1);
-        for (int t = 0; t < n && ok; ++t) {
+        const int ntile = 2 * (it.qb + 1);
+        for (int t = 0; t < ntile && ok; ++t) {
           const int kb = t % (it.qb + 1);
           const uint32_t s = sc % kSlots, ph = (sc / kSlots) & 1u;
           if (!(ok = mbar_wait(bSlotEmpty + 8 * s, ph ^ 1u, abort_flag))) break;
@@ -152,15 +173,18 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       const uint32_t idesc = idesc_bf16_f32(128, 128, 0);
       uint32_t sc = 0, ic = 0, g = 0;
       bool ok = true;
-      for (int w = blockIdx.x; w < nitems && ok; w += gridDim.x) {
+      for (uint32_t n = 0; ok; ++n) {
+        const int w = next_item_consumer(n);
+        if (w != -2) mbar_arrive(bSchedEmpty + 8 * (n & 1u));
+        if (w < 0) { ok = (w == -1); break; }
         const Item it = decode_item(blob, H, prm, w);
         if (!it.valid) continue;
         if (!(ok = mbar_wait(bQFull, ic & 1u, abort_flag))) break;
         ++ic;
-        const int n = 2 * (it.qb + 1);
-        for (int t = 0; t < n && ok; ++t, ++g, ++sc) {
-          const uint32_t buf = g & 1u, s = sc % kSlots;
-          if (!(ok = mbar_wait(bSEmpty + 8 * buf, ((g >> 1) & 1u) ^ 1u, abort_flag))) break;
+        const int ntile = 2 * (it.qb + 1);
+        for (int t = 0; t < ntile && ok; ++t, ++g, ++sc) {
+          const uint32_t buf = g & 3u, s = sc % kSlots;
+          if (!(ok = mbar_wait(bSEmpty + 8 * buf, ((g >> 2) & 1u) ^ 1u, abort_flag))) break;
           if (!(ok = mbar_wait(bSlotFull + 8 * s, (sc / kSlots) & 1u, abort_flag))) break;
           tc_fence_after();
           const uint32_t kaddr = sSlots + s * kSlotBytes;
@@ -172,7 +196,7 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           }
           tc_commit(bSlotEmpty + 8 * s);
           tc_commit(bSFull + 8 * buf);
-          if (t + 1 == n) tc_commit(bQEmpty);
+          if (t + 1 == ntile) tc_commit(bQEmpty);
         }
       }
     }
@@ -182,11 +206,15 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     const int G = (warp - 2) >> 2;
     const int r = (warp & 3) * 32 + lane;
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t tS = tmem + lane_addr + G * 128;
+    const uint32_t tS0 = tmem + lane_addr;
     float2* stat = reinterpret_cast<float2*>(smem + SmemLayout::stat);      // [2 item parities][2 groups][128 rows]
     uint32_t g = 0, cG = 0, nitem = 0;      // g: tiles issued so far (all groups); cG: tiles this group consumed
     bool ok = true;
-    for (int w = blockIdx.x; w < nitems && ok; w += gridDim.x) {
+    for (uint32_t n = 0; ok; ++n) {
+      const int w = next_item_consumer(n);
+      __syncwarp();
+      if (lane == 0 && w != -2) mbar_arrive(bSchedEmpty + 8 * (n & 1u));
+      if (w < 0) { ok = (w == -1); break; }
       const Item it = decode_item(blob, H, prm, w);
       if (!it.valid) continue;
       const int L = it.sq.L, W = it.sq.W;
@@ -195,7 +223,7 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       uint32_t* Mrow = reinterpret_cast<uint32_t*>(blob + H->off_true) + it.sq.true_off + (uint64_t)it.h * L * W + (size_t)i * W;
       float* Prow = prm.dump ? prm.dump + it.sq.p_off + (uint64_t)it.h * L * L + (size_t)i * L : nullptr;
       const int nk = it.qb + 1;
-      float m = -CUDART_INF_F, l = 0.f, inv_l = 0.f;
+      float m = -CUDART_INF_F, l = 0.f, inv_l = 0.f, thr_lo = 0.f;
       for (int t = 0; t < 2 * nk; ++t, ++g) {
         if (t == nk) {
           // both groups have finished sweep A: merge their (max, sum) per row through shared memory
@@ -210,11 +238,14 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           l = (m == -CUDART_INF_F ? 0.f : l * ex2(m - mn)) + (o.x == -CUDART_INF_F ? 0.f : o.y * ex2(o.x - mn));
           m = mn;
           inv_l = l > 0.f ? 1.0f / l : 0.f;
+          thr_lo = log2f(prm.pstar * l) - 0.03125f;
         }
         if ((g & 1u) != (uint32_t)G) continue;
         const int kb = t % nk;
         const bool sweepB = t >= nk;
-        if (!(ok = mbar_wait(bSFull + 8 * G, cG & 1u, abort_flag))) break;
+        const uint32_t buf = (uint32_t)G + 2u * (cG & 1u);          // the group's two buffers alternate
+        const uint32_t tS = tS0 + buf * 128;
+        if (!(ok = mbar_wait(bSFull + 8 * buf, (cG >> 1) & 1u, abort_flag))) break;
         ++cG;
         tc_fence_after();
         // keys beyond the causal limit (and beyond the window, which the limit implies) do not exist
@@ -258,7 +289,8 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
               tsum = tsum * ex2(tmax - mn) + ((a0 + a1) + (a2 + a3));     // tmax = -inf gives a factor 0
               tmax = mn;
             }
-          } else {
+          } else if (Prow) {
+            // the caller wants the map itself: every probability is computed and stored
             uint32_t word = 0u;
 #pragma unroll
             for (int q = 0; q < 32; ++q) {
@@ -267,18 +299,38 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
               word |= (p >= prm.pstar ? 1u : 0u) << q;
             }
             if (c == 0) words.x = word; else if (c == 1) words.y = word; else if (c == 2) words.z = word; else words.w = word;
-            if (Prow && row_valid) {
+            if (row_valid) {
               const int j0 = kb * DAM_TILE + c * 32;
 #pragma unroll
               for (int q = 0; q < 32; ++q)
                 if (j0 + q < L) Prow[j0 + q] = x[q];
             }
+          } else {
+            // only the decision p >= p* is needed.  p = 2^(x - m) / l, so an entry whose x - m lies more than
+            // 2^-5 below log2(p* l) cannot reach p* (the margin is five orders of magnitude above the rounding
+            // of the fast exponential); groups of 8 columns with no candidate in the whole warp skip the
+            // special-function unit.  Candidates are evaluated exactly as in the branch above.
+            uint32_t word = 0u;
+#pragma unroll
+            for (int q8 = 0; q8 < 32; q8 += 8) {
+              bool any = false;
+#pragma unroll
+              for (int u = 0; u < 8; ++u) any |= (x[q8 + u] - m) > thr_lo;
+              if (__any_sync(0xFFFFFFFFu, any)) {
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                  const float p = ex2(x[q8 + u] - m) * inv_l;
+                  word |= (p >= prm.pstar ? 1u : 0u) << (q8 + u);
+                }
+              }
+            }
+            if (c == 0) words.x = word; else if (c == 1) words.y = word; else if (c == 2) words.z = word; else words.w = word;
           }
           if (c < 3) tc_wait_ld();
         }
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(bSEmpty + 8 * G);
+        if (lane == 0) mbar_arrive(bSEmpty + 8 * buf);
         if (!sweepB) {
           if (tmax > -CUDART_INF_F) {
             const float mn = fmaxf(m, tmax);
@@ -333,6 +385,11 @@ cudaError_t dam_launch_scores_sm100(const void* Q, const void* K, const dam_shap
   ScoreParams p;
   p.blob = c.blob; p.dump = dump;
   p.status = reinterpret_cast<uint32_t*>(c.blob) + 1;
+  p.work_counter = reinterpret_cast<uint32_t*>(c.scratch) + 2;
+  {
+    cudaError_t e = cudaMemsetAsync(c.scratch, 0, 256, st);
+    if (e != cudaSuccess) return e;
+  }
   p.num_seqs = c.num_seqs; p.Hq = c.Hq; p.group = c.Hq / c.Hkv; p.max_nL = c.max_nL;
   p.scale_log2 = c.scale * 1.4426950408889634f;
   p.pstar = c.pstar;
