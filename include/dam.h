@@ -201,6 +201,17 @@ dam_status_t dam_mask_expand_rows(const void* mask, const dam_shape_t* shape, in
 dam_status_t dam_poll_status(const void* mask_or_scratch, void* stream);
 
 /*
+ * Self-test of the bounded waits the kernels use (every wait on an mbarrier gives up after a time limit,
+ * records DAM_ERR_DEVICE_TIMEOUT in the status word and lets the kernel return; nothing spins forever).
+ * Launches one tiny kernel that waits, for at most limit_us microseconds (1 .. 1000000), on a barrier
+ * nothing arrives on. Afterwards dam_poll_status(scratch, stream) returns DAM_ERR_DEVICE_TIMEOUT and the
+ * device stays usable. scratch: DEVICE, >= 256 bytes, 256-byte aligned; bytes 8..15 receive the time waited
+ * in nanoseconds. The paper has no counterpart; this exists so that the failure path can be exercised
+ * without faulting or hanging a GPU.
+ */
+dam_status_t dam_selftest_bounded_wait(void* scratch, size_t scratch_bytes, uint32_t limit_us, void* stream);
+
+/*
  * Both stages from HOST buffers: copies Q, K, V (HOST, pinned recommended, layouts from `shape`
  * with dense strides) into the device workspace, runs dam_build_masks and dam_sparse_attention,
  * and copies O and LSE back to HOST; everything on `stream`, which is synchronised before

@@ -23,7 +23,7 @@ STATUS = {0: "DAM_OK", 1: "DAM_ERR_INVALID_ARGUMENT", 2: "DAM_ERR_UNSUPPORTED", 
 
 EXPORTS = ["dam_version", "dam_status_string", "dam_mask_sizes", "dam_build_masks", "dam_build_masks_from_scores",
            "dam_mask_all_ones", "dam_sparse_attention", "dam_mask_stats", "dam_mask_expand_rows", "dam_poll_status",
-           "dam_prefill_host", "dam_build_masks_static", "dam_static_scratch_bytes"]
+           "dam_prefill_host", "dam_build_masks_static", "dam_static_scratch_bytes", "dam_selftest_bounded_wait"]
 
 
 class DamError(RuntimeError):
@@ -244,6 +244,16 @@ def dam_mask_expand_rows(mask: torch.Tensor, shape: Shape, seq: int, head: int, 
 
 def dam_poll_status(buf: torch.Tensor) -> int:
     return int(lib().dam_poll_status(_ptr(buf), _stream(buf.device)))
+
+
+def dam_selftest_bounded_wait(device, limit_us: int = 20000):
+    """Runs the bounded-wait self-test; returns (status read back, nanoseconds waited)."""
+    scr = torch.zeros(256, dtype=torch.uint8, device=device)
+    rc = lib().dam_selftest_bounded_wait(_ptr(scr), ctypes.c_size_t(256), ctypes.c_uint32(limit_us), _stream(device))
+    _check(rc, "dam_selftest_bounded_wait")
+    status = dam_poll_status(scr)
+    waited = int(scr[8:16].cpu().numpy().view(np.uint64)[0])
+    return status, waited
 
 
 def dam_prefill_host(Qh: torch.Tensor, Kh: torch.Tensor, Vh: torch.Tensor, shape: Shape, rule: dam_rule_t,

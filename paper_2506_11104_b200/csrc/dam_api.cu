@@ -334,6 +334,14 @@ dam_status_t dam_poll_status(const void* mask_or_scratch, void* stream) {
   return static_cast<dam_status_t>(w[1]);
 }
 
+dam_status_t dam_selftest_bounded_wait(void* scratch, size_t scratch_bytes, uint32_t limit_us, void* stream) {
+  if (!scratch || !aligned(scratch, 256) || limit_us == 0 || limit_us > 1000000u) return DAM_ERR_INVALID_ARGUMENT;
+  if (scratch_bytes < 256) return DAM_ERR_BUFFER_TOO_SMALL;
+  cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(scratch, 0, 256, cs) != cudaSuccess) return DAM_ERR_CUDA;
+  return dam_launch_bounded_wait_selftest(scratch, 1000ull * limit_us, cs) == cudaSuccess ? DAM_OK : DAM_ERR_CUDA;
+}
+
 dam_status_t dam_prefill_host(const void* Qh, const void* Kh, const void* Vh, const dam_shape_t* shape,
                               const dam_rule_t* rule, int32_t causal, void* Oh, float* lse_h, void* workspace,
                               size_t* workspace_bytes, void* stream) {

@@ -726,7 +726,32 @@ gather_columns_kernel(const unsigned char* __restrict__ blob, const __nv_bfloat1
   }
 }
 
+// Self-test of the bounded wait every kernel in this library uses: waits on an mbarrier that nothing ever
+// arrives on, with the given limit; the wait gives up, the status word is set and the kernel returns normally.
+__global__ void bounded_wait_selftest_kernel(uint32_t* status, unsigned long long limit_ns, unsigned long long* waited_ns) {
+  __shared__ uint64_t bar;
+  __shared__ uint32_t abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0u;
+    mbar_fence_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const uint64_t t0 = globaltimer_ns();
+    const bool ok = mbar_wait(smem_u32(&bar), 0u, &abort_flag, limit_ns);
+    *waited_ns = globaltimer_ns() - t0;
+    if (!ok) atomicMax(status, (uint32_t)DAM_ERR_DEVICE_TIMEOUT);
+  }
+}
+
 }  // namespace
+
+cudaError_t dam_launch_bounded_wait_selftest(void* scratch, unsigned long long limit_ns, cudaStream_t st) {
+  bounded_wait_selftest_kernel<<<1, 32, 0, st>>>(reinterpret_cast<uint32_t*>(scratch) + 1, limit_ns,
+                                                  reinterpret_cast<unsigned long long*>(scratch) + 1);
+  return cudaGetLastError();
+}
 
 cudaError_t dam_launch_attn_sm100(const void* Q, const void* K, const void* V, const void* blob,
                                   const dam_shape_t* s, int causal, float scale, void* O, float* lse, void* scratch,

@@ -216,3 +216,5 @@ cudaError_t dam_launch_attn_sm100(const void* Q, const void* K, const void* V, c
                                   void* scratch, size_t scratch_bytes, cudaStream_t st);
 cudaError_t dam_launch_scores_sm100(const void* Q, const void* K, const dam_shape_t* shape, const DamBuildCtx& c,
                                     float* scores_dump, cudaStream_t st);
+
+cudaError_t dam_launch_bounded_wait_selftest(void* scratch, unsigned long long limit_ns, cudaStream_t st);

@@ -152,3 +152,39 @@ def test_gathered_blob_with_small_scratch_reports_error():
     O, lse, scr = B.dam_sparse_attention(w.Q.to(DEV), w.K.to(DEV), w.V.to(DEV), blob, shape, scratch=small)
     torch.cuda.synchronize()
     assert B.dam_poll_status(scr) == 3
+
+
+def test_bounded_wait_times_out_cleanly():
+    """A wait that nothing satisfies gives up after its limit, the status word says so, and the device keeps
+    working (the next kernel runs and is correct)."""
+    status, waited_ns = B.dam_selftest_bounded_wait(DEV, limit_us=20000)
+    assert status == 5                                   # DAM_ERR_DEVICE_TIMEOUT
+    assert 15e6 <= waited_ns <= 500e6
+    w = synth.small_case(0, 4, 2, 128, 128, seed=9, lengths=[300])
+    shape = _shape(w)
+    blob = B.dam_mask_all_ones(shape, True, DEV)
+    O, lse = _run(w, blob, shape)
+    _check(w, O, lse, None, _all_rows, all_ones=True)
+
+
+def test_strided_qkv_views():
+    """Q, K, V as views of one fused [T, Hq + 2 Hkv, d] tensor: the strides of dam_shape_t are honoured by the
+    TMA descriptors and by the plain kernels."""
+    for dtype, d in ((torch.bfloat16, 128), (torch.float32, 64)):
+        Hq, Hkv = 4, 2
+        w = synth.small_case(0, Hq, Hkv, d, 128, seed=13, dtype=dtype, lengths=[400, 131])
+        T = w.Q.shape[0]
+        fused = torch.zeros(T, Hq + 2 * Hkv, d, dtype=dtype, device=DEV)
+        fused[:, :Hq] = w.Q.to(DEV); fused[:, Hq:Hq + Hkv] = w.K.to(DEV); fused[:, Hq + Hkv:] = w.V.to(DEV)
+        Qv, Kv, Vv = fused[:, :Hq], fused[:, Hq:Hq + Hkv], fused[:, Hq + Hkv:]
+        st = ((Hq + 2 * Hkv) * d, d)
+        shape = B.make_shape(w.cu_seqlens, Hq, Hkv, d, dtype, DEV, q_strides=st, k_strides=st, v_strides=st)
+        rule = B.make_rule(w.pcl_max, w.tau, w.mu, gather_columns=True)
+        n = sum(Hq * min(S, w.pcl_max) ** 2 for S in shape.lengths)
+        dump = torch.zeros(n, dtype=torch.float32, device=DEV)
+        blob, _ = B.dam_build_masks(Qv, Kv, shape, rule, scores_dump=dump)
+        masks = H.oracle_masks_from_dump(w, dump.cpu().numpy())
+        O = torch.empty(T, Hq, d, dtype=dtype, device=DEV)
+        O, lse, scr = B.dam_sparse_attention(Qv, Kv, Vv, blob, shape, O=O)
+        assert B.dam_poll_status(scr) == 0 and B.dam_poll_status(blob) == 0
+        _check(w, O, lse, masks, _all_rows)
