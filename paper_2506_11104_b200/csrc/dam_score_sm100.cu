@@ -8,9 +8,9 @@
 //   sweep A  S = Q K^T (tcgen05, accumulator in TMEM) -> per-row running max and sum;
 //   sweep B  S again -> p = exp2(x - max) / sum in fp32 -> bit = [p >= p*] -> one 16-byte store of the
 //            row's 128 bits per tile (and the optional dump of p).
-// Warp roles: warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 and 6-9 two groups of one thread per query
-// row; group G owns TMEM buffer G, i.e. every other kv tile, and the two groups merge their row statistics
-// through shared memory between the sweeps.  Every wait is bounded.
+// Warp roles: warp 0 TMA producer, warp 1 MMA issuer, warps 2-17 four groups of one thread per query row;
+// group G owns TMEM buffer G, i.e. every fourth kv tile, and the groups merge their row statistics through
+// shared memory between the sweeps.  Every wait is bounded.
 #include <cuda_bf16.h>
 #include <math_constants.h>
 
@@ -23,8 +23,8 @@ namespace {
 
 constexpr int kSlots = 5;
 constexpr int kSlotBytes = 32768;
-constexpr int kThreads = 320;
-constexpr uint32_t kTmemCols = 512;       // four S buffers: tile g uses buffer g & 3, group g & 1 owns buffers {G, G + 2}
+constexpr int kThreads = 576;              // producer warp, MMA warp, four softmax groups of four warps
+constexpr uint32_t kTmemCols = 512;       // four S buffers: tile g uses buffer g & 3, which softmax group g & 3 owns
 
 struct SmemLayout {
   static constexpr int q = 0;
@@ -34,8 +34,8 @@ struct SmemLayout {
   // sched_full[2], sched_empty[2]
   static constexpr int n_bars = 2 + 2 * kSlots + 13;
   static constexpr int sched_items = bars + 8 * n_bars;     // int[2]
-  static constexpr int stat = sched_items + 8;              // float2 [2][2][128]
-  static constexpr int tmem_slot = stat + 2 * 2 * 128 * 8;
+  static constexpr int stat = sched_items + 8;              // float2 [2][4][128]
+  static constexpr int tmem_slot = stat + 2 * 4 * 128 * 8;
   static constexpr int abort_flag = tmem_slot + 4;
   static constexpr int total = abort_flag + 4;
 };
@@ -112,8 +112,8 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     mbar_init(bQFull, 1); mbar_init(bQEmpty, 1);
     for (int s = 0; s < kSlots; ++s) { mbar_init(bSlotFull + 8 * s, 1); mbar_init(bSlotEmpty + 8 * s, 1); }
     for (int s = 0; s < 4; ++s) { mbar_init(bSFull + 8 * s, 1); mbar_init(bSEmpty + 8 * s, 4); }
-    mbar_init(bStat, 8);
-    for (int s = 0; s < 2; ++s) { mbar_init(bSchedFull + 8 * s, 1); mbar_init(bSchedEmpty + 8 * s, 9); }
+    mbar_init(bStat, 16);
+    for (int s = 0; s < 2; ++s) { mbar_init(bSchedFull + 8 * s, 1); mbar_init(bSchedEmpty + 8 * s, 17); }   // MMA thread + 16 softmax warps
     *abort_flag = 0u;
     mbar_fence_init();
     tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK);
@@ -226,26 +226,31 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       float m = -CUDART_INF_F, l = 0.f, inv_l = 0.f, thr_lo = 0.f;
       for (int t = 0; t < 2 * nk; ++t, ++g) {
         if (t == nk) {
-          // both groups have finished sweep A: merge their (max, sum) per row through shared memory
-          float2* mine = stat + ((nitem & 1u) * 2 + G) * DAM_TILE;
-          const float2* other = stat + ((nitem & 1u) * 2 + (G ^ 1)) * DAM_TILE;
-          mine[r] = make_float2(m, l);
+          // all groups have finished sweep A: merge their (max, sum) per row through shared memory
+          float2* base = stat + (nitem & 1u) * 4 * DAM_TILE;
+          base[G * DAM_TILE + r] = make_float2(m, l);
           __syncwarp();
           if (lane == 0) mbar_arrive(bStat);                       // release: the warp's 32 rows are written
           if (!(ok = mbar_wait(bStat, nitem & 1u, abort_flag))) break;
-          const float2 o = other[r];
-          const float mn = fmaxf(m, o.x);
-          l = (m == -CUDART_INF_F ? 0.f : l * ex2(m - mn)) + (o.x == -CUDART_INF_F ? 0.f : o.y * ex2(o.x - mn));
-          m = mn;
+          float mn = m;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) mn = fmaxf(mn, base[q * DAM_TILE + r].x);
+          float ls = 0.f;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const float2 o = base[q * DAM_TILE + r];
+            ls += (o.x == -CUDART_INF_F) ? 0.f : o.y * ex2(o.x - mn);
+          }
+          m = mn; l = ls;
           inv_l = l > 0.f ? 1.0f / l : 0.f;
           thr_lo = log2f(prm.pstar * l) - 0.03125f;
         }
-        if ((g & 1u) != (uint32_t)G) continue;
+        if ((g & 3u) != (uint32_t)G) continue;
         const int kb = t % nk;
         const bool sweepB = t >= nk;
-        const uint32_t buf = (uint32_t)G + 2u * (cG & 1u);          // the group's two buffers alternate
+        const uint32_t buf = (uint32_t)G;
         const uint32_t tS = tS0 + buf * 128;
-        if (!(ok = mbar_wait(bSFull + 8 * buf, (cG >> 1) & 1u, abort_flag))) break;
+        if (!(ok = mbar_wait(bSFull + 8 * buf, cG & 1u, abort_flag))) break;
         ++cG;
         tc_fence_after();
         // keys beyond the causal limit (and beyond the window, which the limit implies) do not exist
@@ -253,14 +258,11 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         const bool diag = kb == it.qb;
         uint4 words = make_uint4(0u, 0u, 0u, 0u);
         float tmax = -CUDART_INF_F, tsum = 0.f;
-        uint32_t ra[32], rb[32];
-        tmem_ld32(tS, ra);
-        tc_wait_ld();
+        uint32_t cur[32];
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-          uint32_t* cur = (c & 1) ? rb : ra;
-          uint32_t* nxt = (c & 1) ? ra : rb;
-          if (c < 3) tmem_ld32(tS + (c + 1) * 32, nxt);
+          tmem_ld32(tS + c * 32, cur);
+          tc_wait_ld();
           float x[32];
 #pragma unroll
           for (int q = 0; q < 32; q += 2)
@@ -326,7 +328,6 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             }
             if (c == 0) words.x = word; else if (c == 1) words.y = word; else if (c == 2) words.z = word; else words.w = word;
           }
-          if (c < 3) tc_wait_ld();
         }
         tc_fence_before();
         __syncwarp();
