@@ -81,7 +81,7 @@ void compute_layout(const dam_shape_t* s, int pcl_max, int all_ones_causal, int 
     gath += (uint64_t)Hq * nL;
     causal_tiles += (uint64_t)Hq * nq * (nq + 1) / 2;
     if (pcl_max > 0) {
-      for (int qb = 0; qb < nq; ++qb) cap += (uint64_t)Hq * dam_row_tile_bound(qb, nL);
+      for (int qb = 0; qb < nq; ++qb) cap += (uint64_t)Hq * dam_row_tile_bound(qb, nL, L, gather);
     } else {
       cap += (uint64_t)Hq * (all_ones_causal ? (uint64_t)nq * (nq + 1) / 2 : (uint64_t)nq * nq);
     }

@@ -691,10 +691,21 @@ gather_columns_kernel(const unsigned char* __restrict__ blob, const __nv_bfloat1
     // exclusive prefix popcounts of the V words (W <= 1024 words, i.e. windows up to 32768 tokens)
     const int W = min(sq.W, 1024);
     __syncthreads();
-    if (tid == 0) {
-      int a = 0;
-      for (int w = 0; w < W; ++w) { pref[w] = a; a += __popc(Vw[w]); }
-      pref[W] = a;
+    if (tid < 32) {                                              // warp 0: 32 words per step
+      int run = 0;
+      for (int w0 = 0; w0 < W; w0 += 32) {
+        const int w = w0 + tid;
+        const int pc = w < W ? __popc(__ldg(Vw + w)) : 0;
+        int inc = pc;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+          if (tid >= o) inc += y;
+        }
+        if (w < W) pref[w] = run + inc - pc;
+        run += __shfl_sync(0xFFFFFFFFu, inc, 31);
+      }
+      if (tid == 0) pref[W] = run;
     }
     __syncthreads();
     const int nV = pref[W];

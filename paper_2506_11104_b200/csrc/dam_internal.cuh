@@ -91,8 +91,15 @@ __host__ __device__ inline uint64_t dam_cnt_stride(int L, int W, int nL) {
 __host__ __device__ inline int dam_words(int L) { return (((L + 31) >> 5) + 3) & ~3; }
 __host__ __device__ inline uint64_t dam_align(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 
-// Upper bound on listed tiles of one q-block row of a DAM mask (see dam_mask_sizes).
-__host__ __device__ inline int dam_row_tile_bound(int qb, int nL) {
+// Upper bound on listed tiles of one q-block row of a DAM mask (see dam_mask_sizes): the window's column
+// tiles plus the diagonal band, never more than the causal tiles of the row.  A row served by gathered-column
+// tiles lists at most nL gathered tiles plus the band tiles [qb - nL, qb].
+__host__ __device__ inline int dam_row_tile_bound(int qb, int nL, int L, int gather) {
+  const int gather_first = (2 * L - 1 + DAM_TILE - 1) / DAM_TILE;
+  if (gather && L > 0 && qb >= gather_first) {
+    const int band = qb + 1 < nL + 1 ? qb + 1 : nL + 1;
+    return nL + band;
+  }
   int a = qb + 1, b = 2 * nL + 1;
   return a < b ? a : b;
 }

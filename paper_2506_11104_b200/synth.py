@@ -120,8 +120,9 @@ def make_sequence(S: int, Hq: int, Hkv: int, d: int, pcl: int, plans: Sequence[H
     ang = 2.0 * math.pi * pos[:, None] * kk[None, :] / P          # [S, n_harm]
     cs = torch.stack([ang.cos(), ang.sin()], dim=-1).reshape(S, band_dims).to(torch.float32)
     K[:, :, :band_dims] = cs[:, None, :]
-    K[0, :, :band_dims] = 0.0
-    K[0, :, sink_dim] = rt
+    if S > 0:
+        K[0, :, :band_dims] = 0.0
+        K[0, :, sink_dim] = rt
     for h, plan in enumerate(plans):
         if plan.band_m > 0:
             m = min(plan.band_m, n_harm)

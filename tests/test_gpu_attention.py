@@ -188,3 +188,14 @@ def test_strided_qkv_views():
         O, lse, scr = B.dam_sparse_attention(Qv, Kv, Vv, blob, shape, O=O)
         assert B.dam_poll_status(scr) == 0 and B.dam_poll_status(blob) == 0
         _check(w, O, lse, masks, _all_rows)
+
+
+@pytest.mark.parametrize("gather", [False, True])
+def test_degenerate_lengths(gather):
+    """Empty and one-token sequences inside a packed batch, a sequence shorter than a tile, MHA (group 1)."""
+    w = synth.small_case(0, 4, 4, 128, 64, seed=17, lengths=[0, 1, 5, 0, 257, 128])
+    _masked_case(w, _all_rows, gather=gather)
+    shape = _shape(w)
+    blob = B.dam_mask_all_ones(shape, True, DEV)
+    O, lse = _run(w, blob, shape)
+    _check(w, O, lse, None, _all_rows, all_ones=True)
