@@ -14,7 +14,7 @@ struct Layout {
   size_t mask_bytes;
   size_t build_scratch_bytes;
   size_t attn_scratch_bytes;
-  uint64_t off_cnt, off_rowstat, off_rowcnt, off_hist, off_cursor;
+  uint64_t off_cnt, off_cnt_end, off_rowcnt, off_hist, off_cursor;
   int max_L, max_W, max_nL, max_nq;
   uint64_t score_elems;
 };
@@ -65,7 +65,7 @@ void compute_layout(const dam_shape_t* s, int pcl_max, int all_ones_causal, int 
   Layout& y = *out;
   memset(&y, 0, sizeof(y));
   const int Hq = s->num_q_heads;
-  uint64_t dv = 0, tr = 0, cnt = 0, cap = 0, causal_tiles = 0, lrows = 0, po = 0, gath = 0;
+  uint64_t dv = 0, tr = 0, cnt = 0, cap = 0, causal_tiles = 0, po = 0, gath = 0;
   int total_qb = 0, total_pairs = 0;
   for (int b = 0; b < s->num_seqs; ++b) {
     int S = s->cu_seqlens_host[b + 1] - s->cu_seqlens_host[b];
@@ -77,7 +77,6 @@ void compute_layout(const dam_shape_t* s, int pcl_max, int all_ones_causal, int 
     tr += (uint64_t)Hq * L * W;
     po += (uint64_t)Hq * L * L;
     cnt += (uint64_t)Hq * dam_cnt_stride(L, W, nL);
-    lrows += (uint64_t)Hq * L;
     gath += (uint64_t)Hq * nL;
     causal_tiles += (uint64_t)Hq * nq * (nq + 1) / 2;
     if (pcl_max > 0) {
@@ -116,10 +115,10 @@ void compute_layout(const dam_shape_t* s, int pcl_max, int all_ones_causal, int 
   h.off_tiles = dam_align(h.off_work + (uint64_t)sizeof(DamItem) * h.prows, 256);
   h.causal_tiles = causal_tiles;
   y.mask_bytes = dam_align(h.off_tiles + 4ull * cap, 256);
-  // build scratch: [0,256) reserved | counts | row stats (2 floats per window row) | row counts | hist | cursor
+  // build scratch: [0,256) status block and work counter | counts | row counts | hist | cursor
   y.off_cnt = 256;
-  y.off_rowstat = dam_align(y.off_cnt + 4ull * cnt, 256);
-  y.off_rowcnt = dam_align(y.off_rowstat + 8ull * lrows, 256);
+  y.off_cnt_end = dam_align(y.off_cnt + 4ull * cnt, 256);
+  y.off_rowcnt = y.off_cnt_end;
   y.off_hist = dam_align(y.off_rowcnt + 4ull * h.rows, 256);
   y.off_cursor = y.off_hist + 4ull * DAM_HIST;
   y.build_scratch_bytes = dam_align(y.off_cursor + 4ull * DAM_HIST, 256);
@@ -184,7 +183,7 @@ dam_status_t fill_ctx(const dam_shape_t* s, const dam_rule_t* r, void* mask, siz
   c->pstar = find_pstar(r->tau, r->eps);
   c->mu = r->mu; c->min_support = r->min_support;
   c->scale = r->softmax_scale > 0.f ? r->softmax_scale : 1.0f / sqrtf((float)s->head_dim);
-  c->off_cnt = y->off_cnt; c->off_rowstat = y->off_rowstat; c->off_rowcnt = y->off_rowcnt;
+  c->off_cnt = y->off_cnt; c->off_cnt_end = y->off_cnt_end; c->off_rowcnt = y->off_rowcnt;
   c->off_hist = y->off_hist; c->off_cursor = y->off_cursor;
   c->gather = gather;
   c->off_true = y->hdr.off_true; c->true_bytes = y->hdr.off_tile_ptr - y->hdr.off_true;
@@ -233,7 +232,7 @@ dam_status_t dam_build_masks(const void* Q, const void* K, const dam_shape_t* sh
   if (!Q || !K || !aligned(Q, 16) || !aligned(K, 16) || (scores_dump && !aligned(scores_dump, 16)))
     return DAM_ERR_INVALID_ARGUMENT;
   cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
-  if (dam_launch_init_blob(shape, rule->pcl_max, y.hdr.flags, mask, y.hdr.tile_capacity, y.hdr, cs) != cudaSuccess)
+  if (dam_launch_init_blob(shape, rule->pcl_max, y.hdr.flags, mask, y.hdr, cs) != cudaSuccess)
     return DAM_ERR_CUDA;
   cudaError_t e = cudaErrorNotSupported;
   if (sm100_shape(shape)) e = dam_launch_scores_sm100(Q, K, shape, c, scores_dump, cs);
@@ -251,7 +250,7 @@ dam_status_t dam_build_masks_from_scores(const float* P, const dam_shape_t* shap
   if (st != DAM_OK) return st;
   if (!P || !aligned(P, 4)) return DAM_ERR_INVALID_ARGUMENT;
   cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
-  if (dam_launch_init_blob(shape, rule->pcl_max, y.hdr.flags, mask, y.hdr.tile_capacity, y.hdr, cs) != cudaSuccess)
+  if (dam_launch_init_blob(shape, rule->pcl_max, y.hdr.flags, mask, y.hdr, cs) != cudaSuccess)
     return DAM_ERR_CUDA;
   if (dam_launch_bits_from_scores(P, c, cs) != cudaSuccess) return DAM_ERR_CUDA;
   if (dam_launch_rule(c, cs) != cudaSuccess) return DAM_ERR_CUDA;
@@ -267,7 +266,7 @@ dam_status_t dam_mask_all_ones(const dam_shape_t* shape, int32_t causal, void* m
   compute_layout(shape, 0, causal != 0, 0, &y);
   if (mask_capacity < y.mask_bytes) return DAM_ERR_BUFFER_TOO_SMALL;
   cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
-  if (dam_launch_init_blob(shape, 0, y.hdr.flags, mask, y.hdr.tile_capacity, y.hdr, cs) != cudaSuccess)
+  if (dam_launch_init_blob(shape, 0, y.hdr.flags, mask, y.hdr, cs) != cudaSuccess)
     return DAM_ERR_CUDA;
   if (dam_launch_all_ones(shape, causal != 0, mask, cs) != cudaSuccess) return DAM_ERR_CUDA;
   return DAM_OK;

@@ -28,7 +28,6 @@
 
 #define DAM_TILE 128
 #define DAM_MAGIC 0x4B4D4144u      /* "DAMK" */
-#define DAM_SCRATCH_MAGIC 0x534D4144u /* "DAMS" */
 #define DAM_KIND_FULL 1u
 #define DAM_KIND_PARTIAL 2u
 #define DAM_KIND_GATHERED 3u    /* entry = gathered tile index | (columns in it - 1) << 16 | kind << 28 */
@@ -201,12 +200,12 @@ struct DamBuildCtx {
   int min_support;
   float scale;
   int gather;        // list gathered-column tiles
-  uint64_t off_cnt, off_rowstat, off_rowcnt, off_hist, off_cursor;   // scratch sections
+  uint64_t off_cnt, off_cnt_end, off_rowcnt, off_hist, off_cursor;   // scratch sections
   uint64_t off_true, true_bytes;                                     // true-mask section of the blob
 };
 
 cudaError_t dam_launch_init_blob(const dam_shape_t* shape, int pcl_max, uint32_t flags, void* blob,
-                                 uint32_t tile_capacity, const DamHeader& host_hdr, cudaStream_t st);
+                                 const DamHeader& host_hdr, cudaStream_t st);
 cudaError_t dam_launch_scores_ref(const void* Q, const void* K, const dam_shape_t* shape, const DamBuildCtx& c,
                                   float* scores_dump, cudaStream_t st);
 cudaError_t dam_launch_bits_from_scores(const float* P, const DamBuildCtx& c, cudaStream_t st);

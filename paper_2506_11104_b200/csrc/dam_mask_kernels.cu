@@ -562,8 +562,7 @@ __global__ void expand_rows_kernel(const unsigned char* blob, int seq, int head,
 }  // namespace
 
 cudaError_t dam_launch_init_blob(const dam_shape_t* shape, int pcl_max, uint32_t flags, void* blob,
-                                 uint32_t tile_capacity, const DamHeader& host_hdr, cudaStream_t st) {
-  (void)tile_capacity;
+                                 const DamHeader& host_hdr, cudaStream_t st) {
   int mode = (flags & DAM_FLAG_ALL_ONES) ? ((flags & DAM_FLAG_CAUSAL_LIST) ? 1 : 0) : -1;
   init_blob_kernel<<<1, 256, 0, st>>>(reinterpret_cast<unsigned char*>(blob), host_hdr, shape->cu_seqlens_dev,
                                       pcl_max, shape->num_q_heads, mode);
@@ -583,7 +582,7 @@ cudaError_t dam_launch_bits_from_scores(const float* P, const DamBuildCtx& c, cu
 cudaError_t dam_launch_rule(const DamBuildCtx& c, cudaStream_t st) {
   cudaError_t e;
   // counters start at zero: counts + prefix + tile popcounts, row counts, histogram, cursors
-  if ((e = cudaMemsetAsync(c.scratch + c.off_cnt, 0, c.off_rowstat - c.off_cnt, st)) != cudaSuccess) return e;
+  if ((e = cudaMemsetAsync(c.scratch + c.off_cnt, 0, c.off_cnt_end - c.off_cnt, st)) != cudaSuccess) return e;
   if ((e = cudaMemsetAsync(c.scratch + c.off_hist, 0, 2ull * DAM_HIST * 4, st)) != cudaSuccess) return e;
   if (c.max_nL > 0) {
     dim3 g(c.max_nL * (c.max_nL + 1) / 2, c.num_seqs * c.Hq);

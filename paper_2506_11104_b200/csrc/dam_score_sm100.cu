@@ -171,6 +171,8 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   } else if (warp == 1) {
     if (lane == 0) {
       const uint32_t idesc = idesc_bf16_f32(128, 128, 0);
+      const uint64_t dQ = smem_desc_sw128(sQ, 16, 1024), dK = smem_desc_sw128(sSlots, 16, 1024);
+      const uint32_t dQ_lo = (uint32_t)dQ, dQ_hi = (uint32_t)(dQ >> 32), dK_lo = (uint32_t)dK, dK_hi = (uint32_t)(dK >> 32);
       uint32_t sc = 0, ic = 0, g = 0;
       bool ok = true;
       for (uint32_t n = 0; ok; ++n) {
@@ -187,12 +189,11 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           if (!(ok = mbar_wait(bSEmpty + 8 * buf, ((g >> 2) & 1u) ^ 1u, abort_flag))) break;
           if (!(ok = mbar_wait(bSlotFull + 8 * s, (sc / kSlots) & 1u, abort_flag))) break;
           tc_fence_after();
-          const uint32_t kaddr = sSlots + s * kSlotBytes;
+          const uint32_t b0 = dK_lo + s * (kSlotBytes >> 4);
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks) {
-            const uint32_t off = (ks >> 2) * 16384 + (ks & 3) * 32;
-            mma_ss(tmem + buf * 128, smem_desc_sw128(sQ + off, 16, 1024), smem_desc_sw128(kaddr + off, 16, 1024), idesc,
-                   ks > 0 ? 1u : 0u);
+            const uint32_t off = ((ks >> 2) * 16384 + (ks & 3) * 32) >> 4;
+            mma_ss_lh(tmem + buf * 128, dQ_lo + off, dQ_hi, b0 + off, dK_hi, idesc, ks > 0 ? 1u : 0u);
           }
           tc_commit(bSlotEmpty + 8 * s);
           tc_commit(bSFull + 8 * buf);
