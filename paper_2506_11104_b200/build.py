@@ -25,6 +25,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not _stale():
         return LIB
     extra = ["-DDAM_PROFILE"] if os.environ.get("DAM_PROFILE") else []   # cycle counters for tuning runs
+    if os.environ.get("DAM_POLY_PER8"):
+        extra.append("-DDAM_POLY_PER8=" + os.environ["DAM_POLY_PER8"])
     objs = []
     procs = []
     for src in SOURCES:

@@ -35,6 +35,10 @@ constexpr uint32_t kColS = 0;      // S_A at 0, S_B at 128 (P_X overwrites colum
 constexpr uint32_t kColO = 256;    // O_A at 256, O_B at 384
 constexpr float kRescaleThreshold = 8.0f;
 constexpr uint32_t kNone = 0xFFFFFFFFu;
+#ifndef DAM_POLY_PER8
+#define DAM_POLY_PER8 2
+#endif
+constexpr int kPolyPer8 = DAM_POLY_PER8;   // of every 8 exponentials, how many use the FMA-pipe polynomial (0, 2 or 4)
 
 struct SmemLayout {
   static constexpr int q = 0;                           // Q_A, Q_B
@@ -74,6 +78,11 @@ struct AttnParams {
   float scale_log2;         // softmax scale * log2(e)
 };
 
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -169,7 +178,7 @@ __device__ __forceinline__ void ex2_poly2(float y0, float y1, float& p0, float& 
 template <bool MASKED>
 __device__ __forceinline__ float sweep_max(uint32_t tS, const uint4& bits) {
   uint32_t ra[32], rb[32];
-  float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F, mx2 = -CUDART_INF_F, mx3 = -CUDART_INF_F;
+  float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F;
   tmem_ld32(tS, ra);
   tc_wait_ld();
 #pragma unroll
@@ -188,11 +197,11 @@ __device__ __forceinline__ float sweep_max(uint32_t tS, const uint4& bits) {
         v2 = ((word >> (q + 2)) & 1u) ? v2 : -CUDART_INF_F;
         v3 = ((word >> (q + 3)) & 1u) ? v3 : -CUDART_INF_F;
       }
-      mx0 = fmaxf(mx0, v0); mx1 = fmaxf(mx1, v1); mx2 = fmaxf(mx2, v2); mx3 = fmaxf(mx3, v3);
+      mx0 = max3(mx0, v0, v1); mx1 = max3(mx1, v2, v3);
     }
     if (c < 3) tc_wait_ld();
   }
-  return fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+  return fmaxf(mx0, mx1);
 }
 
 // Sweep 2: p = 2^(s * scale + neg_m) for the row, packed to bf16 and stored over the first 64 columns of the
@@ -222,8 +231,9 @@ __device__ __forceinline__ float sweep_exp(uint32_t tS, const uint4& bits, float
         for (int u = 0; u < 8; u += 2)
           fma2(y[u], y[u + 1], __uint_as_float(cur[q + u]), __uint_as_float(cur[q + u + 1]), scale, scale, neg_m, neg_m);
 #pragma unroll
-        for (int u = 0; u < 6; ++u) p[u] = ex2(y[u]);
-        ex2_poly2(y[6], y[7], p[6], p[7]);
+        for (int u = 0; u < 8 - kPolyPer8; ++u) p[u] = ex2(y[u]);
+        if (kPolyPer8 >= 2) ex2_poly2(y[6], y[7], p[6], p[7]);
+        if (kPolyPer8 >= 4) ex2_poly2(y[4], y[5], p[4], p[5]);
         if (MASKED) {
 #pragma unroll
           for (int u = 0; u < 8; ++u) p[u] = ((word >> (q + u)) & 1u) ? p[u] : 0.f;
