@@ -173,6 +173,27 @@ dam_status_t dam_sparse_attention(const void* Q, const void* K, const void* V, c
                                   size_t scratch_bytes, void* stream);
 
 /*
+ * Generation-time attention under the stored patterns (Sec. 4.3, Case 2, applied to one new token per
+ * sequence; the paper's efficiency table times generation). For every sequence b the query at position
+ * i = positions[b] attends, among the keys 0..i of the KV cache, to the keys row i of the extended mask
+ * keeps: for i < L_b the row of the true mask; for i >= L_b the matched columns c (V[c] = 1) and the key
+ * i - r of every matched diagonal r (D[r] = 1). Only the pattern bits of the blob are read (no tile list), so
+ * i may exceed the length the blob was built for. Keys with no active entry: O = 0, LSE = -inf.
+ *   q, O : DEVICE, [num_seqs, num_q_heads, head_dim] contiguous, dtype of `shape`. 16-byte aligned.
+ *   K, V : DEVICE, the KV cache: sequence b owns rows cu_seqlens[b] .. cu_seqlens[b+1] - 1 (its capacity) of
+ *          the packed layout `shape` describes (K / V strides used; Q / O strides ignored); rows 0..i valid.
+ *   mask : DEVICE, a blob built for the same number of sequences and query heads (any lengths).
+ *   positions_dev : DEVICE, int32[num_seqs], 0 <= positions[b] < capacity of b (checked on the device:
+ *          a violation gives O = 0 for that sequence and INVALID_ARGUMENT in the status word of `scratch`).
+ *   lse  : DEVICE, float[num_seqs, num_q_heads].   scratch : DEVICE, >= 256 bytes, 256-byte aligned.
+ * head_dim 64 or 128 (UNSUPPORTED otherwise). Errors otherwise as dam_sparse_attention.
+ */
+dam_status_t dam_decode_attention(const void* q, const void* K, const void* V, const void* mask,
+                                  const dam_shape_t* shape, const int32_t* positions_dev, int32_t gqa_group,
+                                  float softmax_scale, void* O, float* lse, void* scratch,
+                                  size_t scratch_bytes, void* stream);
+
+/*
  * Counts taken from a mask blob (DEVICE): out[0] = listed tiles (what the attention kernel executes),
  * out[1] = of those, fully active ones, out[2] = total causal tiles of the shape (for densities),
  * out[3] = bytes of the blob in use, out[4] = 128 x 128 tiles of the masks themselves that hold an

@@ -23,7 +23,8 @@ STATUS = {0: "DAM_OK", 1: "DAM_ERR_INVALID_ARGUMENT", 2: "DAM_ERR_UNSUPPORTED", 
 
 EXPORTS = ["dam_version", "dam_status_string", "dam_mask_sizes", "dam_build_masks", "dam_build_masks_from_scores",
            "dam_mask_all_ones", "dam_sparse_attention", "dam_mask_stats", "dam_mask_expand_rows", "dam_poll_status",
-           "dam_prefill_host", "dam_build_masks_static", "dam_static_scratch_bytes", "dam_selftest_bounded_wait"]
+           "dam_prefill_host", "dam_build_masks_static", "dam_static_scratch_bytes", "dam_selftest_bounded_wait",
+           "dam_decode_attention"]
 
 
 class DamError(RuntimeError):
@@ -220,6 +221,28 @@ def dam_sparse_attention(Q, K, V, mask, shape: Shape, causal: bool = True, softm
                                     _ptr(O), _ptr(lse), _ptr(scratch), ctypes.c_size_t(scratch.numel()),
                                     _stream(Q.device))
     _check(rc, "dam_sparse_attention")
+    return O, lse, scratch
+
+
+def dam_decode_attention(q, K, V, mask, shape: Shape, positions: torch.Tensor, softmax_scale: float = 0.0,
+                         O: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
+                         scratch: Optional[torch.Tensor] = None):
+    """One new token per sequence against the KV cache `shape` describes (q, O: [B, Hq, d]; positions int32 [B]).
+
+    Returns (O, LSE [B, Hq] fp32, scratch)."""
+    B, Hq = shape.c.num_seqs, shape.c.num_q_heads
+    assert q.is_contiguous() and tuple(q.shape) == (B, Hq, shape.c.head_dim)
+    assert positions.dtype == torch.int32 and positions.numel() == B and positions.is_contiguous()
+    if O is None:
+        O = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty(B, Hq, dtype=torch.float32, device=q.device)
+    if scratch is None:
+        scratch = _alloc(256, q.device)
+    rc = lib().dam_decode_attention(_ptr(q), _ptr(K), _ptr(V), _ptr(mask), shape.ref, _ptr(positions),
+                                    Hq // shape.c.num_kv_heads, ctypes.c_float(softmax_scale), _ptr(O), _ptr(lse),
+                                    _ptr(scratch), ctypes.c_size_t(scratch.numel()), _stream(q.device))
+    _check(rc, "dam_decode_attention")
     return O, lse, scratch
 
 

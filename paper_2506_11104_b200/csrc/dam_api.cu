@@ -294,6 +294,27 @@ dam_status_t dam_sparse_attention(const void* Q, const void* K, const void* V, c
   return e == cudaSuccess ? DAM_OK : DAM_ERR_CUDA;
 }
 
+dam_status_t dam_decode_attention(const void* q, const void* K, const void* V, const void* mask,
+                                  const dam_shape_t* shape, const int32_t* positions_dev, int32_t gqa_group,
+                                  float softmax_scale, void* O, float* lse, void* scratch, size_t scratch_bytes,
+                                  void* stream) {
+  dam_status_t st;
+  if ((st = check_shape(shape)) != DAM_OK) return st;
+  if (!q || !K || !V || !mask || !positions_dev || !O || !lse || !scratch) return DAM_ERR_INVALID_ARGUMENT;
+  if (!aligned(q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16) || !aligned(lse, 4) ||
+      !aligned(positions_dev, 4) || !aligned(mask, 256) || !aligned(scratch, 256))
+    return DAM_ERR_INVALID_ARGUMENT;
+  if (gqa_group != shape->num_q_heads / shape->num_kv_heads || softmax_scale < 0.f) return DAM_ERR_INVALID_ARGUMENT;
+  if (shape->head_dim != 64 && shape->head_dim != 128) return DAM_ERR_UNSUPPORTED;
+  if (scratch_bytes < 256) return DAM_ERR_BUFFER_TOO_SMALL;
+  const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)shape->head_dim);
+  cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(scratch, 0, 256, cs) != cudaSuccess) return DAM_ERR_CUDA;
+  cudaError_t e = dam_launch_decode(q, K, V, mask, shape, positions_dev, scale, O, lse, scratch, cs);
+  if (e == cudaErrorNotSupported) return DAM_ERR_UNSUPPORTED;
+  return e == cudaSuccess ? DAM_OK : DAM_ERR_CUDA;
+}
+
 dam_status_t dam_mask_stats(const void* mask, const dam_shape_t* shape, uint64_t* out, void* stream) {
   if (!mask || !out || !shape) return DAM_ERR_INVALID_ARGUMENT;
   cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);

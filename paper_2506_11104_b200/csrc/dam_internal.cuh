@@ -223,4 +223,7 @@ cudaError_t dam_launch_attn_sm100(const void* Q, const void* K, const void* V, c
 cudaError_t dam_launch_scores_sm100(const void* Q, const void* K, const dam_shape_t* shape, const DamBuildCtx& c,
                                     float* scores_dump, cudaStream_t st);
 
+cudaError_t dam_launch_decode(const void* q, const void* K, const void* V, const void* blob, const dam_shape_t* shape,
+                              const int32_t* pos_dev, float scale, void* O, float* lse, void* scratch, cudaStream_t st);
+
 cudaError_t dam_launch_bounded_wait_selftest(void* scratch, unsigned long long limit_ns, cudaStream_t st);
