@@ -70,6 +70,12 @@ def aggregate_over_ranks(total_ms, flops, world, device):
     """Whole-job figures: time = MAX over ranks, work = SUM over ranks.  Returns (ms, flops)."""
     if world <= 1:
         return float(total_ms), float(flops)
+    if args.only_decode:
+        if rank == 0:
+            torch.cuda.set_device(0)
+            print(json.dumps({"decode": decode_leg("cuda:0", num_seqs=args.only_decode, iters=4)}))
+        return
+
     import torch.distributed as dist
     t = torch.tensor([total_ms], dtype=torch.float64, device=device)
     f = torch.tensor([flops], dtype=torch.float64, device=device)
@@ -150,6 +156,66 @@ def oracle_sample(w, n_rows=96, heads=(0, 13)):
     return layer_s, info
 
 
+def decode_leg(dev, num_seqs=64, capacity=32768, pcl=2048, iters=16):
+    """Generation-time attention: one token per sequence against a KV cache, keys chosen by the stored patterns.
+
+    Reported beside the headline, not part of it.  Algorithmic bytes = the K and V rows a launch has to read once:
+    per (sequence, KV head) the union over its query heads of matched columns and matched diagonals, 2 x 256 B
+    each (positions are drawn at or beyond 2 L, where the two sets are disjoint)."""
+    from paper_2506_11104_b200 import binding as B
+    win, Kc, Vc, q = synth.decode_case(num_seqs, capacity, pcl, dev)
+    Hq, Hkv, d = win.num_q_heads, win.num_kv_heads, win.head_dim
+    wshape = B.make_shape(win.cu_seqlens, Hq, Hkv, d, torch.bfloat16, dev)
+    rule = B.make_rule(pcl, win.tau, win.mu)
+    blob, _ = B.dam_build_masks(win.Q, win.K, wshape, rule)
+    assert B.dam_poll_status(blob) == 0
+    mb = B.MaskBlob(blob)
+    g = Hq // Hkv
+    keys_all = keys_unique = 0
+    for b in range(num_seqs):
+        bits = [mb.pattern_bits(b, h) for h in range(Hq)]
+        keys_all += sum(int(D.sum()) + int(V.sum()) for D, _, V in bits)
+        for kv in range(Hkv):
+            uD = np.zeros_like(bits[0][0])
+            uV = np.zeros_like(bits[0][2])
+            for h in range(kv * g, (kv + 1) * g):
+                uD |= bits[h][0]
+                uV |= bits[h][2]
+            keys_unique += int(uD.sum()) + int(uV.sum())
+    cache = B.make_shape([capacity * i for i in range(num_seqs + 1)], Hq, Hkv, d, torch.bfloat16, dev)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(1)
+    poss = [torch.randint(2 * pcl, capacity, (num_seqs,), device=dev, dtype=torch.int32, generator=gen)
+            for _ in range(iters + 3)]
+    O = torch.empty_like(q)
+    lse = torch.empty(num_seqs, Hq, device=dev, dtype=torch.float32)
+    scr = torch.zeros(256, dtype=torch.uint8, device=dev)
+    for p in poss[:3]:
+        B.dam_decode_attention(q, Kc, Vc, blob, cache, p, O=O, lse=lse, scratch=scr)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for p in poss[3:]:
+        B.dam_decode_attention(q, Kc, Vc, blob, cache, p, O=O, lse=lse, scratch=scr)
+    e1.record()
+    torch.cuda.synchronize()
+    assert B.dam_poll_status(scr) == 0
+    us = e0.elapsed_time(e1) / iters * 1e3
+    row_bytes = 2 * d * 2
+    pk = peaks()
+    peak = pk["hbm_gbs"]
+    gbs = keys_unique * row_bytes / (us * 1e-6) / 1e9
+    return {"workload": f"{num_seqs} sequences x {capacity}-token KV cache (8 KV heads, d 128, bf16), one token each, "
+                        f"positions uniform in [2 PCL, capacity), PCL {pcl}; {Kc.numel() * 4 / 2**30:.1f} GiB of cache, a new "
+                        "position vector every launch",
+            "us_per_launch": round(us, 1), "tokens_per_s": round(num_seqs / (us * 1e-6)),
+            "keys_per_query_head": round(keys_all / (num_seqs * Hq), 1),
+            "unique_keys_per_kv_head": round(keys_unique / (num_seqs * Hkv), 1),
+            "roofline": {"bound": "hbm", "kernel": "decode_kernel", "achieved": round(gbs, 1), "peak": peak,
+                         "peak_kind": "copy bandwidth, " + pk["which"], "unit": "GB/s", "frac": round(gbs / peak, 4),
+                         "requested_gbs": round(keys_all * row_bytes / (us * 1e-6) / 1e9, 1)}}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -160,6 +226,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-dense", action="store_true")
+    ap.add_argument("--no-decode", action="store_true", help="skip the generation-time (KV cache) measurement")
+    ap.add_argument("--only-decode", type=int, default=0, metavar="SEQS",
+                    help="run only the generation-time measurement on SEQS sequences and print its object (for profiling)")
     ap.add_argument("--no-gather", action="store_true", help="list one tile per matched column stripe instead of gathered-column tiles")
     args = ap.parse_args()
 
@@ -304,6 +373,9 @@ def main():
                                "speedup_sparse_stage2": round(dense_ms / attn_ms, 2),
                                "speedup_sparse_layer": round(dense_ms / (total_ms_max / args.steps), 2)}
         del dmask
+
+    if rank == 0 and world == 1 and not args.no_decode:
+        out["decode"] = decode_leg(dev)
 
     if not args.no_e2e:
         # end to end through the host-buffer entry point: H2D of Q, K, V and D2H of O, LSE inside the timed region

@@ -5,9 +5,11 @@
 // (V[c] = 1) and, for every matched diagonal r (D[r] = 1), the key i - r.  Nothing else of the blob is used (no
 // tile lists), so i may lie beyond the length the blob was built for.  The work is a gather of a few hundred K
 // and V rows per (sequence, head): bound by memory latency and bandwidth, not by arithmetic, so it runs on the
-// CUDA cores: one block of 8 warps per (sequence, query head); a warp turns 8 words of pattern bits into a key
-// list, 8 lanes share one key (each holds head_dim / 8 dimensions of q and of the output), 8 keys are in
-// flight per warp, online softmax in the log2 domain, partial results merged through shuffles and shared memory.
+// CUDA cores: one block of 8 warps per (sequence, query head).  The block expands the pattern words into a key
+// list in shared memory (a thread per word, block-wide prefix sum), then the keys are dealt to the warps: 8
+// lanes share one key (each holds head_dim / 8 dimensions of q and of the output), every lane group has the
+// K and V rows of 4 keys in flight (16 keys per warp), online softmax in the log2 domain, partial results
+// merged through shuffles and shared memory.
 #include <cuda_bf16.h>
 #include <math_constants.h>
 
@@ -16,7 +18,15 @@
 namespace {
 
 constexpr int kWarps = 8;
-constexpr int kChunkWords = 8;                 // pattern words a warp expands at a time (<= 256 keys)
+#ifndef DAM_DEC_KPG
+#define DAM_DEC_KPG 2
+#endif
+#ifndef DAM_DEC_BPS
+#define DAM_DEC_BPS 4
+#endif
+constexpr int kKeysPerGroup = DAM_DEC_KPG;     // keys a lane group has in flight per step
+constexpr int kBlocksPerSM = DAM_DEC_BPS;      // resident blocks the register budget is sized for
+constexpr int kRoundWords = 256;               // pattern words the block expands at a time (<= 8192 keys, 32 KB)
 
 template <typename T, int N> struct LdN;       // N consecutive elements -> float
 template <int N> struct LdN<float, N> {
@@ -87,14 +97,48 @@ struct Acc {
   }
 };
 
+// Raw (unconverted) loads of N consecutive elements, so that many rows can be in flight per lane.
+template <typename T, int N> struct Raw;
+template <int N> struct Raw<float, N> {
+  float4 v[N / 4];
+  __device__ __forceinline__ void load(const float* p) {
+#pragma unroll
+    for (int t = 0; t < N / 4; ++t) v[t] = __ldg(reinterpret_cast<const float4*>(p) + t);
+  }
+  __device__ __forceinline__ void to_float(float* o) const {
+#pragma unroll
+    for (int t = 0; t < N / 4; ++t) { o[4 * t] = v[t].x; o[4 * t + 1] = v[t].y; o[4 * t + 2] = v[t].z; o[4 * t + 3] = v[t].w; }
+  }
+};
+template <int N> struct Raw<__nv_bfloat16, N> {
+  uint4 v[N / 8];
+  __device__ __forceinline__ void load(const __nv_bfloat16* p) {
+#pragma unroll
+    for (int t = 0; t < N / 8; ++t) v[t] = __ldg(reinterpret_cast<const uint4*>(p) + t);
+  }
+  __device__ __forceinline__ void to_float(float* o) const {
+#pragma unroll
+    for (int t = 0; t < N / 8; ++t) {
+      const uint32_t w[4] = {v[t].x, v[t].y, v[t].z, v[t].w};
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        o[8 * t + 2 * q] = __uint_as_float(w[q] << 16);
+        o[8 * t + 2 * q + 1] = __uint_as_float(w[q] & 0xFFFF0000u);
+      }
+    }
+  }
+};
+
 template <typename T, int D>
-__global__ void __launch_bounds__(kWarps * 32)
+__global__ void __launch_bounds__(kWarps * 32, kBlocksPerSM)
 decode_kernel(const T* __restrict__ q, const T* __restrict__ K, const T* __restrict__ V,
               const unsigned char* __restrict__ blob, const int32_t* __restrict__ cu, const int32_t* __restrict__ pos_dev,
               int num_seqs, int Hq, int group, int64_t kst, int64_t ksh, int64_t vst, int64_t vsh, float scale_log2,
               T* __restrict__ O, float* __restrict__ lse, uint32_t* status) {
   constexpr int DPL = D / 8;
-  __shared__ int keys[kWarps][kChunkWords * 32];
+  constexpr int kThreads = kWarps * 32;
+  __shared__ int keys[kRoundWords * 32];
+  __shared__ int warp_tot[kWarps];
   __shared__ float sm_m[kWarps], sm_l[kWarps];
   __shared__ float sm_o[kWarps][D];
   const int h = blockIdx.x, b = blockIdx.y;
@@ -129,61 +173,85 @@ decode_kernel(const T* __restrict__ q, const T* __restrict__ K, const T* __restr
   for (int t = 0; t < DPL; ++t) qf[t] *= scale_log2;
   Acc<DPL> acc;
   acc.init();
-  int* list = keys[warp];
-  for (int w0 = warp * kChunkWords; w0 < nwords; w0 += kWarps * kChunkWords) {
-    // ---- expand up to 8 words into key indices
-    uint32_t word = 0u;
-    const int wi = w0 + lane;
-    if (lane < kChunkWords && wi < nwords) {
-      if (in_window) {
-        word = __ldg(hb.M + (size_t)pos * W + wi);
-      } else if (wi < W) {
-        word = __ldg(hb.V + wi);
-      } else {
-        // diagonal r = 32 (wi - W) + k selects key pos - r; drop it when that key is a matched column (it
-        // is already in the list): bit k of the reversed 32-bit window of V that ends at key pos - 32 (wi - W)
-        const int r0 = 32 * (wi - W);
-        word = __ldg(hb.D + (wi - W)) & ~__brev(dam_window32(hb.V, W, pos - r0 - 31));
+  for (int w0 = 0; w0 < nwords; w0 += kRoundWords) {
+    // ---- the block expands up to kRoundWords pattern words into one key list (a thread per word)
+    const int nw = min(kRoundWords, nwords - w0);
+    int total = 0;
+    __syncthreads();                                          // the previous round's list is no longer read
+    for (int wb = 0; wb < nw; wb += kThreads) {
+      const int wi = w0 + wb + tid;
+      uint32_t word = 0u;
+      if (wb + tid < nw) {
+        if (in_window) {
+          word = __ldg(hb.M + (size_t)pos * W + wi);
+        } else if (wi < W) {
+          word = __ldg(hb.V + wi);
+        } else {
+          // diagonal r = 32 (wi - W) + k selects key pos - r; drop it when that key is a matched column (it
+          // is already in the list): bit k of the reversed 32-bit window of V that ends at key pos - 32 (wi - W)
+          const int r0 = 32 * (wi - W);
+          word = __ldg(hb.D + (wi - W)) & ~__brev(dam_window32(hb.V, W, pos - r0 - 31));
+        }
       }
-    }
-    const int cnt = __popc(word);
-    int off = cnt;
+      const int cnt = __popc(word);
+      int off = cnt;
 #pragma unroll
-    for (int o = 1; o < kChunkWords; o <<= 1) {
-      const int y = __shfl_up_sync(0xFFFFFFFFu, off, o);
-      if (lane >= o) off += y;
-    }
-    const int total = __shfl_sync(0xFFFFFFFFu, off, kChunkWords - 1);
-    off -= cnt;
-    __syncwarp();
-    while (word) {
-      const int k = __ffs(word) - 1;
-      word &= word - 1u;
-      list[off++] = (in_window || wi < W) ? 32 * wi + k : pos - (32 * (wi - W) + k);
-    }
-    __syncwarp();
-    // ---- 8 keys per step: two per lane group
-    for (int base = 0; base < total; base += 8) {
-      const int i0 = base + g, i1 = base + 4 + g;
-      const bool v0 = i0 < total, v1 = i1 < total;
-      const int j0 = v0 ? list[i0] : 0, j1 = v1 ? list[i1] : 0;
-      float k0[DPL], k1[DPL];
-      LdN<T, DPL>::load(Kb + (int64_t)j0 * kst, k0);
-      LdN<T, DPL>::load(Kb + (int64_t)j1 * kst, k1);
-      float s0 = 0.f, s1 = 0.f;
+      for (int o = 1; o < 32; o <<= 1) {
+        const int y = __shfl_up_sync(0xFFFFFFFFu, off, o);
+        if (lane >= o) off += y;
+      }
+      if (lane == 31) warp_tot[warp] = off;
+      __syncthreads();
+      int before = total;
 #pragma unroll
-      for (int t = 0; t < DPL; ++t) { s0 = fmaf(qf[t], k0[t], s0); s1 = fmaf(qf[t], k1[t], s1); }
-      LdN<T, DPL>::load(Vb + (int64_t)j0 * vst, k0);
-      LdN<T, DPL>::load(Vb + (int64_t)j1 * vst, k1);
+      for (int w = 0; w < kWarps; ++w) {
+        const int wt = warp_tot[w];
+        if (w < warp) before += wt;
+        total += wt;
+      }
+      off += before - cnt;
+      while (word) {
+        const int k = __ffs(word) - 1;
+        word &= word - 1u;
+        keys[off++] = (in_window || wi < W) ? 32 * wi + k : pos - (32 * (wi - W) + k);
+      }
+      __syncthreads();
+    }
+    // ---- every lane group takes 4 keys per step; the K and V rows of all of them are requested before any
+    //      is used
+    for (int base = warp * (4 * kKeysPerGroup); base < total; base += kWarps * 4 * kKeysPerGroup) {
+      Raw<T, DPL> kr[kKeysPerGroup], vr[kKeysPerGroup];
+      bool valid[kKeysPerGroup];
+#pragma unroll
+      for (int u = 0; u < kKeysPerGroup; ++u) {
+        const int idx = base + u * 4 + g;
+        valid[u] = idx < total;
+        const int j = valid[u] ? keys[idx] : 0;
+        kr[u].load(Kb + (int64_t)j * kst);
+        vr[u].load(Vb + (int64_t)j * vst);
+      }
+      float sc[kKeysPerGroup];
+#pragma unroll
+      for (int u = 0; u < kKeysPerGroup; ++u) {
+        float kf[DPL];
+        kr[u].to_float(kf);
+        float s = 0.f;
+#pragma unroll
+        for (int t = 0; t < DPL; ++t) s = fmaf(qf[t], kf[t], s);
+        sc[u] = s;
+      }
 #pragma unroll
       for (int o = 1; o < 8; o <<= 1) {
-        s0 += __shfl_xor_sync(0xFFFFFFFFu, s0, o);
-        s1 += __shfl_xor_sync(0xFFFFFFFFu, s1, o);
+#pragma unroll
+        for (int u = 0; u < kKeysPerGroup; ++u) sc[u] += __shfl_xor_sync(0xFFFFFFFFu, sc[u], o);
       }
-      if (v0) acc.add(s0, k0);
-      if (v1) acc.add(s1, k1);
+#pragma unroll
+      for (int u = 0; u < kKeysPerGroup; ++u) {
+        float vf[DPL];
+        vr[u].to_float(vf);
+        if (valid[u]) acc.add(sc[u], vf);
+      }
     }
-    __syncwarp();
   }
   // ---- merge: the 4 lane groups of the warp, then the warps of the block
   acc.merge_xor(8);

@@ -227,6 +227,31 @@ def config4(device="cpu", lengths=(4096, 16384, 32768, 65536), pcl: int = 1024) 
     return _pack("C4 varlen", seqs, cu, pcl, r["tau"], r["mu"], torch.bfloat16, plans)
 
 
+def decode_case(num_seqs: int = 64, capacity: int = 32768, pcl: int = 2048, device="cpu", seed: int = 6):
+    """Generation-time workload: (window Workload, K cache, V cache, q).
+
+    Every sequence owns `capacity` rows of a Llama-3-8B-shaped KV cache (8 KV heads, d 128, bf16).  Its first
+    `pcl` rows are a planted window drawn like the layers of config 2 (the masks are built from them); the rest of
+    the cache is N(0, 1) noise, which is all a throughput measurement of the gather needs.  q is [num_seqs, 32, 128]."""
+    Hq, Hkv, d = 32, 8, 128
+    r = CONFIG_RULE[2]
+    seqs, plans, cu = [], [], [0]
+    for b in range(num_seqs):
+        p = _draw_plans(Hq, pcl, [seed, 6, 0, b], (2, 3, 4, 6, 8, 12, 16, 24, 40), 16)
+        seqs.append(make_sequence(pcl, Hq, Hkv, d, pcl, p, r["amp"], [seed, 6, 0, b], device))
+        plans.append(p)
+        cu.append(cu[-1] + pcl)
+    win = _pack(f"decode windows {num_seqs} x {pcl}", seqs, cu, pcl, r["tau"], r["mu"], torch.bfloat16, plans)
+    gen = _gen([seed, 6, 1], device)
+    Kc = torch.randn(num_seqs * capacity, Hkv, d, generator=gen, device=device, dtype=torch.bfloat16)
+    Vc = torch.randn(num_seqs * capacity, Hkv, d, generator=gen, device=device, dtype=torch.bfloat16)
+    for b in range(num_seqs):
+        Kc[b * capacity: b * capacity + pcl] = win.K[b * pcl: (b + 1) * pcl]
+        Vc[b * capacity: b * capacity + pcl] = win.V[b * pcl: (b + 1) * pcl]
+    q = torch.randn(num_seqs, Hq, d, generator=gen, device=device, dtype=torch.bfloat16)
+    return win, Kc, Vc, q
+
+
 def small_case(S: int, Hq: int, Hkv: int, d: int, pcl: int, seed: int = 1, dtype=torch.bfloat16, device="cpu",
                lengths: Optional[Sequence[int]] = None, tau: float = 0.05, mu: float = 0.8, amp: float = 8.0,
                max_stripes: int = 3) -> Workload:
