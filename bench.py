@@ -70,12 +70,6 @@ def aggregate_over_ranks(total_ms, flops, world, device):
     """Whole-job figures: time = MAX over ranks, work = SUM over ranks.  Returns (ms, flops)."""
     if world <= 1:
         return float(total_ms), float(flops)
-    if args.only_decode:
-        if rank == 0:
-            torch.cuda.set_device(0)
-            print(json.dumps({"decode": decode_leg("cuda:0", num_seqs=args.only_decode, iters=4)}))
-        return
-
     import torch.distributed as dist
     t = torch.tensor([total_ms], dtype=torch.float64, device=device)
     f = torch.tensor([flops], dtype=torch.float64, device=device)
@@ -240,6 +234,12 @@ def main():
         if rank != 0:
             return
         run_reference(args)
+        return
+
+    if args.only_decode:
+        if rank == 0:
+            torch.cuda.set_device(0)
+            print(json.dumps({"decode": decode_leg("cuda:0", num_seqs=args.only_decode, iters=4)}))
         return
 
     import torch.distributed as dist

@@ -71,15 +71,6 @@ struct Acc {
 #pragma unroll
     for (int t = 0; t < DPL; ++t) o[t] = 0.f;
   }
-  __device__ __forceinline__ void add(float s, const float* v) {
-    const float mn = fmaxf(m, s);
-    const float a = fast_ex2(m - mn);          // m = -inf: 2^-inf = 0
-    const float p = fast_ex2(s - mn);
-    l = l * a + p;
-#pragma unroll
-    for (int t = 0; t < DPL; ++t) o[t] = fmaf(p, v[t], o[t] * a);
-    m = mn;
-  }
   // state of another lane (same dimensions, other keys) fetched with a shuffle
   __device__ __forceinline__ void merge_xor(int mask) {
     const float m2 = __shfl_xor_sync(0xFFFFFFFFu, m, mask);
@@ -217,8 +208,8 @@ decode_kernel(const T* __restrict__ q, const T* __restrict__ K, const T* __restr
       }
       __syncthreads();
     }
-    // ---- every lane group takes 4 keys per step; the K and V rows of all of them are requested before any
-    //      is used
+    // ---- every lane group takes kKeysPerGroup keys per step; the K and V rows of all of them are requested
+    //      before any is used
     for (int base = warp * (4 * kKeysPerGroup); base < total; base += kWarps * 4 * kKeysPerGroup) {
       Raw<T, DPL> kr[kKeysPerGroup], vr[kKeysPerGroup];
       bool valid[kKeysPerGroup];
@@ -245,11 +236,26 @@ decode_kernel(const T* __restrict__ q, const T* __restrict__ K, const T* __restr
 #pragma unroll
         for (int u = 0; u < kKeysPerGroup; ++u) sc[u] += __shfl_xor_sync(0xFFFFFFFFu, sc[u], o);
       }
+      // one reference move per step: all keys of the step are added against the same maximum
+      float mn = acc.m;
 #pragma unroll
-      for (int u = 0; u < kKeysPerGroup; ++u) {
-        float vf[DPL];
-        vr[u].to_float(vf);
-        if (valid[u]) acc.add(sc[u], vf);
+      for (int u = 0; u < kKeysPerGroup; ++u) mn = fmaxf(mn, valid[u] ? sc[u] : -CUDART_INF_F);
+      if (mn != -CUDART_INF_F) {
+        const float a = fast_ex2(acc.m - mn);                // m = -inf: 2^-inf = 0
+        float pr[kKeysPerGroup], ps = 0.f;
+#pragma unroll
+        for (int u = 0; u < kKeysPerGroup; ++u) { pr[u] = valid[u] ? fast_ex2(sc[u] - mn) : 0.f; ps += pr[u]; }
+        acc.l = acc.l * a + ps;
+#pragma unroll
+        for (int t = 0; t < DPL; ++t) acc.o[t] *= a;
+#pragma unroll
+        for (int u = 0; u < kKeysPerGroup; ++u) {
+          float vf[DPL];
+          vr[u].to_float(vf);
+#pragma unroll
+          for (int t = 0; t < DPL; ++t) acc.o[t] = fmaf(pr[u], vf[t], acc.o[t]);
+        }
+        acc.m = mn;
       }
     }
   }
