@@ -173,6 +173,24 @@ dam_status_t dam_sparse_attention(const void* Q, const void* K, const void* V, c
                                   size_t scratch_bytes, void* stream);
 
 /*
+ * Chunked prefill: dam_sparse_attention restricted, per sequence b, to the query rows
+ * [row_ranges[2b], row_ranges[2b+1]) (indices inside the sequence). The blob is the one built for the full
+ * lengths (stage 1 reads only the first L_b rows of Q and K, so it can be built as soon as the window has been
+ * computed); K and V must hold the keys 0 .. end-1 of every sequence; rows outside the ranges of O and LSE are
+ * neither read nor written. The paper has no counterpart (its Sec. 4.3 extends the mask to "longer sequences"
+ * without saying how they arrive); the arithmetic per row is exactly that of dam_sparse_attention.
+ * Work is dealt in pairs of 128-row query blocks, so every begin must be a multiple of 256 and every end a
+ * multiple of 256 or the sequence length (INVALID_ARGUMENT otherwise); an empty range skips the sequence.
+ *   row_ranges_host : HOST, int32[2 * num_seqs] (validated);  row_ranges_dev : DEVICE, the same values.
+ * Everything else as dam_sparse_attention.
+ */
+dam_status_t dam_sparse_attention_rows(const void* Q, const void* K, const void* V, const void* mask,
+                                       const dam_shape_t* shape, int32_t causal, int32_t gqa_group,
+                                       float softmax_scale, void* O, float* lse,
+                                       const int32_t* row_ranges_host, const int32_t* row_ranges_dev,
+                                       void* scratch, size_t scratch_bytes, void* stream);
+
+/*
  * Generation-time attention under the stored patterns (Sec. 4.3, Case 2, applied to one new token per
  * sequence; the paper's efficiency table times generation). For every sequence b the query at position
  * i = positions[b] attends, among the keys 0..i of the KV cache, to the keys row i of the extended mask

@@ -24,7 +24,7 @@ STATUS = {0: "DAM_OK", 1: "DAM_ERR_INVALID_ARGUMENT", 2: "DAM_ERR_UNSUPPORTED", 
 EXPORTS = ["dam_version", "dam_status_string", "dam_mask_sizes", "dam_build_masks", "dam_build_masks_from_scores",
            "dam_mask_all_ones", "dam_sparse_attention", "dam_mask_stats", "dam_mask_expand_rows", "dam_poll_status",
            "dam_prefill_host", "dam_build_masks_static", "dam_static_scratch_bytes", "dam_selftest_bounded_wait",
-           "dam_decode_attention"]
+           "dam_decode_attention", "dam_sparse_attention_rows"]
 
 
 class DamError(RuntimeError):
@@ -222,6 +222,27 @@ def dam_sparse_attention(Q, K, V, mask, shape: Shape, causal: bool = True, softm
                                     _stream(Q.device))
     _check(rc, "dam_sparse_attention")
     return O, lse, scratch
+
+
+def dam_sparse_attention_rows(Q, K, V, mask, shape: Shape, row_ranges, O: torch.Tensor, lse: torch.Tensor,
+                              causal: bool = True, softmax_scale: float = 0.0,
+                              scratch: Optional[torch.Tensor] = None):
+    """Chunked prefill: stage 2 for the query rows [begin, end) of every sequence (row_ranges: [(begin, end)] per
+    sequence).  O and LSE are updated in place on those rows only.  Returns scratch."""
+    flat = [int(x) for pair in row_ranges for x in pair]
+    assert len(flat) == 2 * shape.c.num_seqs
+    host = (ctypes.c_int32 * len(flat))(*flat)
+    dev = torch.tensor(flat, dtype=torch.int32, device=Q.device)
+    if scratch is None:
+        off = _HDR.fields["attn_scratch_bytes"][1]
+        need = int(mask[off: off + 8].cpu().numpy().view(np.uint64)[0]) if mask.numel() >= 256 else 256
+        scratch = _alloc(max(256, need), Q.device)
+    rc = lib().dam_sparse_attention_rows(_ptr(Q), _ptr(K), _ptr(V), _ptr(mask), shape.ref, int(causal),
+                                         shape.c.num_q_heads // shape.c.num_kv_heads, ctypes.c_float(softmax_scale),
+                                         _ptr(O), _ptr(lse), host, _ptr(dev), _ptr(scratch),
+                                         ctypes.c_size_t(scratch.numel()), _stream(Q.device))
+    _check(rc, "dam_sparse_attention_rows")
+    return scratch
 
 
 def dam_decode_attention(q, K, V, mask, shape: Shape, positions: torch.Tensor, softmax_scale: float = 0.0,

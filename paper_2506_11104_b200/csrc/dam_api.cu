@@ -272,9 +272,11 @@ dam_status_t dam_mask_all_ones(const dam_shape_t* shape, int32_t causal, void* m
   return DAM_OK;
 }
 
-dam_status_t dam_sparse_attention(const void* Q, const void* K, const void* V, const void* mask,
-                                  const dam_shape_t* shape, int32_t causal, int32_t gqa_group, float softmax_scale,
-                                  void* O, float* lse, void* scratch, size_t scratch_bytes, void* stream) {
+static dam_status_t sparse_attention_impl(const void* Q, const void* K, const void* V, const void* mask,
+                                          const dam_shape_t* shape, int32_t causal, int32_t gqa_group,
+                                          float softmax_scale, void* O, float* lse, const int32_t* ranges_host,
+                                          const int32_t* ranges_dev, void* scratch, size_t scratch_bytes,
+                                          void* stream) {
   dam_status_t st;
   if ((st = check_shape(shape)) != DAM_OK) return st;
   if (!Q || !K || !V || !mask || !O || !lse || !scratch) return DAM_ERR_INVALID_ARGUMENT;
@@ -282,6 +284,17 @@ dam_status_t dam_sparse_attention(const void* Q, const void* K, const void* V, c
       !aligned(mask, 256) || !aligned(scratch, 256))
     return DAM_ERR_INVALID_ARGUMENT;
   if (gqa_group != shape->num_q_heads / shape->num_kv_heads || softmax_scale < 0.f) return DAM_ERR_INVALID_ARGUMENT;
+  if ((ranges_host == nullptr) != (ranges_dev == nullptr)) return DAM_ERR_INVALID_ARGUMENT;
+  if (ranges_host) {
+    if (!aligned(ranges_dev, 4)) return DAM_ERR_INVALID_ARGUMENT;
+    for (int b = 0; b < shape->num_seqs; ++b) {
+      const int S = shape->cu_seqlens_host[b + 1] - shape->cu_seqlens_host[b];
+      const int r0 = ranges_host[2 * b], r1 = ranges_host[2 * b + 1];
+      // whole pairs of query blocks: begin on a multiple of 256, end on a multiple of 256 or the sequence end
+      if (r0 < 0 || r1 < r0 || r1 > S || r0 % (2 * DAM_TILE) || (r1 % (2 * DAM_TILE) && r1 != S))
+        return DAM_ERR_INVALID_ARGUMENT;
+    }
+  }
   if (scratch_bytes < 256) return DAM_ERR_BUFFER_TOO_SMALL;
   const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)shape->head_dim);
   cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
@@ -289,9 +302,27 @@ dam_status_t dam_sparse_attention(const void* Q, const void* K, const void* V, c
   if (cudaMemsetAsync(scratch, 0, 256, cs) != cudaSuccess) return DAM_ERR_CUDA;
   cudaError_t e = cudaErrorNotSupported;
   if (sm100_shape(shape))
-    e = dam_launch_attn_sm100(Q, K, V, mask, shape, causal != 0, scale, O, lse, scratch, scratch_bytes, cs);
-  if (e == cudaErrorNotSupported) e = dam_launch_attn_ref(Q, K, V, mask, shape, causal != 0, scale, O, lse, scratch, cs);
+    e = dam_launch_attn_sm100(Q, K, V, mask, shape, causal != 0, scale, O, lse, scratch, scratch_bytes, ranges_dev, cs);
+  if (e == cudaErrorNotSupported)
+    e = dam_launch_attn_ref(Q, K, V, mask, shape, causal != 0, scale, O, lse, scratch, ranges_dev, cs);
   return e == cudaSuccess ? DAM_OK : DAM_ERR_CUDA;
+}
+
+dam_status_t dam_sparse_attention(const void* Q, const void* K, const void* V, const void* mask,
+                                  const dam_shape_t* shape, int32_t causal, int32_t gqa_group, float softmax_scale,
+                                  void* O, float* lse, void* scratch, size_t scratch_bytes, void* stream) {
+  return sparse_attention_impl(Q, K, V, mask, shape, causal, gqa_group, softmax_scale, O, lse, nullptr, nullptr,
+                               scratch, scratch_bytes, stream);
+}
+
+dam_status_t dam_sparse_attention_rows(const void* Q, const void* K, const void* V, const void* mask,
+                                       const dam_shape_t* shape, int32_t causal, int32_t gqa_group,
+                                       float softmax_scale, void* O, float* lse, const int32_t* row_ranges_host,
+                                       const int32_t* row_ranges_dev, void* scratch, size_t scratch_bytes,
+                                       void* stream) {
+  if (!row_ranges_host || !row_ranges_dev) return DAM_ERR_INVALID_ARGUMENT;
+  return sparse_attention_impl(Q, K, V, mask, shape, causal, gqa_group, softmax_scale, O, lse, row_ranges_host,
+                               row_ranges_dev, scratch, scratch_bytes, stream);
 }
 
 dam_status_t dam_decode_attention(const void* q, const void* K, const void* V, const void* mask,

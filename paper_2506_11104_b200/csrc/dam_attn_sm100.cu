@@ -76,6 +76,7 @@ struct AttnParams {
   int Hq, group, total_tokens, causal;
   int64_t o_stride_tok, o_stride_head;
   float scale_log2;         // softmax scale * log2(e)
+  const int32_t* ranges;    // row ranges [begin, end) per sequence (chunked prefill), or NULL
 };
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
@@ -258,6 +259,8 @@ __device__ __forceinline__ float sweep_exp(uint32_t tS, const uint4& bits, float
   return (s0 + s1) + (s2 + s3);
 }
 
+// RANGED: only the work items whose first row lies in the row range of their sequence are processed.
+template <bool RANGED>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                   const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
@@ -286,6 +289,11 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   // Dynamic scheduling: the work list is sorted longest first; the producer thread takes positions from a
   // global counter (the first one is the CTA index) and hands each to the other roles through a two-entry
   // ring in shared memory.  A negative position ends the loop.
+  auto item_active = [&](const Item& it) -> bool {
+    if (!RANGED) return true;
+    const int r0 = it.qb0 * DAM_TILE;
+    return r0 >= __ldg(prm.ranges + 2 * it.seq) && r0 < __ldg(prm.ranges + 2 * it.seq + 1);
+  };
   auto next_item_consumer = [&](uint32_t n, bool arrive) -> int {
     const uint32_t slot = n & 1u;
     if (!mbar_wait(bSchedFull + 8 * slot, (n >> 1) & 1u, abort_flag)) return -2;
@@ -341,7 +349,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         mbar_arrive(bSchedFull + 8 * slot);
         if (w < 0) break;
         const Item it = load_item(blob, H, w);
-        if (it.a0 == it.b1) continue;                        // no tile in either list
+        if (it.a0 == it.b1 || !item_active(it)) continue;    // no tile in either list, or outside the row range
         if (!(ok = mbar_wait(bQEmpty, (ic & 1u) ^ 1u, abort_flag))) break;
         const int tokq = it.tok0 + it.qb0 * DAM_TILE;
         mbar_arrive_expect_tx(bQFull, it.hasB ? 2 * kSlotBytes : kSlotBytes);
@@ -427,7 +435,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         const int w = next_item_consumer(n, true);
         if (w < 0) { ok = (w == -1); break; }
         const Item it = load_item(blob, H, w);
-        if (it.a0 == it.b1) continue;
+        if (it.a0 == it.b1 || !item_active(it)) continue;
         Walker wk; wk.init(tiles, it);
         int kb; uint32_t curA, curB;
         wk.next(kb, curA, curB);                               // at least one step exists
@@ -506,7 +514,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       if (lane == 0 && w != -2) mbar_arrive(bSchedEmpty + 8 * (n & 1u));    // the whole warp has read the entry
       if (w < 0) { ok = (w == -1); break; }
       const Item it = load_item(blob, H, w);
-      if (X == 1 && !it.hasB) continue;
+      if ((X == 1 && !it.hasB) || !item_active(it)) continue;
       const int qb = it.qb0 + X;
       const uint32_t t0 = X ? it.b0 : it.a0, t1 = X ? it.b1 : it.a1;
       const int i = qb * DAM_TILE + r;
@@ -776,7 +784,7 @@ cudaError_t dam_launch_bounded_wait_selftest(void* scratch, unsigned long long l
 
 cudaError_t dam_launch_attn_sm100(const void* Q, const void* K, const void* V, const void* blob,
                                   const dam_shape_t* s, int causal, float scale, void* O, float* lse, void* scratch,
-                                  size_t scratch_bytes, cudaStream_t st) {
+                                  size_t scratch_bytes, const int32_t* ranges, cudaStream_t st) {
   if (s->dtype != DAM_BF16 || s->head_dim != 128) return cudaErrorNotSupported;
   if (s->total_tokens == 0) return cudaSuccess;
   static int sm_count = 0, smem_optin = 0;
@@ -789,7 +797,8 @@ cudaError_t dam_launch_attn_sm100(const void* Q, const void* K, const void* V, c
     if (cc_major != 10) return cudaErrorNotSupported;
     cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
     if (smem_optin < kSmemBytes) return cudaErrorNotSupported;
-    if ((e = cudaFuncSetAttribute(attn_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) != cudaSuccess)
+    if ((e = cudaFuncSetAttribute(attn_sm100_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) != cudaSuccess ||
+        (e = cudaFuncSetAttribute(attn_sm100_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) != cudaSuccess)
       return e;
     cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
   }
@@ -826,6 +835,7 @@ cudaError_t dam_launch_attn_sm100(const void* Q, const void* K, const void* V, c
   p.status = reinterpret_cast<uint32_t*>(scratch) + 1;
   p.work_counter = reinterpret_cast<uint32_t*>(scratch) + 2;
   p.scratch_bytes = scratch_bytes;
+  p.ranges = ranges;
   // profile builds keep their cycle counters in the last 8 KiB of the scratch buffer
   p.prof = reinterpret_cast<unsigned long long*>(reinterpret_cast<unsigned char*>(scratch) + (scratch_bytes >= 16384 ? scratch_bytes - 8192 : 256));
   p.Hq = s->num_q_heads; p.group = s->num_q_heads / s->num_kv_heads; p.total_tokens = s->total_tokens;
@@ -833,6 +843,7 @@ cudaError_t dam_launch_attn_sm100(const void* Q, const void* K, const void* V, c
   p.o_stride_tok = s->o_stride_tok; p.o_stride_head = s->o_stride_head;
   p.scale_log2 = scale * 1.4426950408889634f;
   const int grid = pairs < sm_count ? pairs : sm_count;
-  attn_sm100_kernel<<<grid, kThreads, kSmemBytes, st>>>(tq, tk, tv, to, tg, p);
+  if (ranges) attn_sm100_kernel<true><<<grid, kThreads, kSmemBytes, st>>>(tq, tk, tv, to, tg, p);
+  else attn_sm100_kernel<false><<<grid, kThreads, kSmemBytes, st>>>(tq, tk, tv, to, tg, p);
   return cudaGetLastError();
 }

@@ -213,13 +213,15 @@ cudaError_t dam_launch_rule(const DamBuildCtx& c, cudaStream_t st);
 cudaError_t dam_launch_all_ones(const dam_shape_t* shape, int causal, void* blob, cudaStream_t st);
 cudaError_t dam_launch_expand_rows(const void* blob, int seq, int head, int row_begin, int nrows, int words,
                                    int causal, uint32_t* out, cudaStream_t st);
+// `ranges` (device, int32[2 * num_seqs], or NULL): only the pairs of query blocks whose first row lies in
+// [ranges[2b], ranges[2b+1]) of sequence b are computed
 cudaError_t dam_launch_attn_ref(const void* Q, const void* K, const void* V, const void* blob,
                                 const dam_shape_t* shape, int causal, float scale, void* O, float* lse,
-                                void* scratch, cudaStream_t st);
+                                void* scratch, const int32_t* ranges, cudaStream_t st);
 // tensor-core paths (bf16, d = 128); return cudaErrorNotSupported when the shape does not qualify
 cudaError_t dam_launch_attn_sm100(const void* Q, const void* K, const void* V, const void* blob,
                                   const dam_shape_t* shape, int causal, float scale, void* O, float* lse,
-                                  void* scratch, size_t scratch_bytes, cudaStream_t st);
+                                  void* scratch, size_t scratch_bytes, const int32_t* ranges, cudaStream_t st);
 cudaError_t dam_launch_scores_sm100(const void* Q, const void* K, const dam_shape_t* shape, const DamBuildCtx& c,
                                     float* scores_dump, cudaStream_t st);
 

@@ -110,7 +110,8 @@ template <typename T>
 __global__ void attn_ref_kernel(const unsigned char* blob, const T* __restrict__ Q, const T* __restrict__ K,
                                 const T* __restrict__ V, int Hq, int group, int d, int64_t qst, int64_t qsh,
                                 int64_t kst, int64_t ksh, int64_t vst, int64_t vsh, int64_t ost, int64_t osh,
-                                int causal, float scale, T* __restrict__ O, float* __restrict__ lse, int total_tokens) {
+                                int causal, float scale, T* __restrict__ O, float* __restrict__ lse, int total_tokens,
+                                const int32_t* __restrict__ ranges) {
   extern __shared__ float smem[];
   const DamHeader* H = reinterpret_cast<const DamHeader*>(blob);
   const int row = blockIdx.x;
@@ -118,6 +119,10 @@ __global__ void attn_ref_kernel(const unsigned char* blob, const T* __restrict__
   const int b = reinterpret_cast<const int32_t*>(blob + H->off_qbseq)[gqb];
   const DamSeq sq = reinterpret_cast<const DamSeq*>(blob + H->off_seq)[b];
   const int qb = gqb - sq.first_qblock;
+  if (ranges) {                                 // row ranges: whole pairs of query blocks, chosen by the pair's first row
+    const int r0 = (qb & ~1) * DAM_TILE;
+    if (r0 < ranges[2 * b] || r0 >= ranges[2 * b + 1]) return;
+  }
   const uint32_t* tile_ptr = reinterpret_cast<const uint32_t*>(blob + H->off_tile_ptr);
   const uint32_t* tiles = reinterpret_cast<const uint32_t*>(blob + H->off_tiles);
   const uint32_t t0 = tile_ptr[row], t1 = tile_ptr[row + 1];
@@ -205,7 +210,8 @@ cudaError_t dam_launch_scores_ref(const void* Q, const void* K, const dam_shape_
 }
 
 cudaError_t dam_launch_attn_ref(const void* Q, const void* K, const void* V, const void* blob, const dam_shape_t* s,
-                                int causal, float scale, void* O, float* lse, void* scratch, cudaStream_t st) {
+                                int causal, float scale, void* O, float* lse, void* scratch, const int32_t* ranges,
+                                cudaStream_t st) {
   (void)scratch;
   int rows = 0;
   for (int b = 0; b < s->num_seqs; ++b)
@@ -219,11 +225,11 @@ cudaError_t dam_launch_attn_ref(const void* Q, const void* K, const void* V, con
     attn_ref_kernel<float><<<rows, nw * 32, sm, st>>>((const unsigned char*)blob, (const float*)Q, (const float*)K,
         (const float*)V, s->num_q_heads, group, s->head_dim, s->q_stride_tok, s->q_stride_head, s->k_stride_tok,
         s->k_stride_head, s->v_stride_tok, s->v_stride_head, s->o_stride_tok, s->o_stride_head, causal, scale,
-        (float*)O, lse, s->total_tokens);
+        (float*)O, lse, s->total_tokens, ranges);
   else
     attn_ref_kernel<__nv_bfloat16><<<rows, nw * 32, sm, st>>>((const unsigned char*)blob, (const __nv_bfloat16*)Q,
         (const __nv_bfloat16*)K, (const __nv_bfloat16*)V, s->num_q_heads, group, s->head_dim, s->q_stride_tok,
         s->q_stride_head, s->k_stride_tok, s->k_stride_head, s->v_stride_tok, s->v_stride_head, s->o_stride_tok,
-        s->o_stride_head, causal, scale, (__nv_bfloat16*)O, lse, s->total_tokens);
+        s->o_stride_head, causal, scale, (__nv_bfloat16*)O, lse, s->total_tokens, ranges);
   return cudaGetLastError();
 }

@@ -199,3 +199,55 @@ def test_degenerate_lengths(gather):
     blob = B.dam_mask_all_ones(shape, True, DEV)
     O, lse = _run(w, blob, shape)
     _check(w, O, lse, None, _all_rows, all_ones=True)
+
+
+@pytest.mark.parametrize("lengths,Hq,Hkv,d,dtype,gather", [
+    ([1024, 300, 700], 8, 2, 128, torch.bfloat16, False),
+    ([1536], 4, 1, 128, torch.bfloat16, True),
+    ([900, 512], 2, 2, 64, torch.float32, False),
+])
+def test_chunked_prefill_equals_one_call(lengths, Hq, Hkv, d, dtype, gather):
+    """Row ranges: chunks of 256 / 512 rows, with the cache beyond each chunk's end poisoned, give bit for bit the
+    output of the single call (the arithmetic per row is the same and no row reads a key beyond itself)."""
+    w = synth.small_case(0, Hq, Hkv, d, 128, seed=21, dtype=dtype, lengths=lengths)
+    shape = _shape(w)
+    rule = B.make_rule(w.pcl_max, w.tau, w.mu, w.lam, w.eps, gather_columns=gather)
+    Q, K, V = w.Q.to(DEV), w.K.to(DEV), w.V.to(DEV)
+    blob, _ = B.dam_build_masks(Q, K, shape, rule)
+    O_ref, lse_ref, _ = B.dam_sparse_attention(Q, K, V, blob, shape, causal=True)
+    O = torch.full_like(O_ref, 7.0)
+    lse = torch.full_like(lse_ref, 7.0)
+    chunk = 512 if d == 128 else 256
+    done = [0] * len(lengths)
+    while any(dn < S for dn, S in zip(done, lengths)):
+        ranges, Kc, Vc = [], K.clone(), V.clone()
+        for b, S in enumerate(lengths):
+            r0, r1 = (done[b], min(S, done[b] + chunk)) if done[b] < S else (0, 0)
+            ranges.append((r0, r1))
+            t0 = w.cu_seqlens[b]
+            Kc[t0 + r1: t0 + S] = float("nan")               # keys that have not arrived yet
+            Vc[t0 + r1: t0 + S] = float("nan")
+            done[b] = max(done[b], r1)
+        scratch = B.dam_sparse_attention_rows(Q, Kc, Vc, blob, shape, ranges, O, lse)
+        assert B.dam_poll_status(scratch) == 0
+    assert torch.equal(O, O_ref)
+    assert torch.equal(lse, lse_ref)
+
+
+def test_row_ranges_leave_other_rows_alone_and_reject_odd_bounds():
+    w = synth.small_case(0, 4, 2, 128, 128, seed=22, dtype=torch.bfloat16, lengths=[768, 512])
+    shape = _shape(w)
+    rule = B.make_rule(w.pcl_max, w.tau, w.mu, w.lam, w.eps)
+    Q, K, V = w.Q.to(DEV), w.K.to(DEV), w.V.to(DEV)
+    blob, _ = B.dam_build_masks(Q, K, shape, rule)
+    O_ref, lse_ref, _ = B.dam_sparse_attention(Q, K, V, blob, shape, causal=True)
+    O = torch.full_like(O_ref, 7.0)
+    lse = torch.full_like(lse_ref, 7.0)
+    B.dam_sparse_attention_rows(Q, K, V, blob, shape, [(256, 512), (0, 0)], O, lse)
+    assert torch.equal(O[256:512], O_ref[256:512]) and torch.equal(lse[:, 256:512], lse_ref[:, 256:512])
+    keep = torch.ones(O.shape[0], dtype=torch.bool, device=DEV)
+    keep[256:512] = False
+    assert (O[keep] == 7.0).all() and (lse[:, keep] == 7.0).all()
+    for bad in ([(128, 512), (0, 0)], [(0, 300), (0, 0)], [(0, 1024), (0, 0)], [(512, 256), (0, 0)]):
+        with pytest.raises(B.DamError):
+            B.dam_sparse_attention_rows(Q, K, V, blob, shape, bad, O, lse)
