@@ -173,6 +173,27 @@ dam_status_t dam_sparse_attention(const void* Q, const void* K, const void* V, c
                                   size_t scratch_bytes, void* stream);
 
 /*
+ * Multi-sample capture (Sec. 4.2.2: the attention map of a head is the average of the maps of several
+ * inputs, A accumulated attention, C valid-token count, A_bar = A / (C + eps)).
+ *
+ * dam_capture_accumulate adds one batch of samples: P is the fp32 window maps of the batch in the layout of
+ * dam_build_masks' scores_dump for `shape` (sample b: [Hq][L_b][L_b], L_b = min(S_b, pcl_max));
+ *   A[h][i][j] += sum_b P_b[h][i][j]   (fp32, samples added in index order; j <= i < L_b)
+ *   C[i]       += #{b : L_b > i}       (the count depends on the row only: a pair (i, j <= i) is valid in a
+ *                                       sample exactly when the sample is longer than i)
+ * A: DEVICE float[Hq][pcl_max][pcl_max], C: DEVICE int32[pcl_max]; the caller zeroes both before the first batch.
+ *
+ * dam_capture_average writes, for every (sequence b, head h) of `shape` (the inputs the masks are for), the
+ * averaged map A[h][i][j] / ((float)C[i] + eps) restricted to L_b x L_b (IEEE single division, zero above the
+ * diagonal) into P_out, in the layout dam_build_masks_from_scores reads; that call then applies the rule.
+ * Both enqueue on `stream`; errors: INVALID_ARGUMENT (null / misaligned pointers, pcl_max < 1, eps <= 0), CUDA.
+ */
+dam_status_t dam_capture_accumulate(const float* P, const dam_shape_t* shape, int32_t pcl_max, float* A,
+                                    int32_t* C, void* stream);
+dam_status_t dam_capture_average(const float* A, const int32_t* C, int32_t pcl_max, float eps,
+                                 const dam_shape_t* shape, float* P_out, void* stream);
+
+/*
  * Chunked prefill: dam_sparse_attention restricted, per sequence b, to the query rows
  * [row_ranges[2b], row_ranges[2b+1]) (indices inside the sequence). The blob is the one built for the full
  * lengths (stage 1 reads only the first L_b rows of Q and K, so it can be built as soon as the window has been

@@ -171,6 +171,25 @@ def attention_rows(Qh: np.ndarray, Kh: np.ndarray, Vh: np.ndarray, rows: Sequenc
     return O, lse
 
 
+def capture_average(samples: Sequence[np.ndarray], pcl_max: int, eps: float, dtype=np.float64):
+    """Sec. 4.2.2, the averaged attention map of one head over several inputs.
+
+    samples: window maps P_b, each [L_b, L_b] with L_b <= pcl_max (zero above the diagonal).
+    A[i, j] = sum_b P_b[i, j] over the samples that contain the pair, C[i, j] = their number (a causal pair
+    (i, j <= i) is contained exactly when L_b > i), A_bar = A / (C + eps).  Returns (A_bar [pcl_max, pcl_max], C
+    int32 [pcl_max] per row).  With dtype float32 every sum and the division are IEEE single operations taken
+    in sample order, which is the arithmetic two implementations can agree on bit for bit."""
+    A = np.zeros((pcl_max, pcl_max), dtype=dtype)
+    C = np.zeros(pcl_max, dtype=np.int32)
+    for P in samples:
+        L = P.shape[0]
+        assert P.shape == (L, L) and L <= pcl_max
+        A[:L, :L] = A[:L, :L] + np.tril(P).astype(dtype)
+        C[:L] += 1
+    den = C.astype(dtype) + dtype(eps)
+    return (A / den[:, None]).astype(dtype), C
+
+
 # ----------------------------------------------------------------------------------------------
 # Chained helpers
 # ----------------------------------------------------------------------------------------------

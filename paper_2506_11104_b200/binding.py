@@ -24,7 +24,7 @@ STATUS = {0: "DAM_OK", 1: "DAM_ERR_INVALID_ARGUMENT", 2: "DAM_ERR_UNSUPPORTED", 
 EXPORTS = ["dam_version", "dam_status_string", "dam_mask_sizes", "dam_build_masks", "dam_build_masks_from_scores",
            "dam_mask_all_ones", "dam_sparse_attention", "dam_mask_stats", "dam_mask_expand_rows", "dam_poll_status",
            "dam_prefill_host", "dam_build_masks_static", "dam_static_scratch_bytes", "dam_selftest_bounded_wait",
-           "dam_decode_attention", "dam_sparse_attention_rows"]
+           "dam_decode_attention", "dam_sparse_attention_rows", "dam_capture_accumulate", "dam_capture_average"]
 
 
 class DamError(RuntimeError):
@@ -222,6 +222,26 @@ def dam_sparse_attention(Q, K, V, mask, shape: Shape, causal: bool = True, softm
                                     _stream(Q.device))
     _check(rc, "dam_sparse_attention")
     return O, lse, scratch
+
+
+def dam_capture_accumulate(P: torch.Tensor, shape: Shape, pcl_max: int, A: torch.Tensor, C: torch.Tensor):
+    """A += the window maps of one batch of samples (P: the scores_dump of that batch), C += valid counts per row."""
+    Hq = shape.c.num_q_heads
+    assert A.dtype == torch.float32 and A.numel() == Hq * pcl_max * pcl_max and A.is_contiguous()
+    assert C.dtype == torch.int32 and C.numel() == pcl_max
+    assert P.dtype == torch.float32 and P.numel() == sum(Hq * min(S, pcl_max) ** 2 for S in shape.lengths)
+    rc = lib().dam_capture_accumulate(_ptr(P), shape.ref, pcl_max, _ptr(A), _ptr(C), _stream(P.device))
+    _check(rc, "dam_capture_accumulate")
+
+
+def dam_capture_average(A: torch.Tensor, C: torch.Tensor, pcl_max: int, eps: float, shape: Shape) -> torch.Tensor:
+    """Averaged maps for the sequences of `shape`, in the layout dam_build_masks_from_scores reads."""
+    n = sum(shape.c.num_q_heads * min(S, pcl_max) ** 2 for S in shape.lengths)
+    P = torch.empty(n, dtype=torch.float32, device=A.device)
+    rc = lib().dam_capture_average(_ptr(A), _ptr(C), pcl_max, ctypes.c_float(eps), shape.ref, _ptr(P),
+                                   _stream(A.device))
+    _check(rc, "dam_capture_average")
+    return P
 
 
 def dam_sparse_attention_rows(Q, K, V, mask, shape: Shape, row_ranges, O: torch.Tensor, lse: torch.Tensor,

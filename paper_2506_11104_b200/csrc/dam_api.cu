@@ -257,6 +257,25 @@ dam_status_t dam_build_masks_from_scores(const float* P, const dam_shape_t* shap
   return DAM_OK;
 }
 
+dam_status_t dam_capture_accumulate(const float* P, const dam_shape_t* shape, int32_t pcl_max, float* A, int32_t* C,
+                                    void* stream) {
+  dam_status_t st;
+  if ((st = check_shape(shape)) != DAM_OK) return st;
+  if (!P || !A || !C || pcl_max < 1 || !aligned(P, 4) || !aligned(A, 4) || !aligned(C, 4)) return DAM_ERR_INVALID_ARGUMENT;
+  return dam_launch_capture_accumulate(P, shape, pcl_max, A, C, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? DAM_OK : DAM_ERR_CUDA;
+}
+
+dam_status_t dam_capture_average(const float* A, const int32_t* C, int32_t pcl_max, float eps,
+                                 const dam_shape_t* shape, float* P_out, void* stream) {
+  dam_status_t st;
+  if ((st = check_shape(shape)) != DAM_OK) return st;
+  if (!A || !C || !P_out || pcl_max < 1 || !(eps > 0.f) || !aligned(P_out, 4) || !aligned(A, 4) || !aligned(C, 4))
+    return DAM_ERR_INVALID_ARGUMENT;
+  return dam_launch_capture_average(A, C, pcl_max, eps, shape, P_out, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? DAM_OK : DAM_ERR_CUDA;
+}
+
 dam_status_t dam_mask_all_ones(const dam_shape_t* shape, int32_t causal, void* mask, size_t mask_capacity,
                                void* stream) {
   dam_status_t st;

@@ -225,6 +225,10 @@ cudaError_t dam_launch_attn_sm100(const void* Q, const void* K, const void* V, c
 cudaError_t dam_launch_scores_sm100(const void* Q, const void* K, const dam_shape_t* shape, const DamBuildCtx& c,
                                     float* scores_dump, cudaStream_t st);
 
+cudaError_t dam_launch_capture_accumulate(const float* P, const dam_shape_t* shape, int Lmax, float* A, int32_t* C,
+                                          cudaStream_t st);
+cudaError_t dam_launch_capture_average(const float* A, const int32_t* C, int Lmax, float eps, const dam_shape_t* shape,
+                                       float* P_out, cudaStream_t st);
 cudaError_t dam_launch_decode(const void* q, const void* K, const void* V, const void* blob, const dam_shape_t* shape,
                               const int32_t* pos_dev, float scale, void* O, float* lse, void* scratch, cudaStream_t st);
 

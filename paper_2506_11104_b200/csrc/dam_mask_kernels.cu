@@ -579,6 +579,77 @@ cudaError_t dam_launch_bits_from_scores(const float* P, const DamBuildCtx& c, cu
   return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------------------------
+// Multi-sample capture (Sec. 4.2.2): A[h][i][j] += sum over the samples b of a batch of P_b[h][i][j]
+// (i, j < L_b = min(S_b, L_max)), C[i] += #{b : L_b > i}.  One thread per cell of a row; the samples
+// of the batch are added in index order, so the fp32 sums do not depend on the launch.
+// ---------------------------------------------------------------------------------------------
+__global__ void capture_accumulate_kernel(const float* __restrict__ P, const int32_t* __restrict__ cu, int num_seqs,
+                                          int Hq, int Lmax, float* __restrict__ A, int32_t* __restrict__ C) {
+  const int i = blockIdx.x, h = blockIdx.y;
+  unsigned long long p_off = 0;                      // fp32 elements before sample b in the score tensor
+  int cnt = 0;
+  for (int b = 0; b < num_seqs; ++b) {
+    const int S = cu[b + 1] - cu[b];
+    const int L = S < Lmax ? S : Lmax;
+    if (i < L) {
+      ++cnt;
+      const float* Pr = P + p_off + ((unsigned long long)h * L + i) * L;
+      float* Ar = A + ((unsigned long long)h * Lmax + i) * Lmax;
+      for (int j = threadIdx.x; j <= i; j += blockDim.x) Ar[j] += __ldg(Pr + j);
+    }
+    p_off += (unsigned long long)Hq * L * L;
+  }
+  if (h == 0 && threadIdx.x == 0) C[i] += cnt;
+}
+
+// Averaged map in the layout the rule kernels read: for every (sequence b, head h) of the target shape,
+// P_out[i][j] = A[h][i][j] / (float(C[i]) + eps) for j <= i < L_b, 0 above the diagonal (IEEE single division).
+__global__ void capture_average_kernel(const float* __restrict__ A, const int32_t* __restrict__ C, int Lmax, float eps,
+                                       const int32_t* __restrict__ cu, int num_seqs, int Hq, float* __restrict__ P_out) {
+  const int i = blockIdx.x, h = blockIdx.y;
+  const float den = (float)C[i] + eps;
+  const float* Ar = A + ((unsigned long long)h * Lmax + i) * Lmax;
+  unsigned long long p_off = 0;
+  for (int b = 0; b < num_seqs; ++b) {
+    const int S = cu[b + 1] - cu[b];
+    const int L = S < Lmax ? S : Lmax;
+    if (i < L) {
+      float* Pr = P_out + p_off + ((unsigned long long)h * L + i) * L;
+      for (int j = threadIdx.x; j < L; j += blockDim.x) Pr[j] = j <= i ? Ar[j] / den : 0.f;
+    }
+    p_off += (unsigned long long)Hq * L * L;
+  }
+}
+
+cudaError_t dam_launch_capture_accumulate(const float* P, const dam_shape_t* s, int Lmax, float* A, int32_t* C,
+                                          cudaStream_t st) {
+  int maxL = 0;
+  for (int b = 0; b < s->num_seqs; ++b) {
+    int L = s->cu_seqlens_host[b + 1] - s->cu_seqlens_host[b];
+    L = L < Lmax ? L : Lmax;
+    maxL = L > maxL ? L : maxL;
+  }
+  if (maxL == 0) return cudaSuccess;
+  capture_accumulate_kernel<<<dim3(maxL, s->num_q_heads), 256, 0, st>>>(P, s->cu_seqlens_dev, s->num_seqs,
+                                                                        s->num_q_heads, Lmax, A, C);
+  return cudaGetLastError();
+}
+
+cudaError_t dam_launch_capture_average(const float* A, const int32_t* C, int Lmax, float eps, const dam_shape_t* s,
+                                       float* P_out, cudaStream_t st) {
+  int maxL = 0;
+  for (int b = 0; b < s->num_seqs; ++b) {
+    int L = s->cu_seqlens_host[b + 1] - s->cu_seqlens_host[b];
+    L = L < Lmax ? L : Lmax;
+    maxL = L > maxL ? L : maxL;
+  }
+  if (maxL == 0) return cudaSuccess;
+  capture_average_kernel<<<dim3(maxL, s->num_q_heads), 256, 0, st>>>(A, C, Lmax, eps, s->cu_seqlens_dev, s->num_seqs,
+                                                                     s->num_q_heads, P_out);
+  return cudaGetLastError();
+}
+
 cudaError_t dam_launch_rule(const DamBuildCtx& c, cudaStream_t st) {
   cudaError_t e;
   // counters start at zero: counts + prefix + tile popcounts, row counts, histogram, cursors

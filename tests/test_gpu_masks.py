@@ -229,3 +229,46 @@ def test_mask_tile_count_is_independent_of_gathering():
     a, b = B.dam_mask_stats(plain, shape), B.dam_mask_stats(gath, shape)
     assert a["mask_tiles"] == a["tiles"] == b["mask_tiles"]
     assert b["tiles"] < a["tiles"]
+
+
+def test_multi_sample_capture_masks_bit_exact():
+    """Three batches of samples of mixed lengths are accumulated on the GPU; the masks built from the averaged
+    maps equal, bit for bit, the oracle's masks from its own fp32 average of the same per-sample score tensors."""
+    Hq, Hkv, d, pcl = 4, 2, 64, 160
+    batches = [[400, 100], [160, 300, 37], [512]]
+    A = torch.zeros(Hq * pcl * pcl, dtype=torch.float32, device=DEV)
+    C = torch.zeros(pcl, dtype=torch.int32, device=DEV)
+    per_head = [[] for _ in range(Hq)]
+    w_last = None
+    for k, lengths in enumerate(batches):
+        w = synth.small_case(0, Hq, Hkv, d, pcl, seed=30 + k, dtype=torch.bfloat16, lengths=lengths)
+        shape = B.make_shape(w.cu_seqlens, Hq, Hkv, d, w.Q.dtype, DEV)
+        rule = B.make_rule(pcl, w.tau, w.mu, w.lam, w.eps)
+        n = sum(Hq * min(S, pcl) ** 2 for S in lengths)
+        dump = torch.zeros(n, dtype=torch.float32, device=DEV)
+        B.dam_build_masks(w.Q.to(DEV), w.K.to(DEV), shape, rule, scores_dump=dump)
+        B.dam_capture_accumulate(dump, shape, pcl, A, C)
+        P = H.split_dump(dump.cpu().numpy(), lengths, Hq, pcl)
+        for b in range(len(lengths)):
+            for h in range(Hq):
+                per_head[h].append(P[b][h])
+        w_last = w
+    # masks for new inputs (one longer than the window, one shorter) from the averaged maps
+    target = [700, 90]
+    tshape = B.make_shape([0, 700, 790], Hq, Hkv, d, torch.bfloat16, DEV)
+    rule = B.make_rule(pcl, w_last.tau, w_last.mu, w_last.lam, w_last.eps)
+    Pavg = B.dam_capture_average(A, C, pcl, w_last.eps, tshape)
+    blob, _ = B.dam_build_masks_from_scores(Pavg, tshape, rule)
+    assert B.dam_poll_status(blob) == 0
+    want_C = [sum(1 for ls in batches for S in ls if min(S, pcl) > i) for i in range(pcl)]
+    assert C.cpu().tolist() == want_C
+    masks = []
+    for S in target:
+        L = min(S, pcl)
+        row = []
+        for h in range(Hq):
+            Abar, _ = orc.capture_average(per_head[h], pcl, w_last.eps, dtype=np.float32)
+            row.append(orc.head_mask_from_probs(np.ascontiguousarray(Abar[:L, :L]), S, w_last.tau, w_last.mu,
+                                                w_last.lam, w_last.eps))
+        masks.append(row)
+    H.check_blob_against_oracle(blob, tshape, masks)

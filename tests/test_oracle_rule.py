@@ -325,3 +325,43 @@ def test_one_cell_patterns():
         hm = orc.head_mask_from_probs(P, S=L, tau=0.3, mu=0.8)
         assert hm.V[L - 1] == hm.M[L - 1, L - 1]
         assert hm.D[L - 1] == hm.M[L - 1, 0]
+
+
+# ---------------------------------------------------------------------------------------------
+# Multi-sample averaged map (Sec. 4.2.2)
+# ---------------------------------------------------------------------------------------------
+def test_capture_average_hand_example():
+    # three inputs of lengths 1, 2, 3 and a window of 3: every cell is the mean over the inputs that contain it
+    P1 = np.array([[1.0]])
+    P2 = np.array([[1.0, 0.0], [0.25, 0.75]])
+    P3 = np.array([[1.0, 0.0, 0.0], [0.5, 0.5, 0.0], [0.2, 0.3, 0.5]])
+    Abar, C = orc.capture_average([P1, P2, P3], 3, 1e-10)
+    assert C.tolist() == [3, 2, 1]
+    want = np.array([[1.0, 0.0, 0.0], [0.375, 0.625, 0.0], [0.2, 0.3, 0.5]])
+    assert np.allclose(Abar, want, atol=1e-9)
+    assert np.allclose(Abar.sum(axis=1), 1.0, atol=1e-9)          # a mean of distributions is a distribution
+
+
+def test_capture_average_of_copies_is_the_map_and_window_rows_beyond_all_inputs_are_empty():
+    rng = np.random.default_rng(3)
+    P = np.tril(rng.random((6, 6))).astype(np.float32)
+    P /= P.sum(axis=1, keepdims=True)
+    A2, C2 = orc.capture_average([P, P], 8, 1e-8, dtype=np.float32)      # 2 P / 2 is exact in binary
+    assert np.array_equal(A2[:6, :6], P) and C2.tolist() == [2] * 6 + [0, 0]
+    assert not A2[6:].any() and not A2[:, 6:].any()                        # 0 / (0 + eps) = 0
+    # masks of the averaged map of identical inputs = masks of the single input
+    m1 = orc.head_mask_from_probs(P, 6, 0.3, 0.8)
+    m2 = orc.head_mask_from_probs(np.ascontiguousarray(A2[:6, :6]), 6, 0.3, 0.8)
+    assert np.array_equal(m1.M, m2.M) and np.array_equal(m1.D, m2.D) and np.array_equal(m1.V, m2.V)
+
+
+def test_capture_average_float32_tracks_float64():
+    rng = np.random.default_rng(4)
+    samples = []
+    for L in (5, 9, 9, 7, 3):
+        P = np.tril(rng.random((L, L)))
+        samples.append((P / P.sum(axis=1, keepdims=True)).astype(np.float32))
+    a32, c32 = orc.capture_average(samples, 9, 1e-8, dtype=np.float32)
+    a64, c64 = orc.capture_average(samples, 9, 1e-8, dtype=np.float64)
+    assert np.array_equal(c32, c64) and c64.tolist() == [5, 5, 5, 4, 4, 3, 3, 2, 2]
+    assert np.abs(a32 - a64).max() < 1e-6
