@@ -207,6 +207,11 @@ def decode_leg(dev, num_seqs=64, capacity=32768, pcl=2048, iters=16):
             "unique_keys_per_kv_head": round(keys_unique / (num_seqs * Hkv), 1),
             "roofline": {"bound": "hbm", "kernel": "decode_kernel", "achieved": round(gbs, 1), "peak": peak,
                          "peak_kind": "copy bandwidth, " + pk["which"], "unit": "GB/s", "frac": round(gbs / peak, 4),
+                         "traffic": (lambda t: int(t * num_seqs) if t else None)(
+                             (json.load(open(os.path.join(ROOT, "profiles", "traffic.json")))
+                              .get("decode_kernel", {}).get("per_sequence"))
+                             if os.path.exists(os.path.join(ROOT, "profiles", "traffic.json")) else None),
+                         "algorithmic_bytes": keys_unique * row_bytes,
                          "requested_gbs": round(keys_all * row_bytes / (us * 1e-6) / 1e9, 1)}}
 
 
