@@ -76,12 +76,36 @@ typedef struct dam_rule_t {
   int32_t pcl_max;      /* L_max >= 1; per sequence L = min(S, L_max) (Sec. 4.2.1)                  */
   float tau;            /* true-mask threshold on the amplified map, > 0 (Sec. 4.2.3)              */
   float mu;             /* pattern match threshold, gamma >= mu (Sec. 4.2.4)                       */
-  float lambda;         /* Box-Cox lambda; only 0.5 is supported (Sec. 4.2.2)                      */
+  float lambda;         /* lambda of Box-Cox / Yeo-Johnson (Sec. 4.2.2; the paper uses 0.5)         */
   float eps;            /* clamp constant, > 0 (Sec. 4.2.2)                                        */
   float softmax_scale;  /* 0 selects 1 / sqrt(head_dim) (Sec. 3)                                   */
   int32_t min_support;  /* ignore patterns with fewer cells; 1 = the paper's rule                  */
   uint32_t flags;       /* 0 or DAM_RULE_GATHER_COLUMNS                                            */
+  int32_t transform;    /* dam_transform_t: how the map is amplified before tau is applied          */
 } dam_rule_t;
+
+/*
+ * Amplification applied to X = max(map, eps) before the threshold (Appendix B lists nine; the paper settles on
+ * Box-Cox with lambda = 0.5). Each of these is increasing in X and the map is 0 above the diagonal, so the
+ * minimum that is subtracted is f(eps) and the true mask is {f(X) - f(eps) >= tau} = {map >= p*}:
+ *   BOXCOX      (X^lambda - 1) / lambda, log X for lambda = 0
+ *   LOG         log X                        SQRT     sqrt X            ARCSINH   asinh X
+ *   YEO_JOHNSON ((X + 1)^lambda - 1) / lambda, log(X + 1) for lambda = 0   (X >= 0 always holds here)
+ *   AVERAGE     X itself
+ * BOXCOX with lambda = 0.5 is decided by a chain of IEEE single operations (so that two implementations can
+ * agree bit for bit: x = max(p, eps); b = (sqrt(x) - 1) * 2; a = b - (sqrt(eps) - 1) * 2; a >= tau); every
+ * other case is decided in double precision on the fp32 map value, with tau, eps, lambda widened from float.
+ * Z-score and min-max normalisation (which need the mean / deviation / maximum of each map) and the raw sum are
+ * not offered.
+ */
+typedef enum dam_transform_t {
+  DAM_TRANSFORM_BOXCOX = 0,
+  DAM_TRANSFORM_LOG = 1,
+  DAM_TRANSFORM_SQRT = 2,
+  DAM_TRANSFORM_ARCSINH = 3,
+  DAM_TRANSFORM_YEO_JOHNSON = 4,
+  DAM_TRANSFORM_AVERAGE = 5
+} dam_transform_t;
 
 /*
  * dam_rule_t.flags bit: below row 2L - 1 of a sequence the matched columns (all < L) and the matched
@@ -129,7 +153,8 @@ dam_status_t dam_mask_sizes(const dam_shape_t* shape, const dam_rule_t* rule, in
  *   sum_{b' < b} Hq * L_b'^2 + h * L_b^2, row-major [L_b][L_b], zeros above the diagonal. The mask
  *   decisions are taken on exactly these fp32 values.
  * Errors: INVALID_ARGUMENT (null pointers, alignment, Hq % Hkv, tau <= 0, eps <= 0, pcl_max < 1,
- *   bad cu_seqlens, struct sizes), UNSUPPORTED (lambda != 0.5, head_dim), BUFFER_TOO_SMALL, CUDA.
+ *   bad cu_seqlens, struct sizes, unknown transform, non-finite lambda), UNSUPPORTED (head_dim),
+ *   BUFFER_TOO_SMALL, CUDA.
  */
 dam_status_t dam_build_masks(const void* Q, const void* K, const dam_shape_t* shape,
                              const dam_rule_t* rule, void* mask, size_t mask_capacity,

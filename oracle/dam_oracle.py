@@ -171,6 +171,33 @@ def attention_rows(Qh: np.ndarray, Kh: np.ndarray, Vh: np.ndarray, rows: Sequenc
     return O, lse
 
 
+def amplify_transform(P: np.ndarray, method: str, lam: float, eps: float) -> np.ndarray:
+    """Appendix B: the amplification methods that act cell by cell, on X = max(P, eps), in float64,
+    followed by the subtraction of the minimum over the whole map (cells above the diagonal included)."""
+    X = np.maximum(np.asarray(P, dtype=np.float64), np.float64(eps))
+    if method == "boxcox":
+        T = np.log(X) if lam == 0 else (np.power(X, lam) - 1.0) / lam
+    elif method == "log":
+        T = np.log(X)
+    elif method == "sqrt":
+        T = np.sqrt(X)
+    elif method == "arcsinh":
+        T = np.log(X + np.sqrt(X * X + 1.0))
+    elif method == "yeo_johnson":                       # X >= 0 branch only: X = max(P, eps) > 0
+        T = np.log(X + 1.0) if lam == 0 else (np.power(X + 1.0, lam) - 1.0) / lam
+    elif method == "average":
+        T = X.copy()
+    else:
+        raise ValueError(method)
+    return T - T.min()
+
+
+def true_mask_transform(P: np.ndarray, tau: float, method: str, lam: float, eps: float) -> np.ndarray:
+    """Sec. 4.2.3 on an Appendix-B amplification: M = [A_tilde >= tau], nothing above the diagonal."""
+    At = amplify_transform(P, method, lam, eps)
+    return np.tril(At >= np.float64(tau)).astype(np.uint8)
+
+
 def capture_average(samples: Sequence[np.ndarray], pcl_max: int, eps: float, dtype=np.float64):
     """Sec. 4.2.2, the averaged attention map of one head over several inputs.
 
@@ -210,10 +237,14 @@ class HeadMask:
 
 
 def head_mask_from_probs(P, S: int, tau: float, mu: float, lam: float = 0.5, eps: float = 1e-8,
-                         min_support: int = 1, keep_probs: bool = False) -> HeadMask:
-    """Steps after the attention map.  fp32 input -> the single-precision threshold chain."""
+                         min_support: int = 1, keep_probs: bool = False, method: str = "boxcox") -> HeadMask:
+    """Steps after the attention map.  fp32 input -> the single-precision threshold chain (Box-Cox, lambda 0.5);
+    any other amplification is decided in float64 with tau, eps, lambda taken at their float32 values."""
     L = P.shape[0]
-    if P.dtype == np.float32:
+    if method != "boxcox" or (P.dtype == np.float32 and lam != 0.5):
+        f = np.float32
+        M = true_mask_transform(P, float(f(tau)), method, float(f(lam)), float(f(eps)))
+    elif P.dtype == np.float32:
         assert lam == 0.5
         M = true_mask_f32(P, tau, eps)
     else:

@@ -48,7 +48,11 @@ class dam_shape_t(ctypes.Structure):
 class dam_rule_t(ctypes.Structure):
     _fields_ = [("struct_size", ctypes.c_uint32), ("pcl_max", ctypes.c_int32), ("tau", ctypes.c_float),
                 ("mu", ctypes.c_float), ("lambda_", ctypes.c_float), ("eps", ctypes.c_float),
-                ("softmax_scale", ctypes.c_float), ("min_support", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+                ("softmax_scale", ctypes.c_float), ("min_support", ctypes.c_int32), ("flags", ctypes.c_uint32),
+                ("transform", ctypes.c_int32)]
+
+
+TRANSFORMS = {"boxcox": 0, "log": 1, "sqrt": 2, "arcsinh": 3, "yeo_johnson": 4, "average": 5}
 
 
 _lib = None
@@ -126,11 +130,13 @@ DAM_RULE_GATHER_COLUMNS = 1
 
 
 def make_rule(pcl_max: int, tau: float, mu: float, lam: float = 0.5, eps: float = 1e-8,
-              softmax_scale: float = 0.0, min_support: int = 1, gather_columns: bool = False) -> dam_rule_t:
+              softmax_scale: float = 0.0, min_support: int = 1, gather_columns: bool = False,
+              transform: str = "boxcox") -> dam_rule_t:
     r = dam_rule_t()
     r.struct_size = ctypes.sizeof(dam_rule_t)
     r.pcl_max, r.tau, r.mu, r.lambda_, r.eps = pcl_max, tau, mu, lam, eps
     r.softmax_scale, r.min_support, r.flags = softmax_scale, min_support, (DAM_RULE_GATHER_COLUMNS if gather_columns else 0)
+    r.transform = TRANSFORMS[transform]
     return r
 
 

@@ -46,7 +46,8 @@ dam_status_t check_rule(const dam_rule_t* r) {
   if (!(r->tau > 0.f) || !(r->eps > 0.f) || !(r->mu == r->mu)) return DAM_ERR_INVALID_ARGUMENT;
   if (r->min_support < 1 || (r->flags & ~DAM_RULE_GATHER_COLUMNS) != 0 || r->softmax_scale < 0.f)
     return DAM_ERR_INVALID_ARGUMENT;
-  if (r->lambda != 0.5f) return DAM_ERR_UNSUPPORTED;
+  if (r->transform < DAM_TRANSFORM_BOXCOX || r->transform > DAM_TRANSFORM_AVERAGE) return DAM_ERR_INVALID_ARGUMENT;
+  if (!(r->lambda == r->lambda) || fabsf(r->lambda) > 64.f) return DAM_ERR_INVALID_ARGUMENT;
   return DAM_OK;
 }
 
@@ -144,23 +145,47 @@ bool chain_active(float p, float tau, float eps) {
   return a >= tau;
 }
 
-float find_pstar(float tau, float eps) {
-  if (!chain_active(1.0f, tau, eps)) {
+// Every other amplification (Appendix B), decided in double precision on the fp32 map value.
+double amplify_f64(double X, int transform, double lam) {
+  switch (transform) {
+    case DAM_TRANSFORM_BOXCOX: return lam == 0.0 ? log(X) : (pow(X, lam) - 1.0) / lam;
+    case DAM_TRANSFORM_LOG: return log(X);
+    case DAM_TRANSFORM_SQRT: return sqrt(X);
+    case DAM_TRANSFORM_ARCSINH: return asinh(X);
+    case DAM_TRANSFORM_YEO_JOHNSON: return lam == 0.0 ? log(X + 1.0) : (pow(X + 1.0, lam) - 1.0) / lam;
+    default: return X;
+  }
+}
+
+struct Rule64 { int transform; double tau, eps, lam; bool chain; float ftau, feps; };
+
+bool rule_active(float p, const Rule64& r) {
+  if (r.chain) return chain_active(p, r.ftau, r.feps);
+  const double X = (double)p > r.eps ? (double)p : r.eps;
+  return amplify_f64(X, r.transform, r.lam) - amplify_f64(r.eps, r.transform, r.lam) >= r.tau;
+}
+
+float find_pstar(const dam_rule_t* rule) {
+  Rule64 r;
+  r.transform = rule->transform; r.tau = (double)rule->tau; r.eps = (double)rule->eps; r.lam = (double)rule->lambda;
+  r.chain = rule->transform == DAM_TRANSFORM_BOXCOX && rule->lambda == 0.5f;
+  r.ftau = rule->tau; r.feps = rule->eps;
+  if (!rule_active(1.0f, r)) {
     // no probability reaches tau; larger (non-softmax) inputs may: search up to the largest float
     uint32_t lo = 0x3F800000u, hi = 0x7F7FFFFFu;
     float fh; memcpy(&fh, &hi, 4);
-    if (!chain_active(fh, tau, eps)) return INFINITY;
+    if (!rule_active(fh, r)) return INFINITY;
     while (hi - lo > 1) {
       uint32_t mid = lo + (hi - lo) / 2; float fm; memcpy(&fm, &mid, 4);
-      if (chain_active(fm, tau, eps)) hi = mid; else lo = mid;
+      if (rule_active(fm, r)) hi = mid; else lo = mid;
     }
     memcpy(&fh, &hi, 4);
     return fh;
   }
-  uint32_t lo = 0u, hi = 0x3F800000u;     // chain(0) is inactive because tau > 0
+  uint32_t lo = 0u, hi = 0x3F800000u;     // the rule is inactive at 0 because tau > 0
   while (hi - lo > 1) {
     uint32_t mid = lo + (hi - lo) / 2; float fm; memcpy(&fm, &mid, 4);
-    if (chain_active(fm, tau, eps)) hi = mid; else lo = mid;
+    if (rule_active(fm, r)) hi = mid; else lo = mid;
   }
   float f; memcpy(&f, &hi, 4);
   return f;
@@ -180,7 +205,7 @@ dam_status_t fill_ctx(const dam_shape_t* s, const dam_rule_t* r, void* mask, siz
   c->num_seqs = s->num_seqs; c->Hq = s->num_q_heads; c->Hkv = s->num_kv_heads; c->d = s->head_dim; c->dtype = s->dtype;
   c->total_qblocks = y->hdr.total_qblocks; c->rows = y->hdr.rows; c->prows = y->hdr.prows;
   c->max_L = y->max_L; c->max_W = y->max_W; c->max_nL = y->max_nL; c->max_nq = y->max_nq;
-  c->pstar = find_pstar(r->tau, r->eps);
+  c->pstar = find_pstar(r);
   c->mu = r->mu; c->min_support = r->min_support;
   c->scale = r->softmax_scale > 0.f ? r->softmax_scale : 1.0f / sqrtf((float)s->head_dim);
   c->off_cnt = y->off_cnt; c->off_cnt_end = y->off_cnt_end; c->off_rowcnt = y->off_rowcnt;

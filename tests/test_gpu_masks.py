@@ -272,3 +272,29 @@ def test_multi_sample_capture_masks_bit_exact():
                                                 w_last.lam, w_last.eps))
         masks.append(row)
     H.check_blob_against_oracle(blob, tshape, masks)
+
+
+@pytest.mark.parametrize("transform,lam,tau", [
+    ("log", 0.0, 13.0), ("sqrt", 0.0, 0.1), ("arcsinh", 0.0, 0.01), ("average", 0.0, 0.01),
+    ("boxcox", 0.25, 1.5), ("boxcox", 0.0, 13.0), ("yeo_johnson", 0.5, 0.01), ("yeo_johnson", 0.0, 0.01),
+])
+def test_other_amplifications_bit_exact_from_scores(transform, lam, tau):
+    """The Appendix-B amplifications through the C ABI: the same fp32 score tensor on both sides, masks bit-exact
+    (true mask, D, V and the tile lists of sampled query blocks)."""
+    w = synth.small_case(0, 4, 2, 64, 160, seed=40, dtype=torch.bfloat16, lengths=[500, 120])
+    shape = B.make_shape(w.cu_seqlens, 4, 2, 64, w.Q.dtype, DEV)
+    n = sum(4 * min(S, 160) ** 2 for S in shape.lengths)
+    dump = torch.zeros(n, dtype=torch.float32, device=DEV)
+    B.dam_build_masks(w.Q.to(DEV), w.K.to(DEV), shape, B.make_rule(160, w.tau, w.mu), scores_dump=dump)
+    rule = B.make_rule(160, tau, w.mu, lam, w.eps, transform=transform)
+    blob, _ = B.dam_build_masks_from_scores(dump, shape, rule)
+    assert B.dam_poll_status(blob) == 0
+    # and the fused scoring path decides on the same values
+    blob2, _ = B.dam_build_masks(w.Q.to(DEV), w.K.to(DEV), shape, rule)
+    P = H.split_dump(dump.cpu().numpy(), shape.lengths, 4, 160)
+    masks = [[orc.head_mask_from_probs(np.ascontiguousarray(P[b][h]), S, tau, w.mu, lam, w.eps, method=transform)
+              for h in range(4)] for b, S in enumerate(shape.lengths)]
+    active = sum(int(m.M.sum()) for row in masks for m in row)
+    assert active > 0
+    H.check_blob_against_oracle(blob, shape, masks)
+    H.check_blob_against_oracle(blob2, shape, masks)

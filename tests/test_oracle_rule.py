@@ -365,3 +365,59 @@ def test_capture_average_float32_tracks_float64():
     a64, c64 = orc.capture_average(samples, 9, 1e-8, dtype=np.float64)
     assert np.array_equal(c32, c64) and c64.tolist() == [5, 5, 5, 4, 4, 3, 3, 2, 2]
     assert np.abs(a32 - a64).max() < 1e-6
+
+
+# ---------------------------------------------------------------------------------------------
+# Other amplifications (Appendix B): each is increasing, so its mask is a threshold on the map at the
+# inverse function's value; the inverses below are written out independently of the oracle's forward formulas
+# ---------------------------------------------------------------------------------------------
+def _inverse_threshold(method, tau, lam, eps):
+    if method == "log":
+        return eps * math.exp(tau)
+    if method == "sqrt":
+        return (tau + math.sqrt(eps)) ** 2
+    if method == "arcsinh":
+        return math.sinh(tau + math.asinh(eps))
+    if method == "average":
+        return tau + eps
+    if method == "boxcox":
+        return eps * math.exp(tau) if lam == 0 else (lam * tau + eps ** lam) ** (1.0 / lam)
+    if method == "yeo_johnson":
+        return (eps + 1.0) * math.exp(tau) - 1.0 if lam == 0 else (lam * tau + (eps + 1.0) ** lam) ** (1.0 / lam) - 1.0
+    raise ValueError(method)
+
+
+@pytest.mark.parametrize("method,lam,tau", [
+    ("log", 0.0, 12.0), ("sqrt", 0.0, 0.15), ("arcsinh", 0.0, 0.02), ("average", 0.0, 0.03),
+    ("boxcox", 0.5, 0.3), ("boxcox", 0.25, 1.0), ("boxcox", 0.0, 12.0), ("boxcox", 1.0, 0.03),
+    ("yeo_johnson", 0.5, 0.02), ("yeo_johnson", 0.0, 0.02), ("yeo_johnson", 2.0, 0.05),
+])
+def test_transform_mask_is_threshold_at_inverse(method, lam, tau):
+    eps = 1e-8
+    rng = np.random.default_rng(11)
+    L = 96
+    P = np.tril(rng.random((L, L)) ** 6)
+    P /= P.sum(axis=1, keepdims=True)
+    M = orc.true_mask_transform(P, tau, method, lam, eps)
+    x = _inverse_threshold(method, tau, lam, eps)
+    near = np.abs(P - x) <= 1e-9 * max(x, 1e-30)                   # cells within rounding of the threshold
+    want = np.tril(P >= x)
+    assert np.array_equal(M.astype(bool) | near, want | near)
+    assert 0 < M.sum() < L * (L + 1) // 2                            # the case separates something
+    assert not np.triu(M, 1).any()
+
+
+def test_transform_boxcox_half_equals_the_default_path_and_sqrt_is_its_half():
+    rng = np.random.default_rng(12)
+    P = np.tril(rng.random((64, 64)) ** 4)
+    P /= P.sum(axis=1, keepdims=True)
+    A = orc.amplify_transform(P, "boxcox", 0.5, 1e-8)
+    assert np.allclose(A, orc.amplify_f64(P, 0.5, 1e-8), atol=1e-12)
+    assert np.allclose(A, 2.0 * orc.amplify_transform(P, "sqrt", 0.0, 1e-8), atol=1e-12)   # 2 (sqrt X - sqrt eps)
+    assert np.array_equal(orc.true_mask_transform(P, 0.3, "boxcox", 0.5, 1e-8), orc.true_mask_f64(P, 0.3, 0.5, 1e-8))
+    # every amplification is zero at its minimum and increasing in the map value
+    for m, lam in (("log", 0), ("arcsinh", 0), ("average", 0), ("yeo_johnson", 0.5), ("boxcox", 0.1)):
+        T = orc.amplify_transform(P, m, lam, 1e-8)
+        assert T.min() == 0.0
+        order = np.argsort(P, axis=None)
+        assert np.all(np.diff(T.reshape(-1)[order]) >= -1e-15)
