@@ -561,8 +561,15 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         PROF_LAP(1)
         ++cS;
         tc_fence_after();
-        // ---- sweep 1: row maximum of the raw dot products (masked entries excluded)
-        const float mx = need_mask ? sweep_max<true>(tS, bits) : sweep_max<false>(tS, bits);
+        // ---- sweep 1: row maximum of the raw dot products.  On a masked tile the maximum over all entries is
+        //      tried first: it bounds the masked one from above, so when it does not exceed the reference by more
+        //      than the threshold for any row of the warp, the reference stays where it is and the masked
+        //      maximum (two more instructions per element) is never needed.  The result is the same either way.
+        float mx = sweep_max<false>(tS, bits);
+        if (need_mask) {
+          const bool over = (t == t0) || (mx * prm.scale_log2 - m_ref > kRescaleThreshold);   // -inf reference: true
+          mx = __any_sync(0xFFFFFFFFu, over) ? sweep_max<true>(tS, bits) : -CUDART_INF_F;
+        }
         PROF_LAP(2)
         const float m_new = fmaxf(m_ref, mx * prm.scale_log2);
         // move the reference only on the first tile or when the max grew by more than the threshold
