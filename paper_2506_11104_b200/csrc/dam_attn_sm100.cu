@@ -565,11 +565,14 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         //      tried first: it bounds the masked one from above, so when it does not exceed the reference by more
         //      than the threshold for any row of the warp, the reference stays where it is and the masked
         //      maximum (two more instructions per element) is never needed.  The result is the same either way.
-        float mx = sweep_max<false>(tS, bits);
-        if (need_mask) {
-          const bool over = (t == t0) || (mx * prm.scale_log2 - m_ref > kRescaleThreshold);   // -inf reference: true
-          mx = __any_sync(0xFFFFFFFFu, over) ? sweep_max<true>(tS, bits) : -CUDART_INF_F;
+        bool masked_max = need_mask && (t == t0);            // the first tile sets the reference
+        float mx = -CUDART_INF_F;
+        if (!masked_max) {
+          const float mu = sweep_max<false>(tS, bits);
+          if (!need_mask) mx = mu;
+          else masked_max = __any_sync(0xFFFFFFFFu, mu * prm.scale_log2 - m_ref > kRescaleThreshold);   // -inf reference: true
         }
+        if (masked_max) mx = sweep_max<true>(tS, bits);
         PROF_LAP(2)
         const float m_new = fmaxf(m_ref, mx * prm.scale_log2);
         // move the reference only on the first tile or when the max grew by more than the threshold
