@@ -257,6 +257,7 @@ dam_status_t dam_build_masks(const void* Q, const void* K, const dam_shape_t* sh
   if (!Q || !K || !aligned(Q, 16) || !aligned(K, 16) || (scores_dump && !aligned(scores_dump, 16)))
     return DAM_ERR_INVALID_ARGUMENT;
   cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
+  if (dam_launch_rule_prepare(c, cs) != cudaSuccess) return DAM_ERR_CUDA;
   if (dam_launch_init_blob(shape, rule->pcl_max, y.hdr.flags, mask, y.hdr, cs) != cudaSuccess)
     return DAM_ERR_CUDA;
   cudaError_t e = cudaErrorNotSupported;
@@ -275,6 +276,7 @@ dam_status_t dam_build_masks_from_scores(const float* P, const dam_shape_t* shap
   if (st != DAM_OK) return st;
   if (!P || !aligned(P, 4)) return DAM_ERR_INVALID_ARGUMENT;
   cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
+  if (dam_launch_rule_prepare(c, cs) != cudaSuccess) return DAM_ERR_CUDA;
   if (dam_launch_init_blob(shape, rule->pcl_max, y.hdr.flags, mask, y.hdr, cs) != cudaSuccess)
     return DAM_ERR_CUDA;
   if (dam_launch_bits_from_scores(P, c, cs) != cudaSuccess) return DAM_ERR_CUDA;

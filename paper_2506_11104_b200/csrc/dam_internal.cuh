@@ -209,6 +209,7 @@ cudaError_t dam_launch_init_blob(const dam_shape_t* shape, int pcl_max, uint32_t
 cudaError_t dam_launch_scores_ref(const void* Q, const void* K, const dam_shape_t* shape, const DamBuildCtx& c,
                                   float* scores_dump, cudaStream_t st);
 cudaError_t dam_launch_bits_from_scores(const float* P, const DamBuildCtx& c, cudaStream_t st);
+cudaError_t dam_launch_rule_prepare(const DamBuildCtx& c, cudaStream_t st);   // before the true mask is produced
 cudaError_t dam_launch_rule(const DamBuildCtx& c, cudaStream_t st);
 cudaError_t dam_launch_all_ones(const dam_shape_t* shape, int causal, void* blob, cudaStream_t st);
 cudaError_t dam_launch_expand_rows(const void* blob, int seq, int head, int row_begin, int nrows, int words,

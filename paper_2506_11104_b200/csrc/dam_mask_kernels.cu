@@ -7,6 +7,26 @@
 
 namespace {
 
+// The rule kernels form a chain of short, dependent launches.  Each lets the next launch begin as soon as all
+// of its own blocks are running (programmatic dependent launch) and then waits for the kernel before it to
+// have completed with its memory visible: the launch latency of every link is hidden under its predecessor.
+// Both instructions do nothing in a kernel that was launched the ordinary way.
+__device__ __forceinline__ void dam_chain_prologue() {
+  asm volatile("griddepcontrol.launch_dependents;");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = 0; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 __device__ __forceinline__ const DamSeq* blob_seqs(const unsigned char* blob, const DamHeader* h) {
   return reinterpret_cast<const DamSeq*>(blob + h->off_seq);
 }
@@ -86,6 +106,7 @@ __global__ void bits_from_scores_kernel(unsigned char* blob, const float* __rest
 // accumulated in shared memory and flushed with integer atomics (order-independent).
 // ---------------------------------------------------------------------------------------------
 __global__ void counts_kernel(const unsigned char* blob, unsigned char* scratch, uint64_t off_cnt) {
+  dam_chain_prologue();
   const DamHeader* H = reinterpret_cast<const DamHeader*>(blob);
   const int sh = blockIdx.y;
   const int b = sh / H->num_q_heads, h = sh % H->num_q_heads;
@@ -150,6 +171,7 @@ __global__ void counts_kernel(const unsigned char* blob, unsigned char* scratch,
 // as bit sets; Drev = D reversed; prefix popcounts per word for range queries.  Block per (seq, head).
 // ---------------------------------------------------------------------------------------------
 __global__ void match_kernel(unsigned char* blob, unsigned char* scratch, uint64_t off_cnt, float mu, int min_support) {
+  dam_chain_prologue();
   const DamHeader* H = reinterpret_cast<const DamHeader*>(blob);
   const int sh = blockIdx.x;
   const int b = sh / H->num_q_heads, h = sh % H->num_q_heads;
@@ -275,6 +297,7 @@ __device__ __forceinline__ uint32_t classify_band(const HeadView& v, int qb, int
 template <int PASS>
 __global__ void classify_kernel(unsigned char* blob, unsigned char* scratch, uint64_t off_cnt, uint64_t off_rowcnt,
                                 uint64_t off_hist, uint64_t off_cursor) {
+  dam_chain_prologue();
   DamHeader* H = reinterpret_cast<DamHeader*>(blob);
   const int lane = threadIdx.x & 31;
   const int prow = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);   // one warp per (head, q-block pair)
@@ -404,6 +427,7 @@ __device__ uint32_t block_excl_scan(uint32_t x, uint32_t* total, uint32_t* sm /*
 
 __global__ void scan_kernel(unsigned char* blob, unsigned char* scratch, uint64_t off_rowcnt, uint64_t off_hist,
                             uint64_t off_cursor) {
+  dam_chain_prologue();
   DamHeader* H = reinterpret_cast<DamHeader*>(blob);
   __shared__ uint32_t sm[32];
   __shared__ uint32_t tot;
@@ -650,21 +674,30 @@ cudaError_t dam_launch_capture_average(const float* A, const int32_t* C, int Lma
   return cudaGetLastError();
 }
 
+// The counters of the rule kernels start at zero: counts + prefix + tile popcounts, row counts, histogram,
+// cursors.  Enqueued before the kernel that produces the true mask, so that the rule kernels follow it directly.
+cudaError_t dam_launch_rule_prepare(const DamBuildCtx& c, cudaStream_t st) {
+  cudaError_t e;
+  if ((e = cudaMemsetAsync(c.scratch + c.off_cnt, 0, c.off_cnt_end - c.off_cnt, st)) != cudaSuccess) return e;
+  return cudaMemsetAsync(c.scratch + c.off_hist, 0, 2ull * DAM_HIST * 4, st);
+}
+
 cudaError_t dam_launch_rule(const DamBuildCtx& c, cudaStream_t st) {
   cudaError_t e;
-  // counters start at zero: counts + prefix + tile popcounts, row counts, histogram, cursors
-  if ((e = cudaMemsetAsync(c.scratch + c.off_cnt, 0, c.off_cnt_end - c.off_cnt, st)) != cudaSuccess) return e;
-  if ((e = cudaMemsetAsync(c.scratch + c.off_hist, 0, 2ull * DAM_HIST * 4, st)) != cudaSuccess) return e;
   if (c.max_nL > 0) {
     dim3 g(c.max_nL * (c.max_nL + 1) / 2, c.num_seqs * c.Hq);
     counts_kernel<<<g, DAM_TILE, 0, st>>>(c.blob, c.scratch, c.off_cnt);
-    match_kernel<<<c.num_seqs * c.Hq, 256, 0, st>>>(c.blob, c.scratch, c.off_cnt, c.mu, c.min_support);
+    if ((e = launch_chained(match_kernel, dim3(c.num_seqs * c.Hq), dim3(256), st, c.blob, c.scratch, c.off_cnt, c.mu,
+                            c.min_support)) != cudaSuccess) return e;
   }
   if (c.rows > 0) {
     int blocks = (c.prows + 7) / 8;
-    classify_kernel<0><<<blocks, 256, 0, st>>>(c.blob, c.scratch, c.off_cnt, c.off_rowcnt, c.off_hist, c.off_cursor);
-    scan_kernel<<<1, 1024, 0, st>>>(c.blob, c.scratch, c.off_rowcnt, c.off_hist, c.off_cursor);
-    classify_kernel<1><<<blocks, 256, 0, st>>>(c.blob, c.scratch, c.off_cnt, c.off_rowcnt, c.off_hist, c.off_cursor);
+    if ((e = launch_chained(classify_kernel<0>, dim3(blocks), dim3(256), st, c.blob, c.scratch, c.off_cnt, c.off_rowcnt,
+                            c.off_hist, c.off_cursor)) != cudaSuccess) return e;
+    if ((e = launch_chained(scan_kernel, dim3(1), dim3(1024), st, c.blob, c.scratch, c.off_rowcnt, c.off_hist,
+                            c.off_cursor)) != cudaSuccess) return e;
+    if ((e = launch_chained(classify_kernel<1>, dim3(blocks), dim3(256), st, c.blob, c.scratch, c.off_cnt, c.off_rowcnt,
+                            c.off_hist, c.off_cursor)) != cudaSuccess) return e;
   }
   return cudaGetLastError();
 }
