@@ -211,50 +211,58 @@ __device__ __forceinline__ float sweep_max(uint32_t tS, const uint4& bits) {
 // bf16 rounding).  A masked tile skips the arithmetic of a 32-column chunk that is inactive for every row of
 // the warp.
 template <bool MASKED>
+__device__ __forceinline__ void exp_chunk(const uint32_t* cur, uint32_t word, float scale, float neg_m, uint32_t* pk,
+                                          float& s0, float& s1, float& s2, float& s3) {
+  const bool live = !MASKED || __any_sync(0xFFFFFFFFu, word != 0u);
+  if (live) {
+#pragma unroll
+    for (int q = 0; q < 32; q += 8) {
+      float y[8], p[8];
+#pragma unroll
+      for (int u = 0; u < 8; u += 2)
+        fma2(y[u], y[u + 1], __uint_as_float(cur[q + u]), __uint_as_float(cur[q + u + 1]), scale, scale, neg_m, neg_m);
+#pragma unroll
+      for (int u = 0; u < 8 - kPolyPer8; ++u) p[u] = ex2(y[u]);
+      if (kPolyPer8 >= 2) ex2_poly2(y[6], y[7], p[6], p[7]);
+      if (kPolyPer8 >= 4) ex2_poly2(y[4], y[5], p[4], p[5]);
+      if (MASKED) {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) p[u] = ((word >> (q + u)) & 1u) ? p[u] : 0.f;
+      }
+      add2(s0, s1, s0, s1, p[0], p[1]);
+      add2(s2, s3, s2, s3, p[2], p[3]);
+      add2(s0, s1, s0, s1, p[4], p[5]);
+      add2(s2, s3, s2, s3, p[6], p[7]);
+#pragma unroll
+      for (int u = 0; u < 8; u += 2) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(p[u], p[u + 1]);
+        pk[(q + u) >> 1] = *reinterpret_cast<uint32_t*>(&h);
+      }
+    }
+  } else {
+#pragma unroll
+    for (int q = 0; q < 16; ++q) pk[q] = 0u;
+  }
+}
+
+template <bool MASKED>
 __device__ __forceinline__ float sweep_exp(uint32_t tS, const uint4& bits, float scale, float neg_m) {
   uint32_t ra[32], rb[32];
   float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
   tmem_ld32(tS, ra);
   tc_wait_ld();
-#pragma unroll
-  for (int c = 0; c < 4; ++c) {
-    uint32_t* cur = (c & 1) ? rb : ra;
-    uint32_t* nxt = (c & 1) ? ra : rb;
-    if (c < 3) tmem_ld32(tS + (c + 1) * 32, nxt);
-    const uint32_t word = pick_word(bits, c);
+  // two chunks per trip (one in each register set), the loop itself is not unrolled: half the code
+#pragma unroll 1
+  for (int cc = 0; cc < 2; ++cc) {
     uint32_t pk[16];
-    const bool live = !MASKED || __any_sync(0xFFFFFFFFu, word != 0u);
-    if (live) {
-#pragma unroll
-      for (int q = 0; q < 32; q += 8) {
-        float y[8], p[8];
-#pragma unroll
-        for (int u = 0; u < 8; u += 2)
-          fma2(y[u], y[u + 1], __uint_as_float(cur[q + u]), __uint_as_float(cur[q + u + 1]), scale, scale, neg_m, neg_m);
-#pragma unroll
-        for (int u = 0; u < 8 - kPolyPer8; ++u) p[u] = ex2(y[u]);
-        if (kPolyPer8 >= 2) ex2_poly2(y[6], y[7], p[6], p[7]);
-        if (kPolyPer8 >= 4) ex2_poly2(y[4], y[5], p[4], p[5]);
-        if (MASKED) {
-#pragma unroll
-          for (int u = 0; u < 8; ++u) p[u] = ((word >> (q + u)) & 1u) ? p[u] : 0.f;
-        }
-        add2(s0, s1, s0, s1, p[0], p[1]);
-        add2(s2, s3, s2, s3, p[2], p[3]);
-        add2(s0, s1, s0, s1, p[4], p[5]);
-        add2(s2, s3, s2, s3, p[6], p[7]);
-#pragma unroll
-        for (int u = 0; u < 8; u += 2) {
-          __nv_bfloat162 h = __floats2bfloat162_rn(p[u], p[u + 1]);
-          pk[(q + u) >> 1] = *reinterpret_cast<uint32_t*>(&h);
-        }
-      }
-    } else {
-#pragma unroll
-      for (int q = 0; q < 16; ++q) pk[q] = 0u;
-    }
-    if (c < 3) tc_wait_ld();
-    tmem_st16(tS + c * 16, pk);
+    tmem_ld32(tS + (2 * cc + 1) * 32, rb);
+    exp_chunk<MASKED>(ra, cc ? bits.z : bits.x, scale, neg_m, pk, s0, s1, s2, s3);
+    tc_wait_ld();
+    tmem_st16(tS + (2 * cc) * 16, pk);
+    if (cc == 0) tmem_ld32(tS + 2 * 32, ra);
+    exp_chunk<MASKED>(rb, cc ? bits.w : bits.y, scale, neg_m, pk, s0, s1, s2, s3);
+    if (cc == 0) tc_wait_ld();
+    tmem_st16(tS + (2 * cc + 1) * 16, pk);
   }
   return (s0 + s1) + (s2 + s3);
 }
