@@ -260,7 +260,7 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         uint4 words = make_uint4(0u, 0u, 0u, 0u);
         float tmax = -CUDART_INF_F, tsum = 0.f;
         uint32_t cur[32];
-#pragma unroll
+#pragma unroll 1
         for (int c = 0; c < 4; ++c) {
           tmem_ld32(tS + c * 32, cur);
           tc_wait_ld();
