@@ -95,8 +95,12 @@ typedef struct dam_rule_t {
  * BOXCOX with lambda = 0.5 is decided by a chain of IEEE single operations (so that two implementations can
  * agree bit for bit: x = max(p, eps); b = (sqrt(x) - 1) * 2; a = b - (sqrt(eps) - 1) * 2; a >= tau); every
  * other case is decided in double precision on the fp32 map value, with tau, eps, lambda widened from float.
- * Z-score and min-max normalisation (which need the mean / deviation / maximum of each map) and the raw sum are
- * not offered.
+ * ZSCORE and MINMAX normalise each map by its own statistics over all L x L cells of X (cells above the diagonal
+ * count as eps): (X - mean) / (std + eps) with the population deviation, and (X - min) / (max - min + eps). After
+ * the minimum is subtracted they read (X - eps) / (std + eps) >= tau and (X - eps) / (max - eps + eps) >= tau, a
+ * threshold per map, decided in double precision. They need a pass over the finished map, so only
+ * dam_build_masks_from_scores offers them (dam_build_masks returns UNSUPPORTED). The raw sum (Appendix B,
+ * method 1) is the average times the sample count and is not offered separately.
  */
 typedef enum dam_transform_t {
   DAM_TRANSFORM_BOXCOX = 0,
@@ -104,7 +108,9 @@ typedef enum dam_transform_t {
   DAM_TRANSFORM_SQRT = 2,
   DAM_TRANSFORM_ARCSINH = 3,
   DAM_TRANSFORM_YEO_JOHNSON = 4,
-  DAM_TRANSFORM_AVERAGE = 5
+  DAM_TRANSFORM_AVERAGE = 5,
+  DAM_TRANSFORM_ZSCORE = 6,
+  DAM_TRANSFORM_MINMAX = 7
 } dam_transform_t;
 
 /*

@@ -172,8 +172,9 @@ def attention_rows(Qh: np.ndarray, Kh: np.ndarray, Vh: np.ndarray, rows: Sequenc
 
 
 def amplify_transform(P: np.ndarray, method: str, lam: float, eps: float) -> np.ndarray:
-    """Appendix B: the amplification methods that act cell by cell, on X = max(P, eps), in float64,
-    followed by the subtraction of the minimum over the whole map (cells above the diagonal included)."""
+    """Appendix B: the amplification methods on X = max(P, eps), in float64 (z-score and min-max take their
+    statistics over every cell of the map), followed by the subtraction of the minimum over the whole map
+    (cells above the diagonal included)."""
     X = np.maximum(np.asarray(P, dtype=np.float64), np.float64(eps))
     if method == "boxcox":
         T = np.log(X) if lam == 0 else (np.power(X, lam) - 1.0) / lam
@@ -187,6 +188,10 @@ def amplify_transform(P: np.ndarray, method: str, lam: float, eps: float) -> np.
         T = np.log(X + 1.0) if lam == 0 else (np.power(X + 1.0, lam) - 1.0) / lam
     elif method == "average":
         T = X.copy()
+    elif method == "zscore":                            # statistics over every cell of the map, population deviation
+        T = (X - X.mean()) / (X.std() + np.float64(eps))
+    elif method == "minmax":
+        T = (X - X.min()) / (X.max() - X.min() + np.float64(eps))
     else:
         raise ValueError(method)
     return T - T.min()

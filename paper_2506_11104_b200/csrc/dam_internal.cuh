@@ -196,6 +196,8 @@ struct DamBuildCtx {
   int total_qblocks, rows, prows;
   int max_L, max_W, max_nL, max_nq;
   float pstar;       // single-compare threshold on p equivalent to the Box-Cox chain
+  int per_map;       // 0, or the dam_transform_t whose threshold depends on each map's own statistics
+  float tau, eps;    // for the per-map thresholds
   float mu;
   int min_support;
   float scale;

@@ -593,12 +593,97 @@ cudaError_t dam_launch_init_blob(const dam_shape_t* shape, int pcl_max, uint32_t
   return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------------------------
+// Z-score / min-max (Appendix B): statistics of X = max(P, eps) over all L x L cells of one map (cells above
+// the diagonal are eps), in double, one block per map with a fixed reduction order; then the true mask with
+// the map's own threshold  X >= eps + tau (std + eps)  or  X >= eps + tau (max - eps + eps).
+// ---------------------------------------------------------------------------------------------
+struct DamMapStats { double sum, sumsq; float mx; float pad; };
+
+__global__ void __launch_bounds__(1024)
+map_stats_kernel(const unsigned char* blob, const float* __restrict__ P, unsigned char* scratch, uint64_t off_cnt, float eps) {
+  const DamHeader* H = reinterpret_cast<const DamHeader*>(blob);
+  const int sh = blockIdx.x;
+  const int b = sh / H->num_q_heads, h = sh % H->num_q_heads;
+  const DamSeq sq = blob_seqs(blob, H)[b];
+  if (sq.L == 0) return;
+  const int L = sq.L;
+  const float* Ph = P + sq.p_off + (uint64_t)h * L * L;
+  double s = 0.0, s2 = 0.0;
+  float mx = eps;
+  for (long long idx = threadIdx.x; idx < (long long)L * L; idx += blockDim.x) {
+    const int i = (int)(idx / L), j = (int)(idx % L);
+    const float x = fmaxf(j <= i ? __ldg(Ph + idx) : 0.f, eps);
+    s += (double)x; s2 += (double)x * (double)x;
+    mx = fmaxf(mx, x);
+  }
+  __shared__ double sh_s[1024], sh_s2[1024];
+  __shared__ float sh_mx[1024];
+  sh_s[threadIdx.x] = s; sh_s2[threadIdx.x] = s2; sh_mx[threadIdx.x] = mx;
+  __syncthreads();
+  for (int o = blockDim.x >> 1; o > 0; o >>= 1) {
+    if ((int)threadIdx.x < o) {
+      sh_s[threadIdx.x] += sh_s[threadIdx.x + o];
+      sh_s2[threadIdx.x] += sh_s2[threadIdx.x + o];
+      sh_mx[threadIdx.x] = fmaxf(sh_mx[threadIdx.x], sh_mx[threadIdx.x + o]);
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    DamMapStats* st = reinterpret_cast<DamMapStats*>(reinterpret_cast<int32_t*>(scratch + off_cnt) + sq.cnt_off +
+                                                     (uint64_t)h * dam_cnt_stride(sq.L, sq.W, sq.nL));
+    st->sum = sh_s[0]; st->sumsq = sh_s2[0]; st->mx = sh_mx[0]; st->pad = 0.f;
+  }
+}
+
+__global__ void bits_from_scores_per_map_kernel(unsigned char* blob, const float* __restrict__ P,
+                                                const unsigned char* scratch, uint64_t off_cnt, int transform,
+                                                float tau_f, float eps_f) {
+  const DamHeader* H = reinterpret_cast<const DamHeader*>(blob);
+  const int sh = blockIdx.y;
+  const int b = sh / H->num_q_heads, h = sh % H->num_q_heads;
+  const DamSeq sq = blob_seqs(blob, H)[b];
+  if (sq.L == 0) return;
+  const DamMapStats st = *reinterpret_cast<const DamMapStats*>(reinterpret_cast<const int32_t*>(scratch + off_cnt) + sq.cnt_off +
+                                                               (uint64_t)h * dam_cnt_stride(sq.L, sq.W, sq.nL));
+  const double tau = (double)tau_f, eps = (double)eps_f, N = (double)sq.L * (double)sq.L;
+  double thr;
+  if (transform == DAM_TRANSFORM_ZSCORE) {
+    const double mean = st.sum / N;
+    const double var = st.sumsq / N - mean * mean;
+    thr = eps + tau * (sqrt(var > 0.0 ? var : 0.0) + eps);
+  } else {
+    thr = eps + tau * (((double)st.mx - eps) + eps);
+  }
+  uint32_t* M = reinterpret_cast<uint32_t*>(blob + H->off_true) + sq.true_off + (uint64_t)h * sq.L * sq.W;
+  const float* Ph = P + sq.p_off + (uint64_t)h * sq.L * sq.L;
+  const int lane = threadIdx.x & 31;
+  const long long nitems = (long long)sq.L * sq.W;
+  const long long wstride = (long long)gridDim.x * (blockDim.x >> 5);
+  for (long long it = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); it < nitems; it += wstride) {
+    const int i = (int)(it / sq.W), w = (int)(it % sq.W);
+    const int j = w * 32 + lane;
+    const bool in = j < sq.L && j <= i;
+    const float x = fmaxf(in ? __ldg(Ph + (size_t)i * sq.L + j) : 0.0f, eps_f);
+    const uint32_t word = __ballot_sync(0xFFFFFFFFu, in && (double)x >= thr);
+    if (lane == 0) M[(size_t)i * sq.W + w] = word;
+  }
+}
+
 cudaError_t dam_launch_bits_from_scores(const float* P, const DamBuildCtx& c, cudaStream_t st) {
   if (c.max_L == 0) return cudaSuccess;
   long long items = (long long)c.max_L * c.max_W;
   int bx = (int)((items + 7) / 8);
   if (bx > 4096) bx = 4096;
   dim3 grid(bx, c.num_seqs * c.Hq);
+  if (c.per_map) {
+    // the statistics borrow the first bytes of every map's counter area, which is cleared again afterwards
+    map_stats_kernel<<<c.num_seqs * c.Hq, 1024, 0, st>>>(c.blob, P, c.scratch, c.off_cnt, c.eps);
+    bits_from_scores_per_map_kernel<<<grid, 256, 0, st>>>(c.blob, P, c.scratch, c.off_cnt, c.per_map, c.tau, c.eps);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    return cudaMemsetAsync(c.scratch + c.off_cnt, 0, c.off_cnt_end - c.off_cnt, st);
+  }
   bits_from_scores_kernel<<<grid, 256, 0, st>>>(c.blob, P, c.pstar);
   return cudaGetLastError();
 }

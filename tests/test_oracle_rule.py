@@ -421,3 +421,25 @@ def test_transform_boxcox_half_equals_the_default_path_and_sqrt_is_its_half():
         assert T.min() == 0.0
         order = np.argsort(P, axis=None)
         assert np.all(np.diff(T.reshape(-1)[order]) >= -1e-15)
+
+
+def test_zscore_and_minmax_masks_are_thresholds_on_the_map_statistics():
+    """(X - mean) / (std + eps) and (X - min) / (max - min + eps), minus their minima, against the thresholds
+    worked out by hand: X >= eps + tau (std + eps) and X >= eps + tau (max - eps + eps)."""
+    eps = 1e-8
+    rng = np.random.default_rng(21)
+    L = 80
+    P = np.tril(rng.random((L, L)) ** 5)
+    P /= P.sum(axis=1, keepdims=True)
+    X = np.maximum(P, eps)                                   # every cell, eps above the diagonal
+    mean = X.sum() / X.size
+    std = math.sqrt(((X - mean) ** 2).sum() / X.size)        # population deviation, written out
+    for method, tau, thr in (("zscore", 1.5, eps + 1.5 * (std + eps)), ("minmax", 0.2, eps + 0.2 * (X.max() - eps + eps))):
+        M = orc.true_mask_transform(P, tau, method, 0.0, eps)
+        near = np.abs(X - thr) <= 1e-9 * thr
+        assert np.array_equal(M.astype(bool) | near, np.tril(X >= thr) | near)
+        assert 0 < M.sum() < L * (L + 1) // 2
+    A = orc.amplify_transform(P, "minmax", 0.0, eps)
+    assert A.min() == 0.0 and 0.999 < A.max() < 1.0          # (max - min) / (max - min + eps)
+    Z = orc.amplify_transform(P, "zscore", 0.0, eps)
+    assert Z.min() == 0.0 and abs((Z - Z.mean()).std() - std / (std + eps)) < 1e-9
