@@ -251,3 +251,22 @@ def test_row_ranges_leave_other_rows_alone_and_reject_odd_bounds():
     for bad in ([(128, 512), (0, 0)], [(0, 300), (0, 0)], [(0, 1024), (0, 0)], [(512, 256), (0, 0)]):
         with pytest.raises(B.DamError):
             B.dam_sparse_attention_rows(Q, K, V, blob, shape, bad, O, lse)
+
+
+@pytest.mark.parametrize("gather", [False, True])
+def test_inactive_keys_with_huge_logits(gather):
+    """Keys outside every pattern whose logits dwarf the active ones (K rows below the window scaled up): the
+    row maximum over all entries of a tile then lies far above the masked one, which is the case the softmax
+    must detect (the reference may only follow the masked maximum) and must survive without overflow."""
+    w = synth.small_case(0, 4, 2, 128, 128, seed=31, dtype=torch.bfloat16, lengths=[1280, 520])
+    rng = np.random.default_rng(5)
+    K = w.K.clone()
+    for b, S in enumerate([1280, 520]):
+        t0 = w.cu_seqlens[b]
+        rows = rng.choice(np.arange(128, S), size=(S - 128) // 3, replace=False)
+        K[t0 + torch.as_tensor(rows)] *= 12.0                # logits up to a few hundred in either direction
+    w.K = K
+    if hasattr(w, "_host_qkv"):
+        del w._host_qkv
+    _, _, _, _, _, worst = _masked_case(w, _sample_rows(128), gather=gather)
+    assert all(np.isfinite(worst))
