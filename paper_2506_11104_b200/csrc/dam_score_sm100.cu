@@ -55,10 +55,15 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-__device__ __forceinline__ void mul2(float& d0, float& d1, float a0, float a1, float b0, float b1) {
-  asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
-      "mul.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
-      : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+__device__ __forceinline__ void fma2(float& d0, float& d1, float a0, float a1, float b0, float b1, float c0, float c1) {
+  asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%6, %7};\n\t"
+      "fma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1), "f"(c0), "f"(c1));
 }
 __device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1, float b0, float b1) {
   asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
@@ -224,7 +229,7 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       uint32_t* Mrow = reinterpret_cast<uint32_t*>(blob + H->off_true) + it.sq.true_off + (uint64_t)it.h * L * W + (size_t)i * W;
       float* Prow = prm.dump ? prm.dump + it.sq.p_off + (uint64_t)it.h * L * L + (size_t)i * L : nullptr;
       const int nk = it.qb + 1;
-      float m = -CUDART_INF_F, l = 0.f, inv_l = 0.f, thr_lo = 0.f;
+      float m = -CUDART_INF_F, l = 0.f, inv_l = 0.f, thr_raw = 0.f;
       for (int t = 0; t < 2 * nk; ++t, ++g) {
         if (t == nk) {
           // all groups have finished sweep A: merge their (max, sum) per row through shared memory
@@ -244,7 +249,7 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           }
           m = mn; l = ls;
           inv_l = l > 0.f ? 1.0f / l : 0.f;
-          thr_lo = log2f(prm.pstar * l) - 0.03125f;
+          thr_raw = (log2f(prm.pstar * l) - 0.03125f + m) / prm.scale_log2;   // the same bound on the raw dot product
         }
         if ((g & 3u) != (uint32_t)G) continue;
         const int kb = t % nk;
@@ -264,32 +269,31 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         for (int c = 0; c < 4; ++c) {
           tmem_ld32(tS + c * 32, cur);
           tc_wait_ld();
+          // raw dot products; the softmax scale (in log2 units) is applied inside the exponent's multiply-add
           float x[32];
 #pragma unroll
-          for (int q = 0; q < 32; q += 2)
-            mul2(x[q], x[q + 1], __uint_as_float(cur[q]), __uint_as_float(cur[q + 1]), prm.scale_log2, prm.scale_log2);
+          for (int q = 0; q < 32; ++q) x[q] = __uint_as_float(cur[q]);
           if (diag) {
 #pragma unroll
             for (int q = 0; q < 32; ++q) x[q] = (c * 32 + q < nvalid) ? x[q] : -CUDART_INF_F;
           }
           if (!sweepB) {
-            float c0 = -CUDART_INF_F, c1 = -CUDART_INF_F, c2 = -CUDART_INF_F, c3 = -CUDART_INF_F;
+            float c0 = -CUDART_INF_F, c1 = -CUDART_INF_F;
 #pragma unroll
-            for (int q = 0; q < 32; q += 4) {
-              c0 = fmaxf(c0, x[q]); c1 = fmaxf(c1, x[q + 1]); c2 = fmaxf(c2, x[q + 2]); c3 = fmaxf(c3, x[q + 3]);
-            }
-            const float mn = fmaxf(tmax, fmaxf(fmaxf(c0, c1), fmaxf(c2, c3)));
+            for (int q = 0; q < 32; q += 4) { c0 = max3(c0, x[q], x[q + 1]); c1 = max3(c1, x[q + 2], x[q + 3]); }
+            const float mn = fmaxf(tmax, fmaxf(c0, c1));          // maximum of the raw values (the scale is positive)
             if (mn > -CUDART_INF_F) {
+              const float nm = -(mn * prm.scale_log2);
               float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
               for (int q = 0; q < 32; q += 4) {
                 float y0, y1, y2, y3;
-                add2(y0, y1, x[q], x[q + 1], -mn, -mn);
-                add2(y2, y3, x[q + 2], x[q + 3], -mn, -mn);
+                fma2(y0, y1, x[q], x[q + 1], prm.scale_log2, prm.scale_log2, nm, nm);
+                fma2(y2, y3, x[q + 2], x[q + 3], prm.scale_log2, prm.scale_log2, nm, nm);
                 add2(a0, a1, a0, a1, ex2(y0), ex2(y1));
                 add2(a2, a3, a2, a3, ex2(y2), ex2(y3));
               }
-              tsum = tsum * ex2(tmax - mn) + ((a0 + a1) + (a2 + a3));     // tmax = -inf gives a factor 0
+              tsum = tsum * ex2((tmax - mn) * prm.scale_log2) + ((a0 + a1) + (a2 + a3));     // tmax = -inf gives a factor 0
               tmax = mn;
             }
           } else if (Prow) {
@@ -297,7 +301,7 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             uint32_t word = 0u;
 #pragma unroll
             for (int q = 0; q < 32; ++q) {
-              const float p = ex2(x[q] - m) * inv_l;       // x = -inf beyond the causal limit gives 0
+              const float p = ex2(fmaf(x[q], prm.scale_log2, -m)) * inv_l;    // -inf beyond the causal limit gives 0
               x[q] = p;
               word |= (p >= prm.pstar ? 1u : 0u) << q;
             }
@@ -309,20 +313,21 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 if (j0 + q < L) Prow[j0 + q] = x[q];
             }
           } else {
-            // only the decision p >= p* is needed.  p = 2^(x - m) / l, so an entry whose x - m lies more than
-            // 2^-5 below log2(p* l) cannot reach p* (the margin is five orders of magnitude above the rounding
-            // of the fast exponential); groups of 8 columns with no candidate in the whole warp skip the
-            // special-function unit.  Candidates are evaluated exactly as in the branch above.
+            // only the decision p >= p* is needed.  p = 2^(x scale - m) / l, so an entry whose x scale - m lies
+            // more than 2^-5 below log2(p* l) cannot reach p* (the margin is five orders of magnitude above the
+            // rounding of the fast exponential and of the comparison on the raw value); groups of 8 columns with
+            // no candidate in the whole warp skip the special-function unit.  Candidates are evaluated exactly
+            // as in the branch above.
             uint32_t word = 0u;
 #pragma unroll
             for (int q8 = 0; q8 < 32; q8 += 8) {
               bool any = false;
 #pragma unroll
-              for (int u = 0; u < 8; ++u) any |= (x[q8 + u] - m) > thr_lo;
+              for (int u = 0; u < 8; ++u) any |= x[q8 + u] > thr_raw;
               if (__any_sync(0xFFFFFFFFu, any)) {
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
-                  const float p = ex2(x[q8 + u] - m) * inv_l;
+                  const float p = ex2(fmaf(x[q8 + u], prm.scale_log2, -m)) * inv_l;
                   word |= (p >= prm.pstar ? 1u : 0u) << (q8 + u);
                 }
               }
@@ -335,8 +340,9 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         if (lane == 0) mbar_arrive(bSEmpty + 8 * buf);
         if (!sweepB) {
           if (tmax > -CUDART_INF_F) {
-            const float mn = fmaxf(m, tmax);
-            l = l * ex2(m - mn) + tsum * ex2(tmax - mn);
+            const float tm = tmax * prm.scale_log2;               // the tile's maximum in the scaled domain
+            const float mn = fmaxf(m, tm);
+            l = l * ex2(m - mn) + tsum * ex2(tm - mn);
             m = mn;
           }
         } else if (row_valid) {
