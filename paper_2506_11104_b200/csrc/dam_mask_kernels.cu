@@ -409,7 +409,7 @@ __device__ uint32_t block_excl_scan(uint32_t x, uint32_t* total, uint32_t* sm /*
   if (lane == 31) sm[warp] = inc;
   __syncthreads();
   if (warp == 0) {
-    uint32_t s = sm[lane];
+    uint32_t s = lane < (int)(blockDim.x >> 5) ? sm[lane] : 0u;      // blocks of fewer than 32 warps
     uint32_t si = s;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
