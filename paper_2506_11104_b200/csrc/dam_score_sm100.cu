@@ -351,9 +351,13 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       }
       if (!ok) break;
       ++nitem;
-      // dump: zeros above the diagonal for the tiles this item does not visit
-      if (Prow && row_valid && G == 0)
-        for (int j = (it.qb + 1) * DAM_TILE; j < L; ++j) Prow[j] = 0.f;
+      // zeros above the diagonal for the tiles this item does not visit: the true-mask words, and the map itself
+      // when it is dumped
+      if (row_valid && G == 0) {
+        for (int kb = it.qb + 1; kb * 4 < W; ++kb) *reinterpret_cast<uint4*>(Mrow + kb * 4) = make_uint4(0u, 0u, 0u, 0u);
+        if (Prow)
+          for (int j = (it.qb + 1) * DAM_TILE; j < L; ++j) Prow[j] = 0.f;
+      }
     }
   }
 
@@ -385,11 +389,6 @@ cudaError_t dam_launch_scores_sm100(const void* Q, const void* K, const dam_shap
   if (!dam_make_tmap_bf16(&tq, Q, 128, s->num_q_heads, s->total_tokens, s->q_stride_tok, s->q_stride_head) ||
       !dam_make_tmap_bf16(&tk, K, 128, s->num_kv_heads, s->total_tokens, s->k_stride_tok, s->k_stride_head))
     return cudaErrorInvalidValue;
-  // the kernel writes only the tiles on or below the diagonal: everything else of the true mask is zero
-  if (c.true_bytes) {
-    cudaError_t e = cudaMemsetAsync(c.blob + c.off_true, 0, c.true_bytes, st);
-    if (e != cudaSuccess) return e;
-  }
   ScoreParams p;
   p.blob = c.blob; p.dump = dump;
   p.status = reinterpret_cast<uint32_t*>(c.blob) + 1;
