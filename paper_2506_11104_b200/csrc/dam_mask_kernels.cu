@@ -762,9 +762,8 @@ cudaError_t dam_launch_capture_average(const float* A, const int32_t* C, int Lma
 // The counters of the rule kernels start at zero: counts + prefix + tile popcounts, row counts, histogram,
 // cursors.  Enqueued before the kernel that produces the true mask, so that the rule kernels follow it directly.
 cudaError_t dam_launch_rule_prepare(const DamBuildCtx& c, cudaStream_t st) {
-  cudaError_t e;
-  if ((e = cudaMemsetAsync(c.scratch + c.off_cnt, 0, c.off_cnt_end - c.off_cnt, st)) != cudaSuccess) return e;
-  return cudaMemsetAsync(c.scratch + c.off_hist, 0, 2ull * DAM_HIST * 4, st);
+  // the sections are contiguous (counts | row counts | histogram | cursors): one fill
+  return cudaMemsetAsync(c.scratch + c.off_cnt, 0, c.off_cursor + 4ull * DAM_HIST - c.off_cnt, st);
 }
 
 cudaError_t dam_launch_rule(const DamBuildCtx& c, cudaStream_t st) {
