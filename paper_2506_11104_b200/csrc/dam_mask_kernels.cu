@@ -37,6 +37,7 @@ __device__ __forceinline__ const DamSeq* blob_seqs(const unsigned char* blob, co
 // ---------------------------------------------------------------------------------------------
 __global__ void init_blob_kernel(unsigned char* blob, DamHeader hdr, const int32_t* __restrict__ cu,
                                  int pcl_max, int Hq, int all_ones_causal /* -1: DAM mask */) {
+  asm volatile("griddepcontrol.launch_dependents;");     // a kernel chained behind this one may start its prologue
   DamHeader* H = reinterpret_cast<DamHeader*>(blob);
   DamSeq* seqs = reinterpret_cast<DamSeq*>(blob + hdr.off_seq);
   int32_t* qbseq = reinterpret_cast<int32_t*>(blob + hdr.off_qbseq);
@@ -762,8 +763,9 @@ cudaError_t dam_launch_capture_average(const float* A, const int32_t* C, int Lma
 // The counters of the rule kernels start at zero: counts + prefix + tile popcounts, row counts, histogram,
 // cursors.  Enqueued before the kernel that produces the true mask, so that the rule kernels follow it directly.
 cudaError_t dam_launch_rule_prepare(const DamBuildCtx& c, cudaStream_t st) {
-  // the sections are contiguous (counts | row counts | histogram | cursors): one fill
-  return cudaMemsetAsync(c.scratch + c.off_cnt, 0, c.off_cursor + 4ull * DAM_HIST - c.off_cnt, st);
+  // the sections are contiguous (status block and work counter of the scoring kernel | counts | row counts |
+  // histogram | cursors): one fill
+  return cudaMemsetAsync(c.scratch, 0, c.off_cursor + 4ull * DAM_HIST, st);
 }
 
 cudaError_t dam_launch_rule(const DamBuildCtx& c, cudaStream_t st) {

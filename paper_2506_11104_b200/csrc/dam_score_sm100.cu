@@ -128,6 +128,8 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  // everything above is independent of the kernel before this one; the blob it initialises is read from here on
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   if (warp == 0) {
     if (lane == 0) {
@@ -393,15 +395,20 @@ cudaError_t dam_launch_scores_sm100(const void* Q, const void* K, const dam_shap
   p.blob = c.blob; p.dump = dump;
   p.status = reinterpret_cast<uint32_t*>(c.blob) + 1;
   p.work_counter = reinterpret_cast<uint32_t*>(c.scratch) + 2;
-  {
-    cudaError_t e = cudaMemsetAsync(c.scratch, 0, 256, st);
-    if (e != cudaSuccess) return e;
-  }
+  // (the status block and the work counter at the start of the scratch buffer were cleared together with the
+  // rule counters, before the blob was initialised: this kernel follows that one directly)
   p.num_seqs = c.num_seqs; p.Hq = c.Hq; p.group = c.Hq / c.Hkv; p.max_nL = c.max_nL;
   p.scale_log2 = c.scale * 1.4426950408889634f;
   p.pstar = c.pstar;
   const int items = c.max_nL * c.num_seqs * c.Hq;
   const int grid = items < sm_count ? items : sm_count;
-  score_sm100_kernel<<<grid, kThreads, kSmemBytes, st>>>(tq, tk, p);
-  return cudaGetLastError();
+  // launched as a programmatic dependent of the kernel that initialises the blob: its launch latency and its
+  // prologue (barriers, TMEM, descriptors) hide under that kernel; it waits before it reads the blob
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, score_sm100_kernel, tq, tk, p);
 }
