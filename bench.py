@@ -327,6 +327,13 @@ def main():
     flops_tile = 4.0 * TILE * TILE * w0.head_dim
     # executed tiles (what the tensor cores ran) and mask tiles (128 x 128 tiles of the masks with an active
     # cell; the two differ when matched columns are served by gathered-column tiles)
+    # element-level density of one layer's masks (host arithmetic on the pattern bits: the paper's O(s L) figure)
+    elem = None
+    if rank == 0:
+        mbh = B.MaskBlob(mask)
+        nnz = sum(mbh.active_elements(b, h) for b in range(len(shape.lengths)) for h in range(w0.num_q_heads))
+        causal_elems = sum(S * (S + 1) // 2 for S in shape.lengths) * w0.num_q_heads
+        elem = {"layer": int(l), "density": round(nnz / causal_elems, 5), "flops": 4.0 * w0.head_dim * nnz}
     step_tiles = [per_layer_stats[(args.warmup + i) % n_layers]["tiles"] for i in range(args.steps)]
     step_mask_tiles = [per_layer_stats[(args.warmup + i) % n_layers]["mask_tiles"] for i in range(args.steps)]
     total_flops = flops_tile * sum(step_mask_tiles)
@@ -356,6 +363,10 @@ def main():
                                     round(max(step_mask_tiles) / causal_tiles, 4)],
            "executed_tile_density": round(sum(step_tiles) / len(step_tiles) / causal_tiles, 4),
            "executed_tflops": round(flops_tile * sum(step_tiles) / (total_ms_max * 1e-3) / 1e12 * world, 3),
+           "element_active": (None if elem is None else
+                              {"layer": elem["layer"], "element_density": elem["density"],
+                               "tflops": round(elem["flops"] / (total_ms_max / args.steps * 1e-3) / 1e12, 3),
+                               "flops": "4*d per active cell of the masks (one layer, at the mean layer time)"}),
            "roofline": roof, "clocks": clocks, "gpu_launches": (9 if not args.no_gather else 8) * args.steps}
 
     if rank == 0 and not args.no_dense:

@@ -398,6 +398,23 @@ class MaskBlob:
         w = np.frombuffer(self.raw, dtype="<u4", count=L * W, offset=off).reshape(L, W)
         return _unpack_bits(w, L)
 
+    def active_elements(self, seq: int, head: int) -> int:
+        """Number of active cells of the S x S mask of (seq, head): the true mask inside the window, and below
+        it, per row, the matched columns plus the matched diagonals minus the cells that are both (rows
+        L .. 2L-2 only: a correlation of the two bit sets)."""
+        s = self.seqs[seq]
+        S, L, W = int(s["S"]), int(s["L"]), int(s["W"])
+        if L == 0:
+            return 0
+        off = int(self.hdr["off_true"]) + 4 * (int(s["true_off"]) + head * L * W)
+        words = np.frombuffer(self.raw, dtype="<u4", count=L * W, offset=off)
+        n = int(np.unpackbits(words.view(np.uint8)).sum())
+        if S > L:
+            D, _, V = self.pattern_bits(seq, head)
+            both = np.convolve(V.astype(np.int64), D.astype(np.int64))     # index i = column + diagonal
+            n += (S - L) * (int(D.sum()) + int(V.sum())) - int(both[L: min(S, 2 * L - 1)].sum())
+        return n
+
     def row_tiles(self, seq: int, head: int, qb: int):
         """(kv tile indices, kinds) of query block qb of (seq, head)."""
         row = head * int(self.hdr["total_qblocks"]) + int(self.seqs[seq]["first_qblock"]) + qb

@@ -305,3 +305,19 @@ def test_other_amplifications_bit_exact_from_scores(transform, lam, tau):
     assert active > 0
     H.check_blob_against_oracle(blob, shape, masks)
     H.check_blob_against_oracle(blob2, shape, masks)
+
+
+def test_active_element_count_matches_the_extended_mask():
+    """MaskBlob.active_elements (host arithmetic on the pattern bits, used for the element-level density of the
+    bench line) against the sum of the oracle's extended-mask rows."""
+    w = synth.small_case(0, 4, 2, 64, 96, seed=50, dtype=torch.bfloat16, lengths=[400, 150, 60])
+    shape = B.make_shape(w.cu_seqlens, 4, 2, 64, w.Q.dtype, DEV)
+    rule = B.make_rule(96, w.tau, w.mu)
+    n = sum(4 * min(S, 96) ** 2 for S in shape.lengths)
+    dump = torch.zeros(n, dtype=torch.float32, device=DEV)
+    blob, _ = B.dam_build_masks(w.Q.to(DEV), w.K.to(DEV), shape, rule, scores_dump=dump)
+    masks = H.oracle_masks_from_dump(w, dump.cpu().numpy())
+    mb = B.MaskBlob(blob)
+    for b, S in enumerate(shape.lengths):
+        for h in range(4):
+            assert mb.active_elements(b, h) == int(masks[b][h].rows(list(range(S))).sum())
