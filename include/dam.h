@@ -303,12 +303,16 @@ dam_status_t dam_poll_status(const void* mask_or_scratch, void* stream);
 dam_status_t dam_selftest_bounded_wait(void* scratch, size_t scratch_bytes, uint32_t limit_us, void* stream);
 
 /*
- * Both stages from HOST buffers: copies Q, K, V (HOST, pinned recommended, layouts from `shape`
- * with dense strides) into the device workspace, runs dam_build_masks and dam_sparse_attention,
- * and copies O and LSE back to HOST; everything on `stream`, which is synchronised before
- * returning. workspace: DEVICE, >= *workspace_bytes as returned when called with workspace == NULL
- * (in that case only the size is computed). The end-to-end figure of the benchmark is measured
- * through this call.
+ * Both stages from HOST buffers (pinned recommended, layouts from `shape` with dense strides): copies
+ * Q, K, V into the device workspace, runs dam_build_masks and the attention, and copies O and LSE back to
+ * HOST. The work is pipelined over chunks of whole query-block pairs in token order: the pattern-capture
+ * windows go up first and the masks are built from them; the attention of a chunk (causal: it needs the keys
+ * up to the chunk's end only) runs under the upload of the next chunk, and its rows of O and LSE are copied
+ * back under both, on two internal streams besides `stream`. All three are synchronised before returning, so
+ * the host buffers are complete (and reusable) on return; results are identical to the two device calls.
+ * Calls of this entry point are serialised inside the library (one at a time per process).
+ * workspace: DEVICE, >= *workspace_bytes as returned when called with workspace == NULL (in that case
+ * only the size is computed). The end-to-end figure of the benchmark is measured through this call.
  */
 dam_status_t dam_prefill_host(const void* Q_host, const void* K_host, const void* V_host,
                               const dam_shape_t* shape, const dam_rule_t* rule, int32_t causal,

@@ -3,6 +3,7 @@
 #include <math.h>
 #include <string.h>
 
+#include <mutex>
 #include <vector>
 
 #include "dam_internal.cuh"
@@ -325,7 +326,9 @@ static dam_status_t sparse_attention_impl(const void* Q, const void* K, const vo
                                           const dam_shape_t* shape, int32_t causal, int32_t gqa_group,
                                           float softmax_scale, void* O, float* lse, const int32_t* ranges_host,
                                           const int32_t* ranges_dev, void* scratch, size_t scratch_bytes,
-                                          void* stream) {
+                                          void* stream, bool continuation = false) {
+  // continuation: a further row range of the same layer against the same scratch buffer: the status word is
+  // kept, and the gathered-column tiles the first call built are used again
   dam_status_t st;
   if ((st = check_shape(shape)) != DAM_OK) return st;
   if (!Q || !K || !V || !mask || !O || !lse || !scratch) return DAM_ERR_INVALID_ARGUMENT;
@@ -347,11 +350,14 @@ static dam_status_t sparse_attention_impl(const void* Q, const void* K, const vo
   if (scratch_bytes < 256) return DAM_ERR_BUFFER_TOO_SMALL;
   const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)shape->head_dim);
   cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
-  // status word and work counter start at zero
-  if (cudaMemsetAsync(scratch, 0, 256, cs) != cudaSuccess) return DAM_ERR_CUDA;
+  // status word and work counter start at zero (a continuation clears the work counter only)
+  if (cudaMemsetAsync(reinterpret_cast<unsigned char*>(scratch) + (continuation ? 8 : 0), 0, continuation ? 248 : 256, cs) !=
+      cudaSuccess)
+    return DAM_ERR_CUDA;
   cudaError_t e = cudaErrorNotSupported;
   if (sm100_shape(shape))
-    e = dam_launch_attn_sm100(Q, K, V, mask, shape, causal != 0, scale, O, lse, scratch, scratch_bytes, ranges_dev, cs);
+    e = dam_launch_attn_sm100(Q, K, V, mask, shape, causal != 0, scale, O, lse, scratch, scratch_bytes, ranges_dev,
+                              !continuation, cs);
   if (e == cudaErrorNotSupported)
     e = dam_launch_attn_ref(Q, K, V, mask, shape, causal != 0, scale, O, lse, scratch, ranges_dev, cs);
   return e == cudaSuccess ? DAM_OK : DAM_ERR_CUDA;
@@ -442,6 +448,42 @@ dam_status_t dam_selftest_bounded_wait(void* scratch, size_t scratch_bytes, uint
   return dam_launch_bounded_wait_selftest(scratch, 1000ull * limit_us, cs) == cudaSuccess ? DAM_OK : DAM_ERR_CUDA;
 }
 
+// Streams and events of the host-buffer entry point (created on first use, one set per device).
+namespace {
+constexpr int kMaxChunks = 32;
+struct HostPipe {
+  bool ready = false;
+  cudaStream_t h2d = nullptr, d2h = nullptr;
+  cudaEvent_t start = nullptr, window = nullptr, out = nullptr, up[kMaxChunks] = {}, done[kMaxChunks] = {};
+};
+std::mutex g_pipe_mutex;
+HostPipe g_pipes[64];
+
+HostPipe* host_pipe() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  HostPipe& p = g_pipes[dev];
+  if (p.ready) return &p;
+  bool ok = cudaStreamCreateWithFlags(&p.h2d, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaStreamCreateWithFlags(&p.d2h, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming) == cudaSuccess &&
+            cudaEventCreateWithFlags(&p.window, cudaEventDisableTiming) == cudaSuccess &&
+            cudaEventCreateWithFlags(&p.out, cudaEventDisableTiming) == cudaSuccess;
+  for (int c = 0; ok && c < kMaxChunks; ++c)
+    ok = cudaEventCreateWithFlags(&p.up[c], cudaEventDisableTiming) == cudaSuccess &&
+         cudaEventCreateWithFlags(&p.done[c], cudaEventDisableTiming) == cudaSuccess;
+  if (!ok) return nullptr;
+  p.ready = true;
+  return &p;
+}
+}  // namespace
+
+// The copies and the kernels are pipelined over chunks of whole query-block pairs, in token order.  First the
+// pattern-capture windows of all sequences go up (rows [0, L) of Q, K, V: all the mask construction and the
+// gathered-column tiles read); while the masks are built the first chunk follows.  The attention of chunk c
+// (dam_sparse_attention_rows on its row ranges; causal, so it needs the keys up to the chunk's end only) runs as
+// soon as the chunk is on the device, under the upload of chunk c + 1, and its rows of O and LSE go back to the
+// host on a third stream under both.  Uploads use one PCIe direction and downloads the other.
 dam_status_t dam_prefill_host(const void* Qh, const void* Kh, const void* Vh, const dam_shape_t* shape,
                               const dam_rule_t* rule, int32_t causal, void* Oh, float* lse_h, void* workspace,
                               size_t* workspace_bytes, void* stream) {
@@ -451,6 +493,7 @@ dam_status_t dam_prefill_host(const void* Qh, const void* Kh, const void* Vh, co
   if (!workspace_bytes) return DAM_ERR_INVALID_ARGUMENT;
   const size_t es = shape->dtype == DAM_BF16 ? 2 : 4;
   const int64_t T = shape->total_tokens, Hq = shape->num_q_heads, Hkv = shape->num_kv_heads, d = shape->head_dim;
+  const int nb = shape->num_seqs;
   // dense strides only
   if (shape->q_stride_head != d || shape->q_stride_tok != Hq * d || shape->k_stride_head != d ||
       shape->k_stride_tok != Hkv * d || shape->v_stride_head != d || shape->v_stride_tok != Hkv * d ||
@@ -460,29 +503,110 @@ dam_status_t dam_prefill_host(const void* Qh, const void* Kh, const void* Vh, co
   compute_layout(shape, rule->pcl_max, 1, gather_enabled(shape, rule), &y);
   const size_t qb = dam_align((size_t)T * Hq * d * es, 256), kb = dam_align((size_t)T * Hkv * d * es, 256);
   const size_t lb = dam_align((size_t)Hq * T * 4, 256);
+  const size_t rb = dam_align((size_t)kMaxChunks * 2 * (size_t)(nb > 0 ? nb : 1) * sizeof(int32_t), 256);
   size_t off_q = 0, off_k = off_q + qb, off_v = off_k + kb, off_o = off_v + kb, off_l = off_o + qb;
   size_t off_m = off_l + lb, off_bs = off_m + y.mask_bytes, off_as = off_bs + y.build_scratch_bytes;
-  size_t total = off_as + y.attn_scratch_bytes;
+  size_t off_r = off_as + dam_align(y.attn_scratch_bytes, 256);
+  size_t total = off_r + rb;
   if (!workspace) { *workspace_bytes = total; return DAM_OK; }
   if (*workspace_bytes < total) return DAM_ERR_BUFFER_TOO_SMALL;
   if (!Qh || !Kh || !Vh || !Oh || !lse_h || !aligned(workspace, 256)) return DAM_ERR_INVALID_ARGUMENT;
   cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
   unsigned char* w = reinterpret_cast<unsigned char*>(workspace);
-  if (cudaMemcpyAsync(w + off_q, Qh, (size_t)T * Hq * d * es, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
-      cudaMemcpyAsync(w + off_k, Kh, (size_t)T * Hkv * d * es, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
-      cudaMemcpyAsync(w + off_v, Vh, (size_t)T * Hkv * d * es, cudaMemcpyHostToDevice, cs) != cudaSuccess)
-    return DAM_ERR_CUDA;
+  if (T == 0) return cudaStreamSynchronize(cs) == cudaSuccess ? DAM_OK : DAM_ERR_CUDA;
+
+  // ---- chunk plan: pieces of whole query-block pairs of one sequence, grouped in token order
+  const int* cu = shape->cu_seqlens_host;
+  int64_t chunk_rows = (T / 8 + 255) / 256 * 256;          // eight chunks: more gave nothing on PCIe 5 x16
+  if (chunk_rows < 2048) chunk_rows = 2048;
+  struct Chunk { int64_t t0, t1; };
+  std::vector<Chunk> chunks;
+  std::vector<int32_t> ranges;                 // [chunk][2 * seq]
+  for (;;) {
+    chunks.clear(); ranges.clear();
+    for (int b = 0; b < nb; ++b) {
+      const int S = cu[b + 1] - cu[b];
+      for (int64_t r0 = 0; r0 < S; r0 += chunk_rows) {
+        const int64_t r1 = r0 + chunk_rows < S ? r0 + chunk_rows : S;
+        const bool fresh = chunks.empty() || (chunks.back().t1 - chunks.back().t0) + (r1 - r0) > chunk_rows;
+        if (fresh) {
+          chunks.push_back({cu[b] + r0, cu[b] + r0});
+          ranges.resize(ranges.size() + 2 * (size_t)nb, 0);
+        }
+        int32_t* rg = ranges.data() + (chunks.size() - 1) * 2 * (size_t)nb;
+        if (rg[2 * b + 1] == 0) rg[2 * b] = (int32_t)r0;
+        rg[2 * b + 1] = (int32_t)r1;
+        chunks.back().t1 = cu[b] + r1;
+      }
+    }
+    if ((int)chunks.size() <= kMaxChunks) break;
+    chunk_rows *= 2;
+  }
+  const int nc = (int)chunks.size();
+
+  std::lock_guard<std::mutex> lock(g_pipe_mutex);
+  HostPipe* pp = host_pipe();
+  if (!pp) return DAM_ERR_CUDA;
+  HostPipe& P = *pp;
+  const char* Qc = reinterpret_cast<const char*>(Qh);
+  const char* Kc = reinterpret_cast<const char*>(Kh);
+  const char* Vc = reinterpret_cast<const char*>(Vh);
+  const size_t qrow = (size_t)Hq * d * es, krow = (size_t)Hkv * d * es;
+  bool ok = true;
+  auto up = [&](int64_t a, int64_t e, bool with_qk) {   // tokens [a, e): V always, Q and K unless already up
+    if (e <= a || !ok) return;
+    if (with_qk)
+      ok = cudaMemcpyAsync(w + off_q + a * qrow, Qc + a * qrow, (size_t)(e - a) * qrow, cudaMemcpyHostToDevice, P.h2d) == cudaSuccess &&
+           cudaMemcpyAsync(w + off_k + a * krow, Kc + a * krow, (size_t)(e - a) * krow, cudaMemcpyHostToDevice, P.h2d) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(w + off_v + a * krow, Vc + a * krow, (size_t)(e - a) * krow, cudaMemcpyHostToDevice, P.h2d) == cudaSuccess;
+  };
+  // the workspace may still be in use by earlier work of the caller's stream
+  ok = cudaEventRecord(P.start, cs) == cudaSuccess && cudaStreamWaitEvent(P.h2d, P.start, 0) == cudaSuccess &&
+       cudaStreamWaitEvent(P.d2h, P.start, 0) == cudaSuccess;
+  // windows first, with the row ranges of all chunks
+  ok = ok && cudaMemcpyAsync(w + off_r, ranges.data(), ranges.size() * sizeof(int32_t), cudaMemcpyHostToDevice, P.h2d) == cudaSuccess;
+  for (int b = 0; b < nb && ok; ++b) {
+    const int S = cu[b + 1] - cu[b];
+    const int L = S < rule->pcl_max ? S : rule->pcl_max;
+    up(cu[b], cu[b] + L, true);
+  }
+  ok = ok && cudaEventRecord(P.window, P.h2d) == cudaSuccess && cudaStreamWaitEvent(cs, P.window, 0) == cudaSuccess;
+  if (!ok) return DAM_ERR_CUDA;
   st = dam_build_masks(w + off_q, w + off_k, shape, rule, w + off_m, y.mask_bytes, w + off_bs, y.build_scratch_bytes,
                        nullptr, stream);
+  if (st != DAM_OK) { cudaStreamSynchronize(P.h2d); return st; }
+  int b_lo = 0;
+  for (int c = 0; c < nc && ok; ++c) {
+    const int64_t t0 = chunks[c].t0, t1 = chunks[c].t1;
+    // the rest of the chunk: per sequence, what lies below its window
+    while (b_lo + 1 < nb && cu[b_lo + 1] <= t0) ++b_lo;
+    for (int b = b_lo; b < nb && cu[b] < t1; ++b) {
+      const int S = cu[b + 1] - cu[b];
+      const int L = S < rule->pcl_max ? S : rule->pcl_max;
+      const int64_t a = t0 > cu[b] + L ? t0 : cu[b] + L, e = t1 < cu[b + 1] ? t1 : cu[b + 1];
+      up(a, e, true);
+    }
+    ok = ok && cudaEventRecord(P.up[c], P.h2d) == cudaSuccess && cudaStreamWaitEvent(cs, P.up[c], 0) == cudaSuccess;
+    if (!ok) break;
+    const int32_t* rg = ranges.data() + (size_t)c * 2 * nb;
+    st = sparse_attention_impl(w + off_q, w + off_k, w + off_v, w + off_m, shape, causal,
+                               shape->num_q_heads / shape->num_kv_heads, rule->softmax_scale, w + off_o,
+                               reinterpret_cast<float*>(w + off_l), rg,
+                               reinterpret_cast<const int32_t*>(w + off_r) + (size_t)c * 2 * nb, w + off_as,
+                               y.attn_scratch_bytes, stream, c > 0);
+    if (st != DAM_OK) break;
+    ok = cudaEventRecord(P.done[c], cs) == cudaSuccess && cudaStreamWaitEvent(P.d2h, P.done[c], 0) == cudaSuccess &&
+         cudaMemcpyAsync(reinterpret_cast<char*>(Oh) + t0 * qrow, w + off_o + t0 * qrow, (size_t)(t1 - t0) * qrow,
+                         cudaMemcpyDeviceToHost, P.d2h) == cudaSuccess &&
+         cudaMemcpy2DAsync(lse_h + t0, (size_t)T * 4, reinterpret_cast<float*>(w + off_l) + t0, (size_t)T * 4,
+                           (size_t)(t1 - t0) * 4, (size_t)Hq, cudaMemcpyDeviceToHost, P.d2h) == cudaSuccess;
+  }
+  // everything this call queued has finished before it returns, also on an error
+  const bool s1 = cudaStreamSynchronize(P.h2d) == cudaSuccess;
+  const bool s2 = cudaStreamSynchronize(cs) == cudaSuccess;
+  const bool s3 = cudaStreamSynchronize(P.d2h) == cudaSuccess;
   if (st != DAM_OK) return st;
-  st = dam_sparse_attention(w + off_q, w + off_k, w + off_v, w + off_m, shape, causal,
-                            shape->num_q_heads / shape->num_kv_heads, rule->softmax_scale, w + off_o,
-                            reinterpret_cast<float*>(w + off_l), w + off_as, y.attn_scratch_bytes, stream);
-  if (st != DAM_OK) return st;
-  if (cudaMemcpyAsync(Oh, w + off_o, (size_t)T * Hq * d * es, cudaMemcpyDeviceToHost, cs) != cudaSuccess ||
-      cudaMemcpyAsync(lse_h, w + off_l, (size_t)Hq * T * 4, cudaMemcpyDeviceToHost, cs) != cudaSuccess)
-    return DAM_ERR_CUDA;
-  if (cudaStreamSynchronize(cs) != cudaSuccess) return DAM_ERR_CUDA;
+  if (!ok || !s1 || !s2 || !s3) return DAM_ERR_CUDA;
   st = dam_poll_status(w + off_m, stream);
   if (st != DAM_OK) return st;
   return dam_poll_status(w + off_as, stream);

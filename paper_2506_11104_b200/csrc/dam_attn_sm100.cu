@@ -802,7 +802,7 @@ cudaError_t dam_launch_bounded_wait_selftest(void* scratch, unsigned long long l
 
 cudaError_t dam_launch_attn_sm100(const void* Q, const void* K, const void* V, const void* blob,
                                   const dam_shape_t* s, int causal, float scale, void* O, float* lse, void* scratch,
-                                  size_t scratch_bytes, const int32_t* ranges, cudaStream_t st) {
+                                  size_t scratch_bytes, const int32_t* ranges, bool run_gather, cudaStream_t st) {
   if (s->dtype != DAM_BF16 || s->head_dim != 128) return cudaErrorNotSupported;
   if (s->total_tokens == 0) return cudaSuccess;
   static int sm_count = 0, smem_optin = 0;
@@ -827,7 +827,7 @@ cudaError_t dam_launch_attn_sm100(const void* Q, const void* K, const void* V, c
   if (!dam_make_tmap_bf16(&tg, has_g ? reinterpret_cast<const unsigned char*>(scratch) + 256 : Q, 128, 1,
                           has_g ? (int64_t)grows : DAM_TILE, 128, 128))
     return cudaErrorInvalidValue;
-  if (has_g) {
+  if (has_g && run_gather) {
     gather_columns_kernel<<<sm_count * 4, 128, 0, st>>>(
         reinterpret_cast<const unsigned char*>(blob), reinterpret_cast<const __nv_bfloat16*>(K),
         reinterpret_cast<const __nv_bfloat16*>(V), s->num_q_heads, s->num_q_heads / s->num_kv_heads, s->k_stride_tok,

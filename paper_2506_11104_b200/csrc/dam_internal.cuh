@@ -224,7 +224,7 @@ cudaError_t dam_launch_attn_ref(const void* Q, const void* K, const void* V, con
 // tensor-core paths (bf16, d = 128); return cudaErrorNotSupported when the shape does not qualify
 cudaError_t dam_launch_attn_sm100(const void* Q, const void* K, const void* V, const void* blob,
                                   const dam_shape_t* shape, int causal, float scale, void* O, float* lse,
-                                  void* scratch, size_t scratch_bytes, const int32_t* ranges, cudaStream_t st);
+                                  void* scratch, size_t scratch_bytes, const int32_t* ranges, bool run_gather, cudaStream_t st);
 cudaError_t dam_launch_scores_sm100(const void* Q, const void* K, const dam_shape_t* shape, const DamBuildCtx& c,
                                     float* scores_dump, cudaStream_t st);
 

@@ -772,7 +772,7 @@ cudaError_t dam_launch_rule(const DamBuildCtx& c, cudaStream_t st) {
   cudaError_t e;
   if (c.max_nL > 0) {
     dim3 g(c.max_nL * (c.max_nL + 1) / 2, c.num_seqs * c.Hq);
-    counts_kernel<<<g, DAM_TILE, 0, st>>>(c.blob, c.scratch, c.off_cnt);
+    if ((e = launch_chained(counts_kernel, g, dim3(DAM_TILE), st, c.blob, c.scratch, c.off_cnt)) != cudaSuccess) return e;
     if ((e = launch_chained(match_kernel, dim3(c.num_seqs * c.Hq), dim3(256), st, c.blob, c.scratch, c.off_cnt, c.mu,
                             c.min_support)) != cudaSuccess) return e;
   }
