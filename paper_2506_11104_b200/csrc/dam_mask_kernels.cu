@@ -101,10 +101,21 @@ __global__ void bits_from_scores_kernel(unsigned char* blob, const float* __rest
   }
 }
 
+// Transpose of a 32 x 32 bit matrix held one row per lane: lane c returns column c (bit r = bit c of row r).
+__device__ __forceinline__ uint32_t dam_transpose32(uint32_t x, int lane) {
+#pragma unroll
+  for (int j = 16; j >= 1; j >>= 1) {
+    const uint32_t m = j == 16 ? 0x0000FFFFu : j == 8 ? 0x00FF00FFu : j == 4 ? 0x0F0F0F0Fu : j == 2 ? 0x33333333u : 0x55555555u;
+    const uint32_t y = __shfl_xor_sync(0xFFFFFFFFu, x, j);
+    x = (lane & j) ? ((x & ~m) | ((y >> j) & m)) : ((x & m) | ((y & m) << j));
+  }
+  return x;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Counts: one block per 128 x 128 tile (qb, kb <= qb) of the window.  Thread t owns row qb*128+t
-// and its 128 bits.  Column counts (128), diagonal counts (255) and the tile's popcount are
-// accumulated in shared memory and flushed with integer atomics (order-independent).
+// and its 128 bits.  Column counts (128), diagonal counts (255) and the tile's popcount are made per warp
+// with bit-matrix transposes, summed in shared memory and flushed with integer atomics (order-independent).
 // ---------------------------------------------------------------------------------------------
 __global__ void counts_kernel(const unsigned char* blob, unsigned char* scratch, uint64_t off_cnt) {
   dam_chain_prologue();
@@ -130,7 +141,7 @@ __global__ void counts_kernel(const unsigned char* blob, unsigned char* scratch,
   __shared__ int sV[DAM_TILE];
   __shared__ int sD[2 * DAM_TILE];
   __shared__ int sPop;
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int i = qb * DAM_TILE + tid;
   uint4 bits = make_uint4(0, 0, 0, 0);
   if (i < sq.L) bits = __ldg(reinterpret_cast<const uint4*>(M + (size_t)i * sq.W + kb * 4));
@@ -139,21 +150,37 @@ __global__ void counts_kernel(const unsigned char* blob, unsigned char* scratch,
   sV[tid] = 0; sD[tid] = 0; sD[tid + DAM_TILE] = 0;
   if (tid == 0) sPop = 0;
   __syncthreads();
-  if (nz) {
-    uint32_t w[4] = {bits.x, bits.y, bits.z, bits.w};
+  // The patterns being counted are whole columns and whole diagonals, i.e. the same counter for every row: a
+  // counter update per set bit would serialise.  Instead every warp transposes its 32 x 32 bit blocks with
+  // shuffles, so that lane c holds column c of the block and one population count gives the column's count.
+  // Diagonals are columns of the rows reversed and shifted by the row index: bit 127 + row - c of a 160-bit row.
+  if (__any_sync(0xFFFFFFFFu, nz)) {
+    const uint32_t w[4] = {bits.x, bits.y, bits.z, bits.w};
     int pop = 0;
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      uint32_t x = w[q];
-      pop += __popc(x);
-      while (x) {
-        int c = q * 32 + (__ffs(x) - 1);
-        x &= x - 1;
-        atomicAdd(&sV[c], 1);
-        atomicAdd(&sD[tid - c + (DAM_TILE - 1)], 1);
+      pop += __popc(w[q]);
+      if (__any_sync(0xFFFFFFFFu, w[q] != 0u)) {
+        const int n = __popc(dam_transpose32(w[q], lane));
+        if (n) atomicAdd(&sV[q * 32 + lane], n);
       }
     }
-    atomicAdd(&sPop, pop);
+    const uint32_t rev[4] = {__brev(w[3]), __brev(w[2]), __brev(w[1]), __brev(w[0])};   // bit 127 - c
+    uint32_t R[5];
+    R[0] = rev[0] << lane;
+#pragma unroll
+    for (int k = 1; k < 4; ++k) R[k] = __funnelshift_l(rev[k - 1], rev[k], lane);
+    R[4] = __funnelshift_l(rev[3], 0u, lane);
+#pragma unroll
+    for (int k = 0; k < 5; ++k) {
+      if (__any_sync(0xFFFFFFFFu, R[k] != 0u)) {
+        const int n = __popc(dam_transpose32(R[k], lane));
+        if (n) atomicAdd(&sD[warp * 32 + k * 32 + lane], n);       // index row_in_tile - c + 127
+      }
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) pop += __shfl_xor_sync(0xFFFFFFFFu, pop, o);
+    if (lane == 0) atomicAdd(&sPop, pop);
   }
   __syncthreads();
   {
