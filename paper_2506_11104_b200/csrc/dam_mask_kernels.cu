@@ -462,32 +462,62 @@ __global__ void scan_kernel(unsigned char* blob, unsigned char* scratch, uint64_
   const uint32_t* rowcnt = reinterpret_cast<const uint32_t*>(scratch + off_rowcnt);
   uint32_t* tile_ptr = reinterpret_cast<uint32_t*>(blob + H->off_tile_ptr);
   const int rows = H->rows;
-  // every warp owns a contiguous segment of rows and walks it 32 rows at a time (coalesced): first the
-  // segment totals, one block-wide scan over them, then the rows again with the segment's base
+  // every thread owns a contiguous run of rows (a multiple of 4, read with 16-byte loads that are all in flight
+  // at once): run totals, one block-wide scan over them, then the rows again from registers
   {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
-    const int seg = ((rows + nw - 1) / nw + 31) & ~31;
-    const int r0 = warp * seg, r1 = min(rows, r0 + seg);
-    uint32_t local = 0;
-    for (int r = r0 + lane; r < r1; r += 32) local += rowcnt[r];
+    constexpr int kMaxPer = 32;                                  // rows per thread held in registers
+    const int per = (((rows + (int)blockDim.x - 1) / (int)blockDim.x) + 3) & ~3;
+    if (per <= kMaxPer) {
+      const int r0 = threadIdx.x * per;
+      uint4 v[kMaxPer / 4];
+      uint32_t local = 0;
 #pragma unroll
-    for (int o = 16; o; o >>= 1) local += __shfl_xor_sync(0xFFFFFFFFu, local, o);
-    __shared__ uint32_t seg_base[32];
-    uint32_t e = block_excl_scan(lane == 0 ? local : 0u, &tot, sm);
-    if (lane == 0) seg_base[warp] = e;
-    __syncthreads();
-    uint32_t run = seg_base[warp];
-    for (int rb = r0; rb < r1; rb += 32) {
-      const int r = rb + lane;
-      const uint32_t x = r < r1 ? rowcnt[r] : 0u;
-      uint32_t inc = x;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-        if (lane >= o) inc += y;
+      for (int q = 0; q < kMaxPer / 4; ++q) {
+        v[q] = make_uint4(0u, 0u, 0u, 0u);
+        const int r = r0 + 4 * q;
+        if (4 * q < per && r < rows) {
+          if (r + 3 < rows) v[q] = *reinterpret_cast<const uint4*>(rowcnt + r);
+          else { v[q].x = rowcnt[r]; if (r + 1 < rows) v[q].y = rowcnt[r + 1]; if (r + 2 < rows) v[q].z = rowcnt[r + 2]; }
+        }
+        local += v[q].x + v[q].y + v[q].z + v[q].w;
       }
-      if (r < r1) tile_ptr[r] = run + inc - x;
-      run += __shfl_sync(0xFFFFFFFFu, inc, 31);
+      uint32_t run = block_excl_scan(local, &tot, sm);
+#pragma unroll
+      for (int q = 0; q < kMaxPer / 4; ++q) {
+        const int r = r0 + 4 * q;
+        if (4 * q < per && r < rows) {
+          const uint4 o = make_uint4(run, run + v[q].x, run + v[q].x + v[q].y, run + v[q].x + v[q].y + v[q].z);
+          if (r + 3 < rows) *reinterpret_cast<uint4*>(tile_ptr + r) = o;
+          else { tile_ptr[r] = o.x; if (r + 1 < rows) tile_ptr[r + 1] = o.y; if (r + 2 < rows) tile_ptr[r + 2] = o.z; }
+          run += v[q].x + v[q].y + v[q].z + v[q].w;
+        }
+      }
+    } else {
+      // more rows than the registers hold: every warp walks a contiguous segment 32 rows at a time, twice
+      const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+      const int seg = ((rows + nw - 1) / nw + 31) & ~31;
+      const int r0 = warp * seg, r1 = min(rows, r0 + seg);
+      uint32_t local = 0;
+      for (int r = r0 + lane; r < r1; r += 32) local += rowcnt[r];
+#pragma unroll
+      for (int o = 16; o; o >>= 1) local += __shfl_xor_sync(0xFFFFFFFFu, local, o);
+      __shared__ uint32_t seg_base[32];
+      uint32_t e = block_excl_scan(lane == 0 ? local : 0u, &tot, sm);
+      if (lane == 0) seg_base[warp] = e;
+      __syncthreads();
+      uint32_t run = seg_base[warp];
+      for (int rb = r0; rb < r1; rb += 32) {
+        const int r = rb + lane;
+        const uint32_t x = r < r1 ? rowcnt[r] : 0u;
+        uint32_t inc = x;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+          if (lane >= o) inc += y;
+        }
+        if (r < r1) tile_ptr[r] = run + inc - x;
+        run += __shfl_sync(0xFFFFFFFFu, inc, 31);
+      }
     }
     if (threadIdx.x == 0) {
       const uint32_t total = tot;
@@ -800,7 +830,7 @@ cudaError_t dam_launch_rule(const DamBuildCtx& c, cudaStream_t st) {
   if (c.max_nL > 0) {
     dim3 g(c.max_nL * (c.max_nL + 1) / 2, c.num_seqs * c.Hq);
     if ((e = launch_chained(counts_kernel, g, dim3(DAM_TILE), st, c.blob, c.scratch, c.off_cnt)) != cudaSuccess) return e;
-    if ((e = launch_chained(match_kernel, dim3(c.num_seqs * c.Hq), dim3(256), st, c.blob, c.scratch, c.off_cnt, c.mu,
+    if ((e = launch_chained(match_kernel, dim3(c.num_seqs * c.Hq), dim3(1024), st, c.blob, c.scratch, c.off_cnt, c.mu,
                             c.min_support)) != cudaSuccess) return e;
   }
   if (c.rows > 0) {
