@@ -5,10 +5,13 @@
 // K / V tile that either of them lists, so a kv tile is brought into shared memory once per 256 query rows.
 // Warp roles:
 //   warp 0      TMA producer: both Q tiles once per item, then K and V of every kv tile in the union of
-//               the two tile lists into a ring of 32 KB shared-memory slots (128-byte swizzle);
-//   warp 1      MMA issuer (one elected thread): S_X = Q_X K^T into the stream's TMEM columns, then
-//               O_X += P_X V with P_X read from TMEM (it overwrites the first half of S_X); the two streams
-//               are interleaved so that one stream's softmax runs under the other stream's MMAs;
+//               the two tile lists ("step") into a ring of 32 KB shared-memory slots (128-byte swizzle); for
+//               every step it leaves a descriptor word in shared memory (which streams have a tile in it, whether
+//               it is a stream's last, whether the item goes on);
+//   warp 1      MMA issuer (one elected thread), driven by those descriptors alone (it reads no global memory):
+//               S_X = Q_X K^T into the stream's TMEM columns, then O_X += P_X V with P_X read from TMEM (it
+//               overwrites the first half of S_X); the two streams are interleaved so that one stream's softmax
+//               runs under the other stream's MMAs;
 //   warps 2-5   softmax of stream A, warps 6-9 of stream B: one thread per query row reads its S row from
 //               TMEM (twice: running max, then probabilities), applies the tile's mask bits where the tile
 //               is not fully active, writes P (bf16) back to TMEM, rescales O in TMEM when the running max
@@ -35,6 +38,10 @@ constexpr uint32_t kColS = 0;      // S_A at 0, S_B at 128 (P_X overwrites colum
 constexpr uint32_t kColO = 256;    // O_A at 256, O_B at 384
 constexpr float kRescaleThreshold = 8.0f;
 constexpr uint32_t kNone = 0xFFFFFFFFu;
+constexpr int kSchedNoSteps = 1 << 30;       // work-list entry handed to the consumers: nothing to multiply for it
+// Step descriptor bits: stream A / B has a tile in the step; it is the stream's last tile of the item; the item has
+// another step.
+constexpr uint32_t kStepA = 1u, kStepB = 2u, kStepLastA = 4u, kStepLastB = 8u, kStepMore = 16u;
 #ifndef DAM_POLY_PER8
 #define DAM_POLY_PER8 2
 #endif
@@ -49,7 +56,8 @@ struct SmemLayout {
   // sched_full[2], sched_empty[2]
   static constexpr int n_bars = 2 + 2 * kSlots + 10;
   static constexpr int sched_items = bars + 8 * n_bars;     // int[2]: work-list positions handed to the consumers
-  static constexpr int tmem_slot = sched_items + 8;
+  static constexpr int step_desc = sched_items + 8;         // u32[16]: what the producer found at each step (kStep*)
+  static constexpr int tmem_slot = step_desc + 64;
   static constexpr int abort_flag = tmem_slot + 4;
   static constexpr int total = abort_flag + 4;
 };
@@ -284,6 +292,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   const uint32_t bSFull = bSlotEmpty + 8 * kSlots, bPFull = bSFull + 16, bOFinal = bPFull + 16;
   const uint32_t bSchedFull = bOFinal + 16, bSchedEmpty = bSchedFull + 16;
   volatile int* sched_items = reinterpret_cast<volatile int*>(smem + SmemLayout::sched_items);
+  volatile uint32_t* step_desc = reinterpret_cast<volatile uint32_t*>(smem + SmemLayout::step_desc);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + SmemLayout::tmem_slot);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + SmemLayout::abort_flag);
 
@@ -328,7 +337,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      uint32_t sc = 0, ic = 0;
+      uint32_t sc = 0, ic = 0, step = 0;
       uint32_t armed[kSlots];
 #pragma unroll
       for (int s = 0; s < kSlots; ++s) armed[s] = 2u;      // 2 = never armed
@@ -353,11 +362,17 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (!(ok = mbar_wait(bSchedEmpty + 8 * slot, ((n >> 1) & 1u) ^ 1u, abort_flag))) break;
         int w = n == 0 ? (int)blockIdx.x : (int)(gridDim.x + atomicAdd(prm.work_counter, 1u));
         if (w >= nitems) w = -1;
-        sched_items[slot] = w;
+        Item it;
+        bool skip = false;
+        if (w >= 0) {
+          it = load_item(blob, H, w);
+          skip = it.a0 == it.b1 || !item_active(it);         // no tile in either list, or outside the row range
+        }
+        // the entry tells the MMA thread whether the item has steps at all, so that it never reads the work list
+        sched_items[slot] = w < 0 ? w : (w | (skip ? kSchedNoSteps : 0));
         mbar_arrive(bSchedFull + 8 * slot);
         if (w < 0) break;
-        const Item it = load_item(blob, H, w);
-        if (it.a0 == it.b1 || !item_active(it)) continue;    // no tile in either list, or outside the row range
+        if (skip) continue;
         if (!(ok = mbar_wait(bQEmpty, (ic & 1u) ^ 1u, abort_flag))) break;
         const int tokq = it.tok0 + it.qb0 * DAM_TILE;
         mbar_arrive_expect_tx(bQFull, it.hasB ? 2 * kSlotBytes : kSlotBytes);
@@ -378,6 +393,9 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         Walker wk; wk.init(tiles, it);
         int kb; uint32_t kA, kB;
         while (ok && wk.next(kb, kA, kB)) {
+          // what the MMA thread needs to know about this step, visible to it once the step's K tile has landed
+          step_desc[step++ & 15u] = (kA ? kStepA : 0u) | (kB ? kStepB : 0u) | (kA && wk.a_done() ? kStepLastA : 0u) |
+                                    (kB && wk.b_done() ? kStepLastB : 0u) | (wk.a_done() && wk.b_done() ? 0u : kStepMore);
           if (kA == DAM_KIND_GATHERED || kB == DAM_KIND_GATHERED) {
             const int row = (int)((gtile0 + kb) * 2 * DAM_TILE);
             ok = load_tile(&tmG, 0, row);
@@ -403,7 +421,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     if (lane == 0) {
       const uint32_t idesc_qk = idesc_bf16_f32(128, 128, 0);
       const uint32_t idesc_pv = idesc_bf16_f32(128, 128, 1);
-      uint32_t sc = 0, ic = 0;
+      uint32_t sc = 0, ic = 0, step = 0;
       uint32_t cP[2] = {0u, 0u};           // P tiles consumed per stream (phase of p_full)
       bool ok = true;
       PROF_DECL(6)
@@ -442,59 +460,53 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       for (uint32_t n = 0; ok; ++n) {
         const int w = next_item_consumer(n, true);
         if (w < 0) { ok = (w == -1); break; }
-        const Item it = load_item(blob, H, w);
-        if (it.a0 == it.b1 || !item_active(it)) continue;
-        Walker wk; wk.init(tiles, it);
-        int kb; uint32_t curA, curB;
-        wk.next(kb, curA, curB);                               // at least one step exists
+        if (w & kSchedNoSteps) continue;
         PROF_LAP(0)
         if (!(ok = mbar_wait(bQFull, ic & 1u, abort_flag))) break;
         PROF_LAP(3)
         ++ic;
-        // S of the first step
+        // S of the first step (the producer's descriptor of a step is readable once its K tile is)
+        uint32_t d;
         {
           const uint32_t s = sc % kSlots;
           if (!(ok = mbar_wait(bSlotFull + 8 * s, (sc / kSlots) & 1u, abort_flag))) break;
           PROF_LAP(4)
+          d = step_desc[step & 15u];
           tc_fence_after();
-          if (curA) issue_s(0, s);
-          if (curB) issue_s(1, s);
+          if (d & kStepA) issue_s(0, s);
+          if (d & kStepB) issue_s(1, s);
           tc_commit(bSlotEmpty + 8 * s);
           ++sc;
         }
         bool accA = false, accB = false;
         while (ok) {
-          uint32_t nxtA = 0, nxtB = 0;
-          const bool have_nxt = wk.next(kb, nxtA, nxtB);
+          const bool have_nxt = (d & kStepMore) != 0u;
           if (!have_nxt) tc_commit(bQEmpty);                   // every S of this item has been issued
           const uint32_t sv = sc % kSlots;                     // V of the current step
           PROF_LAP(0)
           if (!(ok = mbar_wait(bSlotFull + 8 * sv, (sc / kSlots) & 1u, abort_flag))) break;
           PROF_LAP(4)
           ++sc;
-          uint32_t sk = 0;
+          uint32_t sk = 0, dn = 0;
           // a stream's output is final right after the P V of its last listed tile
-          const bool lastA = curA && nxtA == 0u && wk.a_done();
-          const bool lastB = curB && nxtB == 0u && wk.b_done();
-          if (curA) { if (!(ok = issue_pv(0, sv, accA))) break; accA = true; if (lastA) tc_commit(bOFinal); }
+          if (d & kStepA) { if (!(ok = issue_pv(0, sv, accA))) break; accA = true; if (d & kStepLastA) tc_commit(bOFinal); }
           if (have_nxt) {                                      // K of the next step
             sk = sc % kSlots;
             PROF_LAP(0)
             if (!(ok = mbar_wait(bSlotFull + 8 * sk, (sc / kSlots) & 1u, abort_flag))) break;
             PROF_LAP(4)
             ++sc;
+            dn = step_desc[(step + 1u) & 15u];
             tc_fence_after();
-            if (nxtA) issue_s(0, sk);
+            if (dn & kStepA) issue_s(0, sk);
           }
-          if (curB) { if (!(ok = issue_pv(1, sv, accB))) break; accB = true; if (lastB) tc_commit(bOFinal + 8); }
+          if (d & kStepB) { if (!(ok = issue_pv(1, sv, accB))) break; accB = true; if (d & kStepLastB) tc_commit(bOFinal + 8); }
           tc_commit(bSlotEmpty + 8 * sv);
-          if (have_nxt) {
-            if (nxtB) issue_s(1, sk);
-            tc_commit(bSlotEmpty + 8 * sk);
-          } else {
-            break;
-          }
-          curA = nxtA; curB = nxtB;
+          ++step;
+          if (!have_nxt) break;
+          if (dn & kStepB) issue_s(1, sk);
+          tc_commit(bSlotEmpty + 8 * sk);
+          d = dn;
         }
       }
       PROF_LAP(0)
@@ -517,10 +529,11 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     bool ok = true;
     PROF_DECL(8)
     for (uint32_t n = 0; ok; ++n) {
-      const int w = next_item_consumer(n, false);
+      const int ws = next_item_consumer(n, false);
       __syncwarp();
-      if (lane == 0 && w != -2) mbar_arrive(bSchedEmpty + 8 * (n & 1u));    // the whole warp has read the entry
-      if (w < 0) { ok = (w == -1); break; }
+      if (lane == 0 && ws != -2) mbar_arrive(bSchedEmpty + 8 * (n & 1u));   // the whole warp has read the entry
+      if (ws < 0) { ok = (ws == -1); break; }
+      const int w = ws & ~kSchedNoSteps;
       const Item it = load_item(blob, H, w);
       if ((X == 1 && !it.hasB) || !item_active(it)) continue;
       const int qb = it.qb0 + X;
