@@ -346,10 +346,10 @@ _HDR = np.dtype([("magic", "<u4"), ("status", "<u4"), ("version", "<u4"), ("flag
                  ("off_seq", "<u8"), ("off_qbseq", "<u8"), ("off_dv", "<u8"), ("off_true", "<u8"),
                  ("off_tile_ptr", "<u8"), ("off_work", "<u8"), ("off_tiles", "<u8"), ("bytes_used", "<u8"),
                  ("causal_tiles", "<u8"), ("off_pairtab", "<u8"), ("total_pairs", "<i4"), ("prows", "<i4"),
-                 ("gath_tiles", "<u8"), ("attn_scratch_bytes", "<u8"), ("mask_tiles", "<u8"), ("reserved", "<u8", (12,))])
+                 ("gath_tiles", "<u8"), ("attn_scratch_bytes", "<u8"), ("mask_tiles", "<u8"), ("head_tile_cap", "<u8"), ("reserved", "<u8", (11,))])
 _SEQ = np.dtype([("tok_start", "<i4"), ("S", "<i4"), ("L", "<i4"), ("nq", "<i4"), ("first_qblock", "<i4"),
                  ("W", "<i4"), ("nL", "<i4"), ("first_pair", "<i4"), ("dv_off", "<u8"), ("true_off", "<u8"),
-                 ("p_off", "<u8"), ("cnt_off", "<u8"), ("gath_off", "<u8"), ("reserved", "<u8")])
+                 ("p_off", "<u8"), ("cnt_off", "<u8"), ("gath_off", "<u8"), ("tile_base", "<u8")])
 
 
 _ITEM = np.dtype([("head", "<i4"), ("tok0", "<i4"), ("qb0", "<i4"), ("S", "<i4"), ("a0", "<u4"), ("a1", "<u4"),
@@ -379,7 +379,8 @@ class MaskBlob:
                                    offset=int(self.hdr["off_work"]))
         self.pair_tab = np.frombuffer(self.raw, dtype="<u4", count=int(self.hdr["total_pairs"]),
                                       offset=int(self.hdr["off_pairtab"]))
-        self.tiles = np.frombuffer(self.raw, dtype="<u4", count=int(self.hdr["total_tiles"]),
+        # every row owns a fixed range of tiles[]: its entries, then possibly zero entries (kind 0) as padding
+        self.tiles = np.frombuffer(self.raw, dtype="<u4", count=int(self.tile_ptr[rows]),
                                    offset=int(self.hdr["off_tiles"]))
 
     def pattern_bits(self, seq: int, head: int):
@@ -418,11 +419,12 @@ class MaskBlob:
     def row_tiles(self, seq: int, head: int, qb: int):
         """(kv tile indices, kinds) of query block qb of (seq, head)."""
         row = head * int(self.hdr["total_qblocks"]) + int(self.seqs[seq]["first_qblock"]) + qb
-        e = self.tiles[self.tile_ptr[row]: self.tile_ptr[row + 1]]
+        e = self.row_entries(seq, head, qb)
         kinds = (e >> 28).astype(np.int64)
         idx = np.where(kinds == 3, e & 0xFFFF, e & 0x0FFFFFFF).astype(np.int64)
         return idx, kinds
 
     def row_entries(self, seq: int, head: int, qb: int) -> np.ndarray:
         row = head * int(self.hdr["total_qblocks"]) + int(self.seqs[seq]["first_qblock"]) + qb
-        return self.tiles[self.tile_ptr[row]: self.tile_ptr[row + 1]]
+        e = self.tiles[self.tile_ptr[row]: self.tile_ptr[row + 1]]
+        return e[(e >> 28) != 0]                                    # without the padding

@@ -15,7 +15,7 @@ struct Layout {
   size_t mask_bytes;
   size_t build_scratch_bytes;
   size_t attn_scratch_bytes;
-  uint64_t off_cnt, off_cnt_end, off_rowcnt, off_hist, off_cursor;
+  uint64_t off_cnt, off_cnt_end, off_rowcnt, off_hist, off_cursor, off_items;
   int max_L, max_W, max_nL, max_nq;
   uint64_t score_elems;
 };
@@ -117,13 +117,14 @@ void compute_layout(const dam_shape_t* s, int pcl_max, int all_ones_causal, int 
   h.off_tiles = dam_align(h.off_work + (uint64_t)sizeof(DamItem) * h.prows, 256);
   h.causal_tiles = causal_tiles;
   y.mask_bytes = dam_align(h.off_tiles + 4ull * cap, 256);
-  // build scratch: [0,256) status block and work counter | counts | row counts | hist | cursor
+  // build scratch: [0,256) status block and work counter | counts | row counts | hist | cursor | unordered items
   y.off_cnt = 256;
   y.off_cnt_end = dam_align(y.off_cnt + 4ull * cnt, 256);
   y.off_rowcnt = y.off_cnt_end;
   y.off_hist = dam_align(y.off_rowcnt + 4ull * h.rows, 256);
   y.off_cursor = y.off_hist + 4ull * DAM_HIST;
-  y.build_scratch_bytes = dam_align(y.off_cursor + 4ull * DAM_HIST, 256);
+  y.off_items = dam_align(y.off_cursor + 4ull * DAM_HIST, 256);          // work items before they are ordered
+  y.build_scratch_bytes = dam_align(y.off_items + (uint64_t)sizeof(DamItem) * h.prows, 256);
   // attention scratch: 256-byte status block, then (gathered columns only) one K tile and one V tile of
   // 128 keys per gathered-column tile
   h.gath_tiles = (pcl_max > 0 && gather) ? gath : 0;
@@ -211,7 +212,7 @@ dam_status_t fill_ctx(const dam_shape_t* s, const dam_rule_t* r, void* mask, siz
   c->pstar = c->per_map ? INFINITY : find_pstar(r);
   c->mu = r->mu; c->min_support = r->min_support;
   c->scale = r->softmax_scale > 0.f ? r->softmax_scale : 1.0f / sqrtf((float)s->head_dim);
-  c->off_cnt = y->off_cnt; c->off_cnt_end = y->off_cnt_end; c->off_rowcnt = y->off_rowcnt;
+  c->off_cnt = y->off_cnt; c->off_cnt_end = y->off_cnt_end; c->off_rowcnt = y->off_rowcnt; c->off_items = y->off_items;
   c->off_hist = y->off_hist; c->off_cursor = y->off_cursor;
   c->gather = gather;
   c->off_true = y->hdr.off_true; c->true_bytes = y->hdr.off_tile_ptr - y->hdr.off_true;

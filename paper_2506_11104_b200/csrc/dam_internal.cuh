@@ -12,7 +12,12 @@
 //   per (seq, head) true mask    L rows x W words, bit (j % 32) of word (j / 32) = M[i][j]
 //   pair_tab[total_pairs]        first global q-block of every pair of adjacent q-blocks (2p, 2p+1) of a
 //                                sequence; bit 31 set when the second block exists
-//   tile_ptr[rows + 1]           CSR over rows = head * total_qblocks + global q-block
+//   tile_ptr[rows + 1]           start of every row's entries in tiles[], rows = head * total_qblocks + global
+//                                q-block.  Every pair of adjacent q-blocks owns a fixed range of tiles[] (the sum
+//                                of the two rows' upper bounds, known from the shapes alone): the first row's
+//                                entries, directly followed by the second row's, then zero entries (kind 0) up to
+//                                the next pair.  [tile_ptr[r], tile_ptr[r + 1]) therefore holds row r's entries
+//                                and possibly zero entries behind them, which every reader skips.
 //   items[prows]                 work list of the attention kernel (DamItem, 32 B): one entry per
 //                                (head, pair), the pair with the most listed tiles (both blocks
 //                                together) first, with everything a CTA needs to start on it
@@ -58,7 +63,8 @@ struct DamHeader {
   uint64_t gath_tiles;      // gathered-column tiles over all (seq, head): sum Hq * nL (capacity, 128 keys each)
   uint64_t attn_scratch_bytes;   // scratch dam_sparse_attention needs for this blob
   uint64_t mask_tiles;      // 128 x 128 tiles of the masks that hold an active cell (= total_tiles unless gathered)
-  uint64_t reserved[12];
+  uint64_t head_tile_cap;   // entries of tiles[] every head owns (sum of the row bounds of all sequences)
+  uint64_t reserved[11];
 };
 static_assert(sizeof(DamHeader) == 256, "DamHeader must be 256 bytes");
 
@@ -77,7 +83,7 @@ struct DamSeq {
   uint64_t p_off;      // fp32 elements into a score tensor: head h at p_off + h * L * L
   uint64_t cnt_off;    // int32 elements into the build scratch count area: head h at cnt_off + h * cnt_stride
   uint64_t gath_off;   // gathered-column tiles: head h owns tiles [gath_off + h * nL, +nL)
-  uint64_t reserved;
+  uint64_t tile_base;  // first entry of the sequence's rows inside a head's range of tiles[]
 };
 static_assert(sizeof(DamSeq) == 80, "DamSeq must be 80 bytes");
 
@@ -101,6 +107,17 @@ __host__ __device__ inline int dam_row_tile_bound(int qb, int nL, int L, int gat
   }
   int a = qb + 1, b = 2 * nL + 1;
   return a < b ? a : b;
+}
+
+// Sum of dam_row_tile_bound over the query blocks 0 .. qb-1 of a sequence: where block qb's entries start inside
+// the sequence's range of a head.  (From the first gathered block on every bound is 2 nL + 1: nL gathered tiles
+// and the nL + 1 band tiles; before it, min(q + 1, 2 nL + 1).)
+__host__ __device__ inline uint64_t dam_row_tile_prefix(int qb, int nL, int L, int gather) {
+  const int gather_first = (2 * L - 1 + DAM_TILE - 1) / DAM_TILE;
+  const uint64_t m = 2ull * nL + 1;
+  const uint64_t k = (gather && L > 0 && qb > gather_first) ? (uint64_t)gather_first : (uint64_t)qb;   // blocks on the plain rule
+  const uint64_t j = k < m ? k : m;
+  return j * (j + 1) / 2 + (k - j) * m + ((uint64_t)qb - k) * m;
 }
 
 // Gathered-column tiles serve the query blocks that start at or after row 2L - 1 (first multiple of 128).
@@ -202,7 +219,7 @@ struct DamBuildCtx {
   int min_support;
   float scale;
   int gather;        // list gathered-column tiles
-  uint64_t off_cnt, off_cnt_end, off_rowcnt, off_hist, off_cursor;   // scratch sections
+  uint64_t off_cnt, off_cnt_end, off_rowcnt, off_hist, off_cursor, off_items;   // scratch sections
   uint64_t off_true, true_bytes;                                     // true-mask section of the blob
 };
 

@@ -44,8 +44,9 @@ __global__ void init_blob_kernel(unsigned char* blob, DamHeader hdr, const int32
   uint32_t* pairtab = reinterpret_cast<uint32_t*>(blob + hdr.off_pairtab);
   if (threadIdx.x == 0) {
     *H = hdr;
-    uint64_t dv = 0, tr = 0, po = 0, co = 0, go = 0;
+    uint64_t dv = 0, tr = 0, po = 0, co = 0, go = 0, tb = 0;
     int fq = 0, fp = 0;
+    const int gather = (hdr.flags & DAM_FLAG_GATHER) ? 1 : 0;
     for (int b = 0; b < hdr.num_seqs; ++b) {
       int t0 = cu[b], S = cu[b + 1] - t0;
       int L = S < pcl_max ? S : pcl_max;
@@ -56,7 +57,7 @@ __global__ void init_blob_kernel(unsigned char* blob, DamHeader hdr, const int32
       DamSeq s;
       s.tok_start = t0; s.S = S; s.L = L; s.nq = nq;
       s.first_qblock = fq; s.W = W; s.nL = nL; s.first_pair = fp;
-      s.dv_off = dv; s.true_off = tr; s.p_off = po; s.cnt_off = co; s.gath_off = go; s.reserved = 0;
+      s.dv_off = dv; s.true_off = tr; s.p_off = po; s.cnt_off = co; s.gath_off = go; s.tile_base = tb;
       seqs[b] = s;
       dv += (uint64_t)Hq * 3 * W;
       tr += (uint64_t)Hq * L * W;
@@ -64,8 +65,15 @@ __global__ void init_blob_kernel(unsigned char* blob, DamHeader hdr, const int32
       if (all_ones_causal < 0) co += (uint64_t)Hq * dam_cnt_stride(L, W, nL);
       else co += all_ones_causal ? (uint64_t)nq * (nq + 1) / 2 : (uint64_t)nq * nq;   // tile base per head
       go += (uint64_t)Hq * nL;
+      if (all_ones_causal < 0) tb += dam_row_tile_prefix(nq, nL, L, gather);
       fq += nq;
       fp += (nq + 1) / 2;
+    }
+    H->head_tile_cap = tb;
+    if (all_ones_causal < 0) {
+      // the tile lists have a fixed place per row (see the layout notes): nothing to compact, no sizes to wait for
+      H->bytes_used = hdr.off_tiles + 4ull * Hq * tb;
+      reinterpret_cast<uint32_t*>(blob + hdr.off_tile_ptr)[hdr.rows] = (uint32_t)(Hq * tb);
     }
   }
   __syncthreads();
@@ -258,7 +266,8 @@ __global__ void match_kernel(unsigned char* blob, unsigned char* scratch, uint64
 
 // ---------------------------------------------------------------------------------------------
 // Tile classification.  One warp per row = (head, global q-block); lanes test candidate kv tiles in
-// ascending order.  pass 0 counts, pass 1 writes entries at tile_ptr[row] + rank.
+// ascending order and writes the kept ones into the pair's fixed range of tiles[] (one pass: nothing is counted
+// first, nothing is compacted afterwards).
 // ---------------------------------------------------------------------------------------------
 struct HeadView {
   const uint32_t* Dw; const uint32_t* Vw;
@@ -322,14 +331,17 @@ __device__ __forceinline__ uint32_t classify_band(const HeadView& v, int qb, int
   return (whole && n == 2 * DAM_TILE - 1) ? DAM_KIND_FULL : DAM_KIND_PARTIAL;
 }
 
-template <int PASS>
-__global__ void classify_kernel(unsigned char* blob, unsigned char* scratch, uint64_t off_cnt, uint64_t off_rowcnt,
-                                uint64_t off_hist, uint64_t off_cursor) {
+__global__ void classify_kernel(unsigned char* blob, unsigned char* scratch, uint64_t off_cnt, uint64_t off_items) {
   dam_chain_prologue();
   DamHeader* H = reinterpret_cast<DamHeader*>(blob);
   const int lane = threadIdx.x & 31;
   const int prow = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);   // one warp per (head, q-block pair)
-  if (prow >= H->prows) return;
+  // block totals of the three statistics: one global atomic per block instead of one per warp on the same address
+  __shared__ unsigned long long s_mask_tiles;
+  __shared__ uint32_t s_total, s_full;
+  if (threadIdx.x == 0) { s_mask_tiles = 0ull; s_total = 0u; s_full = 0u; }
+  __syncthreads();
+  if (prow < H->prows) {
   const int h = prow / H->total_pairs, gp = prow % H->total_pairs;
   const uint32_t pt = reinterpret_cast<const uint32_t*>(blob + H->off_pairtab)[gp];
   const int gqb0 = (int)(pt & 0x7FFFFFFFu), nblk = (pt >> 31) ? 2 : 1;
@@ -342,9 +354,15 @@ __global__ void classify_kernel(unsigned char* blob, unsigned char* scratch, uin
   v.Dw = dv; v.Vw = dv + 2 * sq.W;
   v.prefD = cnt + 2 * sq.L; v.prefV = v.prefD + (sq.W + 1); v.tile_pop = v.prefV + (sq.W + 1);
   v.L = sq.L; v.W = sq.W; v.nL = sq.nL; v.S = sq.S;
-  uint32_t* rowcnt = reinterpret_cast<uint32_t*>(scratch + off_rowcnt);
   uint32_t* tile_ptr = reinterpret_cast<uint32_t*>(blob + H->off_tile_ptr);
   uint32_t* tiles = reinterpret_cast<uint32_t*>(blob + H->off_tiles);
+  const int gflag = (H->flags & DAM_FLAG_GATHER) ? 1 : 0;
+  const int qb0 = gqb0 - sq.first_qblock;
+  // the pair's fixed range of tiles[]: entries of block qb0, then of block qb0 + 1, then zeros
+  const uint64_t head_base = (uint64_t)h * H->head_tile_cap + sq.tile_base;
+  const uint32_t pair_begin = (uint32_t)(head_base + dam_row_tile_prefix(qb0, sq.nL, sq.L, gflag));
+  const uint32_t pair_end = (uint32_t)(head_base + dam_row_tile_prefix(qb0 + nblk, sq.nL, sq.L, gflag));
+  uint32_t base = pair_begin, a1 = pair_begin;
   int pair_total = 0, nfull = 0, mask_tiles = 0;
   for (int x = 0; x < nblk; ++x) {
     const int gqb = gqb0 + x;
@@ -353,22 +371,20 @@ __global__ void classify_kernel(unsigned char* blob, unsigned char* scratch, uin
     // candidates, ascending: [0, min(qb, nL-1)] then [max(that + 1, qb - nL), qb].  From row 2L - 1 on
     // (gathered columns enabled) the first range is replaced by the gathered tiles and the second range
     // is classified on the matched diagonals alone.
-    const bool gathered = (H->flags & DAM_FLAG_GATHER) && sq.L > 0 && qb >= dam_gather_first_qblock(sq.L);
+    const bool gathered = gflag && sq.L > 0 && qb >= dam_gather_first_qblock(sq.L);
     const int nV = gathered ? v.prefV[sq.W] : 0;
     const int n1 = gathered ? (nV + DAM_TILE - 1) / DAM_TILE : min(qb, sq.nL - 1) + 1;
     const int lo2 = gathered ? max(0, qb - sq.nL) : max(n1, qb - sq.nL);
     const int n2 = max(0, qb - lo2 + 1);
-    uint32_t base = 0;
-    bool write = PASS == 1;
-    if (PASS == 1) {
-      base = tile_ptr[row];
-      if (base + rowcnt[row] > H->tile_capacity) write = false;   // overflow already flagged by the scan
-    }
-    int total = 0;
-    for (int c0 = 0; c0 < n1 + n2; c0 += 32) {
+    // tiles of the mask itself (128 x 128 grid) with an active cell are counted in the same sweep (their loads
+    // overlap the classification's): they equal the listed tiles unless the row is served by gathered tiles
+    const int m1 = min(qb, sq.nL - 1) + 1, l2 = max(m1, qb - sq.nL), m2 = max(0, qb - l2 + 1);
+    const int ncand = n1 + n2, nmask = gathered ? m1 + m2 : 0;
+    int total = 0, nat = 0;
+    for (int c0 = 0; c0 < max(ncand, nmask); c0 += 32) {
       int idx = c0 + lane;
       uint32_t kind = 0, entry = 0;
-      if (idx < n1 + n2) {
+      if (idx < ncand) {
         if (gathered && idx < n1) {
           kind = DAM_KIND_GATHERED;
           entry = (uint32_t)idx | ((uint32_t)(min(DAM_TILE, nV - idx * DAM_TILE) - 1) << 16) | (kind << 28);
@@ -378,53 +394,48 @@ __global__ void classify_kernel(unsigned char* blob, unsigned char* scratch, uin
           entry = (uint32_t)kb | (kind << 28);
         }
       }
+      const bool act = idx < nmask && classify_tile(v, qb, idx < m1 ? idx : l2 + (idx - m1)) != 0u;
       uint32_t m = __ballot_sync(0xFFFFFFFFu, kind != 0);
-      if (write && kind) {
+      if (kind) {
         int rank = __popc(m & ((1u << lane) - 1u));
-        tiles[base + total + rank] = entry;
+        if (base + total + rank < pair_end) tiles[base + total + rank] = entry;     // always true: the range is the bound
       }
-      if (PASS == 1) nfull += __popc(__ballot_sync(0xFFFFFFFFu, kind == DAM_KIND_FULL || (kind == DAM_KIND_GATHERED && ((entry >> 16) & 0xFFu) == DAM_TILE - 1)));
+      nfull += __popc(__ballot_sync(0xFFFFFFFFu, kind == DAM_KIND_FULL || (kind == DAM_KIND_GATHERED && ((entry >> 16) & 0xFFu) == DAM_TILE - 1)));
       total += __popc(m);
+      nat += __popc(__ballot_sync(0xFFFFFFFFu, act));
     }
-    if (PASS == 0 && lane == 0) rowcnt[row] = total;
+    if (lane == 0) tile_ptr[row] = base;
+    base += total;
+    if (x == 0) a1 = base;
     pair_total += total;
-    if (PASS == 0) {
-      // tiles of the mask itself (128 x 128 grid) with an active cell: equals `total` unless gathered
-      int nat = total;
-      if (gathered) {
-        nat = 0;
-        const int m1 = min(qb, sq.nL - 1) + 1, l2 = max(m1, qb - sq.nL), m2 = max(0, qb - l2 + 1);
-        for (int c0 = 0; c0 < m1 + m2; c0 += 32) {
-          const int idx = c0 + lane;
-          const bool act = idx < m1 + m2 && classify_tile(v, qb, idx < m1 ? idx : l2 + (idx - m1)) != 0u;
-          nat += __popc(__ballot_sync(0xFFFFFFFFu, act));
-        }
-      }
-      mask_tiles += nat;
-    }
+    if (!gathered) nat = total;
+    mask_tiles += nat;
   }
+  // zero entries up to the next pair
+  for (uint32_t t = base + lane; t < pair_end; t += 32) tiles[t] = 0u;
   if (lane == 0) {
-    const int key = min(pair_total, DAM_HIST - 1);
-    if (PASS == 0) {
-      atomicAdd(reinterpret_cast<uint32_t*>(scratch + off_hist) + key, 1u);
-      atomicAdd(reinterpret_cast<unsigned long long*>(&H->mask_tiles), (unsigned long long)mask_tiles);
-    } else {
-      uint32_t pos = atomicAdd(reinterpret_cast<uint32_t*>(scratch + off_cursor) + key, 1u);
-      const int rowA = h * H->total_qblocks + gqb0;
-      DamItem it;
-      it.head = h; it.tok0 = sq.tok_start; it.qb0 = gqb0 - sq.first_qblock; it.S = sq.S;
-      it.a0 = tile_ptr[rowA]; it.a1 = it.a0 + rowcnt[rowA];
-      it.b1 = it.a1 + (nblk == 2 ? rowcnt[rowA + 1] : 0u);
-      it.seq_hasB = (uint32_t)b | (nblk == 2 ? 0x80000000u : 0u);
-      reinterpret_cast<DamItem*>(blob + H->off_work)[pos] = it;
-      if (nfull) atomicAdd(&H->full_tiles, (uint32_t)nfull);
-    }
+    // the work item, at the pair's own index for now: the ordering kernel moves it to its place in the work list
+    DamItem it;
+    it.head = h; it.tok0 = sq.tok_start; it.qb0 = qb0; it.S = sq.S;
+    it.a0 = pair_begin; it.a1 = a1; it.b1 = base;
+    it.seq_hasB = (uint32_t)b | (nblk == 2 ? 0x80000000u : 0u);
+    reinterpret_cast<DamItem*>(scratch + off_items)[prow] = it;
+    atomicAdd(&s_mask_tiles, (unsigned long long)mask_tiles);
+    atomicAdd(&s_total, (uint32_t)pair_total);
+    atomicAdd(&s_full, (uint32_t)nfull);
+  }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    if (s_mask_tiles) atomicAdd(reinterpret_cast<unsigned long long*>(&H->mask_tiles), s_mask_tiles);
+    if (s_total) atomicAdd(&H->total_tiles, s_total);
+    if (s_full) atomicAdd(&H->full_tiles, s_full);
   }
 }
 
 // ---------------------------------------------------------------------------------------------
-// Exclusive scans, one block of 1024 threads: tile_ptr over row counts, and the work-order
-// cursors (rows with more tiles first) over the histogram.
+// Work order: the pairs are sorted by listed tiles, most first (a counting sort: histogram, exclusive scan,
+// placement).  Blocks of 1024 threads; every block places 1024 pairs.
 // ---------------------------------------------------------------------------------------------
 __device__ uint32_t block_excl_scan(uint32_t x, uint32_t* total, uint32_t* sm /* 32 */) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -453,91 +464,72 @@ __device__ uint32_t block_excl_scan(uint32_t x, uint32_t* total, uint32_t* sm /*
   return r;
 }
 
-__global__ void scan_kernel(unsigned char* blob, unsigned char* scratch, uint64_t off_rowcnt, uint64_t off_hist,
-                            uint64_t off_cursor) {
+__global__ void __launch_bounds__(1024)
+order_kernel(unsigned char* blob, unsigned char* scratch, uint64_t off_items) {
   dam_chain_prologue();
   DamHeader* H = reinterpret_cast<DamHeader*>(blob);
   __shared__ uint32_t sm[32];
   __shared__ uint32_t tot;
-  const uint32_t* rowcnt = reinterpret_cast<const uint32_t*>(scratch + off_rowcnt);
-  uint32_t* tile_ptr = reinterpret_cast<uint32_t*>(blob + H->off_tile_ptr);
-  const int rows = H->rows;
-  // every thread owns a contiguous run of rows (a multiple of 4, read with 16-byte loads that are all in flight
-  // at once): run totals, one block-wide scan over them, then the rows again from registers
-  {
-    constexpr int kMaxPer = 32;                                  // rows per thread held in registers
-    const int per = (((rows + (int)blockDim.x - 1) / (int)blockDim.x) + 3) & ~3;
-    if (per <= kMaxPer) {
-      const int r0 = threadIdx.x * per;
-      uint4 v[kMaxPer / 4];
-      uint32_t local = 0;
+  __shared__ uint32_t start[DAM_HIST];      // pairs per key, then the first place of the key's bucket
+  __shared__ uint32_t before[DAM_HIST];     // pairs per key that precede this block's share, then the running cursor
+  const uint4* src = reinterpret_cast<const uint4*>(scratch + off_items);
+  uint4* dst = reinterpret_cast<uint4*>(blob + H->off_work);
+  const int prows = H->prows, total_pairs = H->total_pairs, Hq = H->num_q_heads;
+  for (int k = threadIdx.x; k < DAM_HIST; k += blockDim.x) { start[k] = 0u; before[k] = 0u; }
+  __syncthreads();
+  // Every block places blockDim.x pairs and needs nothing from the other blocks: it counts all pairs per key
+  // itself, and those that precede its share.  Inside a bucket the pairs keep the order (pair, head): the query
+  // heads of one KV head at the same pair of query blocks list the same kv tiles, and neighbours in the work
+  // list run at the same time on different SMs, so the second to fourth find the K and V tiles in L2.  An item
+  // is two 16-byte words: head, tok0, qb0, S | a0, a1, b1, seq_hasB; its key is the number of listed tiles.
+  const int lane = threadIdx.x & 31;
+  const int my_begin = blockIdx.x * (int)blockDim.x;
+  auto item_of = [&](int idx) -> size_t { return 2 * (size_t)((idx % Hq) * total_pairs + idx / Hq); };
+  auto key_of = [](const uint4& v) -> uint32_t { return min(v.z - v.x, (uint32_t)(DAM_HIST - 1)); };
+  // lanes of a warp that share a key count together (most pairs of a layer share one key)
+  auto count = [&](uint32_t* hist, uint32_t key) {
+    const uint32_t same = __match_any_sync(0xFFFFFFFFu, key);
+    if (key != 0xFFFFFFFFu && lane == __ffs(same) - 1) atomicAdd(&hist[key], (uint32_t)__popc(same));
+  };
+  for (int i0 = 0; i0 < prows; i0 += 4 * (int)blockDim.x) {
+    uint32_t k[4];
 #pragma unroll
-      for (int q = 0; q < kMaxPer / 4; ++q) {
-        v[q] = make_uint4(0u, 0u, 0u, 0u);
-        const int r = r0 + 4 * q;
-        if (4 * q < per && r < rows) {
-          if (r + 3 < rows) v[q] = *reinterpret_cast<const uint4*>(rowcnt + r);
-          else { v[q].x = rowcnt[r]; if (r + 1 < rows) v[q].y = rowcnt[r + 1]; if (r + 2 < rows) v[q].z = rowcnt[r + 2]; }
-        }
-        local += v[q].x + v[q].y + v[q].z + v[q].w;
-      }
-      uint32_t run = block_excl_scan(local, &tot, sm);
-#pragma unroll
-      for (int q = 0; q < kMaxPer / 4; ++q) {
-        const int r = r0 + 4 * q;
-        if (4 * q < per && r < rows) {
-          const uint4 o = make_uint4(run, run + v[q].x, run + v[q].x + v[q].y, run + v[q].x + v[q].y + v[q].z);
-          if (r + 3 < rows) *reinterpret_cast<uint4*>(tile_ptr + r) = o;
-          else { tile_ptr[r] = o.x; if (r + 1 < rows) tile_ptr[r + 1] = o.y; if (r + 2 < rows) tile_ptr[r + 2] = o.z; }
-          run += v[q].x + v[q].y + v[q].z + v[q].w;
-        }
-      }
-    } else {
-      // more rows than the registers hold: every warp walks a contiguous segment 32 rows at a time, twice
-      const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
-      const int seg = ((rows + nw - 1) / nw + 31) & ~31;
-      const int r0 = warp * seg, r1 = min(rows, r0 + seg);
-      uint32_t local = 0;
-      for (int r = r0 + lane; r < r1; r += 32) local += rowcnt[r];
-#pragma unroll
-      for (int o = 16; o; o >>= 1) local += __shfl_xor_sync(0xFFFFFFFFu, local, o);
-      __shared__ uint32_t seg_base[32];
-      uint32_t e = block_excl_scan(lane == 0 ? local : 0u, &tot, sm);
-      if (lane == 0) seg_base[warp] = e;
-      __syncthreads();
-      uint32_t run = seg_base[warp];
-      for (int rb = r0; rb < r1; rb += 32) {
-        const int r = rb + lane;
-        const uint32_t x = r < r1 ? rowcnt[r] : 0u;
-        uint32_t inc = x;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-          if (lane >= o) inc += y;
-        }
-        if (r < r1) tile_ptr[r] = run + inc - x;
-        run += __shfl_sync(0xFFFFFFFFu, inc, 31);
-      }
+    for (int j = 0; j < 4; ++j) {
+      const int idx = i0 + j * (int)blockDim.x + (int)threadIdx.x;
+      k[j] = idx < prows ? key_of(src[item_of(idx) + 1]) : 0xFFFFFFFFu;
     }
-    if (threadIdx.x == 0) {
-      const uint32_t total = tot;
-      tile_ptr[rows] = total;
-      H->total_tiles = total;
-      H->bytes_used = H->off_tiles + 4ull * total;
-      if (total > H->tile_capacity) H->status = DAM_ERR_BUFFER_TOO_SMALL;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int idx0 = i0 + j * (int)blockDim.x;                  // first index of this warp-uniform batch
+      count(start, k[j]);
+      if (idx0 + (int)blockDim.x <= my_begin) count(before, k[j]);   // batches are aligned to the blocks' shares
     }
-    __syncthreads();
   }
-  // cursors: bucket c starts after all buckets with more tiles (descending order of the key)
+  __syncthreads();
+  // first place of every bucket: after all buckets with more tiles (descending order of the key)
   {
-    const uint32_t* hist = reinterpret_cast<const uint32_t*>(scratch + off_hist);
-    uint32_t* cursor = reinterpret_cast<uint32_t*>(scratch + off_cursor);
     const int per = (DAM_HIST + blockDim.x - 1) / blockDim.x;
-    const int k0 = threadIdx.x * per, k1 = min(DAM_HIST, k0 + per);     // positions in descending-key order
+    const int q0 = threadIdx.x * per, q1 = min(DAM_HIST, q0 + per);     // positions in descending-key order
     uint32_t local = 0;
-    for (int k = k0; k < k1; ++k) local += hist[DAM_HIST - 1 - k];
+    for (int k = q0; k < q1; ++k) local += start[DAM_HIST - 1 - k];
     uint32_t e = block_excl_scan(local, &tot, sm);
-    for (int k = k0; k < k1; ++k) { cursor[DAM_HIST - 1 - k] = e; e += hist[DAM_HIST - 1 - k]; }
+    for (int k = q0; k < q1; ++k) { const uint32_t c = start[DAM_HIST - 1 - k]; start[DAM_HIST - 1 - k] = e; e += c; }
+  }
+  __syncthreads();
+  {
+    const int idx = my_begin + (int)threadIdx.x;
+    uint4 u = make_uint4(0u, 0u, 0u, 0u), v = u;
+    uint32_t key = 0xFFFFFFFFu;
+    if (idx < prows) { u = src[item_of(idx)]; v = src[item_of(idx) + 1]; key = key_of(v); }
+    const uint32_t same = __match_any_sync(0xFFFFFFFFu, key);
+    const int leader = __ffs(same) - 1;
+    uint32_t base = 0u;
+    if (key != 0xFFFFFFFFu && lane == leader) base = start[key] + atomicAdd(&before[key], (uint32_t)__popc(same));
+    base = __shfl_sync(0xFFFFFFFFu, base, leader);
+    if (key != 0xFFFFFFFFu) {
+      const uint32_t pos = base + (uint32_t)__popc(same & ((1u << lane) - 1u));
+      dst[2 * (size_t)pos] = u; dst[2 * (size_t)pos + 1] = v;
+    }
   }
 }
 
@@ -606,7 +598,7 @@ __global__ void expand_rows_kernel(const unsigned char* blob, int seq, int head,
   DamHeadBits hb = dam_head_bits(blob, H, sq, head);
   for (uint32_t t = tile_ptr[row] + threadIdx.x; t < tile_ptr[row + 1]; t += blockDim.x) {
     uint32_t e = tiles[t];
-    if ((e >> 28) == DAM_KIND_GATHERED) continue;          // handled below
+    if ((e >> 28) == 0u || (e >> 28) == DAM_KIND_GATHERED) continue;   // padding; gathered tiles are handled below
     int kb = (int)(e & 0x0FFFFFFFu);
     uint4 bits = dam_apply_bits(hb, e >> 28, i, kb, causal);
     if (kb * 4 + 3 < words) {
@@ -835,12 +827,11 @@ cudaError_t dam_launch_rule(const DamBuildCtx& c, cudaStream_t st) {
   }
   if (c.rows > 0) {
     int blocks = (c.prows + 7) / 8;
-    if ((e = launch_chained(classify_kernel<0>, dim3(blocks), dim3(256), st, c.blob, c.scratch, c.off_cnt, c.off_rowcnt,
-                            c.off_hist, c.off_cursor)) != cudaSuccess) return e;
-    if ((e = launch_chained(scan_kernel, dim3(1), dim3(1024), st, c.blob, c.scratch, c.off_rowcnt, c.off_hist,
-                            c.off_cursor)) != cudaSuccess) return e;
-    if ((e = launch_chained(classify_kernel<1>, dim3(blocks), dim3(256), st, c.blob, c.scratch, c.off_cnt, c.off_rowcnt,
-                            c.off_hist, c.off_cursor)) != cudaSuccess) return e;
+    if ((e = launch_chained(classify_kernel, dim3(blocks), dim3(256), st, c.blob, c.scratch, c.off_cnt, c.off_items)) !=
+        cudaSuccess) return e;
+    if ((e = launch_chained(order_kernel, dim3((c.prows + 1023) / 1024), dim3(1024), st, c.blob, c.scratch, c.off_items)) !=
+        cudaSuccess)
+      return e;
   }
   return cudaGetLastError();
 }

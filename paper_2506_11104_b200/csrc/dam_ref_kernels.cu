@@ -146,6 +146,7 @@ __global__ void attn_ref_kernel(const unsigned char* blob, const T* __restrict__
     float m = -CUDART_INF_F, l = 0.f;
     for (uint32_t t = t0; t < t1; ++t) {
       const uint32_t e = __ldg(tiles + t);
+      if ((e >> 28) == 0u) continue;                    // padding behind the row's entries
       const int kb = (int)(e & 0x0FFFFFFFu);
       const uint4 bits = dam_apply_bits(hb, e >> 28, i, kb, causal);
       const uint32_t w4[4] = {bits.x, bits.y, bits.z, bits.w};

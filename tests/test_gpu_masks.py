@@ -130,8 +130,14 @@ def _build_and_check(w, qblocks=None, gather=False):
         row = int(it["head"]) * tq + int(sq["first_qblock"]) + int(it["qb0"])
         assert int(it["qb0"]) % 2 == 0 and int(it["tok0"]) == int(sq["tok_start"]) and int(it["S"]) == int(sq["S"])
         assert has2 == (int(it["qb0"]) + 1 < int(sq["nq"]))
-        assert int(it["a0"]) == int(mb1.tile_ptr[row]) and int(it["a1"]) == int(mb1.tile_ptr[row + 1])
-        assert int(it["b1"]) == int(mb1.tile_ptr[row + 1 + has2])
+        # the pair's entries: block 2p from tile_ptr[row], block 2p+1 directly behind, then zero padding
+        qb0 = int(it["qb0"])
+        nA, nB = len(mb1.row_entries(b, int(it["head"]), qb0)), (len(mb1.row_entries(b, int(it["head"]), qb0 + 1)) if has2 else 0)
+        assert int(it["a0"]) == int(mb1.tile_ptr[row]) and int(it["a1"]) == int(it["a0"]) + nA
+        assert int(it["b1"]) == int(it["a1"]) + nB and int(it["b1"]) <= int(mb1.tile_ptr[row + 1 + has2])
+        if has2:
+            assert int(it["a1"]) == int(mb1.tile_ptr[row + 1])
+        assert not mb1.tiles[int(it["b1"]): int(mb1.tile_ptr[row + 1 + has2])].any()
         seen.add((int(it["head"]), b, int(it["qb0"])))
         keys.append(int(it["b1"]) - int(it["a0"]))
     assert len(seen) == int(mb1.hdr["prows"]) == len(mb1.items)
