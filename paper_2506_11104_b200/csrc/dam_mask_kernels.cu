@@ -331,7 +331,8 @@ __device__ __forceinline__ uint32_t classify_band(const HeadView& v, int qb, int
   return (whole && n == 2 * DAM_TILE - 1) ? DAM_KIND_FULL : DAM_KIND_PARTIAL;
 }
 
-__global__ void classify_kernel(unsigned char* blob, unsigned char* scratch, uint64_t off_cnt, uint64_t off_items) {
+__global__ void classify_kernel(unsigned char* blob, unsigned char* scratch, uint64_t off_cnt, uint64_t off_items,
+                                uint64_t off_keys) {
   dam_chain_prologue();
   DamHeader* H = reinterpret_cast<DamHeader*>(blob);
   const int lane = threadIdx.x & 31;
@@ -414,12 +415,15 @@ __global__ void classify_kernel(unsigned char* blob, unsigned char* scratch, uin
   // zero entries up to the next pair
   for (uint32_t t = base + lane; t < pair_end; t += 32) tiles[t] = 0u;
   if (lane == 0) {
-    // the work item, at the pair's own index for now: the ordering kernel moves it to its place in the work list
+    // the work item and its key (listed tiles): the ordering kernel moves the item to its place in the work list
     DamItem it;
     it.head = h; it.tok0 = sq.tok_start; it.qb0 = qb0; it.S = sq.S;
     it.a0 = pair_begin; it.a1 = a1; it.b1 = base;
     it.seq_hasB = (uint32_t)b | (nblk == 2 ? 0x80000000u : 0u);
-    reinterpret_cast<DamItem*>(scratch + off_items)[prow] = it;
+    // index (pair, head): the order the pairs keep inside a bucket of the work list
+    const size_t at = (size_t)gp * H->num_q_heads + h;
+    reinterpret_cast<DamItem*>(scratch + off_items)[at] = it;
+    reinterpret_cast<uint32_t*>(scratch + off_keys)[at] = (uint32_t)min(pair_total, DAM_HIST - 1);
     atomicAdd(&s_mask_tiles, (unsigned long long)mask_tiles);
     atomicAdd(&s_total, (uint32_t)pair_total);
     atomicAdd(&s_full, (uint32_t)nfull);
@@ -465,16 +469,17 @@ __device__ uint32_t block_excl_scan(uint32_t x, uint32_t* total, uint32_t* sm /*
 }
 
 __global__ void __launch_bounds__(1024)
-order_kernel(unsigned char* blob, unsigned char* scratch, uint64_t off_items) {
+order_kernel(unsigned char* blob, unsigned char* scratch, uint64_t off_items, uint64_t off_keys) {
   dam_chain_prologue();
   DamHeader* H = reinterpret_cast<DamHeader*>(blob);
   __shared__ uint32_t sm[32];
   __shared__ uint32_t tot;
   __shared__ uint32_t start[DAM_HIST];      // pairs per key, then the first place of the key's bucket
   __shared__ uint32_t before[DAM_HIST];     // pairs per key that precede this block's share, then the running cursor
-  const uint4* src = reinterpret_cast<const uint4*>(scratch + off_items);
+  const uint4* src = reinterpret_cast<const uint4*>(scratch + off_items);      // items in (pair, head) order
+  const uint32_t* keys = reinterpret_cast<const uint32_t*>(scratch + off_keys);
   uint4* dst = reinterpret_cast<uint4*>(blob + H->off_work);
-  const int prows = H->prows, total_pairs = H->total_pairs, Hq = H->num_q_heads;
+  const int prows = H->prows;
   for (int k = threadIdx.x; k < DAM_HIST; k += blockDim.x) { start[k] = 0u; before[k] = 0u; }
   __syncthreads();
   // Every block places blockDim.x pairs and needs nothing from the other blocks: it counts all pairs per key
@@ -482,21 +487,18 @@ order_kernel(unsigned char* blob, unsigned char* scratch, uint64_t off_items) {
   // heads of one KV head at the same pair of query blocks list the same kv tiles, and neighbours in the work
   // list run at the same time on different SMs, so the second to fourth find the K and V tiles in L2.  An item
   // is two 16-byte words: head, tok0, qb0, S | a0, a1, b1, seq_hasB; its key is the number of listed tiles.
-  const int lane = threadIdx.x & 31;
   const int my_begin = blockIdx.x * (int)blockDim.x;
-  auto item_of = [&](int idx) -> size_t { return 2 * (size_t)((idx % Hq) * total_pairs + idx / Hq); };
-  auto key_of = [](const uint4& v) -> uint32_t { return min(v.z - v.x, (uint32_t)(DAM_HIST - 1)); };
-  // lanes of a warp that share a key count together (most pairs of a layer share one key)
+  // (in this order the lanes of a warp are the heads of one pair: their keys mostly differ, so plain shared-memory
+  // atomics do not collide inside an instruction)
   auto count = [&](uint32_t* hist, uint32_t key) {
-    const uint32_t same = __match_any_sync(0xFFFFFFFFu, key);
-    if (key != 0xFFFFFFFFu && lane == __ffs(same) - 1) atomicAdd(&hist[key], (uint32_t)__popc(same));
+    if (key != 0xFFFFFFFFu) atomicAdd(&hist[key], 1u);
   };
   for (int i0 = 0; i0 < prows; i0 += 4 * (int)blockDim.x) {
     uint32_t k[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const int idx = i0 + j * (int)blockDim.x + (int)threadIdx.x;
-      k[j] = idx < prows ? key_of(src[item_of(idx) + 1]) : 0xFFFFFFFFu;
+      k[j] = idx < prows ? keys[idx] : 0xFFFFFFFFu;
     }
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
@@ -520,14 +522,9 @@ order_kernel(unsigned char* blob, unsigned char* scratch, uint64_t off_items) {
     const int idx = my_begin + (int)threadIdx.x;
     uint4 u = make_uint4(0u, 0u, 0u, 0u), v = u;
     uint32_t key = 0xFFFFFFFFu;
-    if (idx < prows) { u = src[item_of(idx)]; v = src[item_of(idx) + 1]; key = key_of(v); }
-    const uint32_t same = __match_any_sync(0xFFFFFFFFu, key);
-    const int leader = __ffs(same) - 1;
-    uint32_t base = 0u;
-    if (key != 0xFFFFFFFFu && lane == leader) base = start[key] + atomicAdd(&before[key], (uint32_t)__popc(same));
-    base = __shfl_sync(0xFFFFFFFFu, base, leader);
+    if (idx < prows) { u = src[2 * (size_t)idx]; v = src[2 * (size_t)idx + 1]; key = keys[idx]; }
     if (key != 0xFFFFFFFFu) {
-      const uint32_t pos = base + (uint32_t)__popc(same & ((1u << lane) - 1u));
+      const uint32_t pos = start[key] + atomicAdd(&before[key], 1u);
       dst[2 * (size_t)pos] = u; dst[2 * (size_t)pos + 1] = v;
     }
   }
@@ -827,10 +824,10 @@ cudaError_t dam_launch_rule(const DamBuildCtx& c, cudaStream_t st) {
   }
   if (c.rows > 0) {
     int blocks = (c.prows + 7) / 8;
-    if ((e = launch_chained(classify_kernel, dim3(blocks), dim3(256), st, c.blob, c.scratch, c.off_cnt, c.off_items)) !=
-        cudaSuccess) return e;
-    if ((e = launch_chained(order_kernel, dim3((c.prows + 1023) / 1024), dim3(1024), st, c.blob, c.scratch, c.off_items)) !=
-        cudaSuccess)
+    if ((e = launch_chained(classify_kernel, dim3(blocks), dim3(256), st, c.blob, c.scratch, c.off_cnt, c.off_items,
+                            c.off_rowcnt)) != cudaSuccess) return e;
+    if ((e = launch_chained(order_kernel, dim3((c.prows + 1023) / 1024), dim3(1024), st, c.blob, c.scratch, c.off_items,
+                            c.off_rowcnt)) != cudaSuccess)
       return e;
   }
   return cudaGetLastError();
