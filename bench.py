@@ -347,7 +347,7 @@ def main():
     peak = pk["bf16_sustained"] or pk["bf16"]
     roof = {"bound": "tensor", "kernel": "attn_sm100_kernel", "achieved": round(attn_tflops, 2), "peak": peak,
             "peak_kind": f"sustained cuBLAS bf16, {pk['which']}", "unit": "TFLOP/s", "frac": round(attn_tflops / peak, 4),
-            "frac_of_burst": round(attn_tflops / pk["bf16"], 4), "traffic": measured_traffic("attn_sm100_kernel", cfg),
+            "frac_of_burst": round(attn_tflops / pk["bf16"], 4), "traffic": None if args.no_gather else measured_traffic("attn_sm100_kernel", cfg),   # captured with gathered tiles
             "avg_launch_ms": round(attn_ms, 4)}
 
     out = {"metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
