@@ -57,10 +57,12 @@ struct SmemLayout {
   static constexpr int n_bars = 2 + 2 * kSlots + 10;
   static constexpr int sched_items = bars + 8 * n_bars;     // int[2]: work-list positions handed to the consumers
   static constexpr int step_desc = sched_items + 8;         // u32[16]: what the producer found at each step (kStep*)
-  static constexpr int tmem_slot = step_desc + 64;
+  static constexpr int item_rec = (step_desc + 64 + 15) & ~15;   // ItemRec[2] (16-byte aligned): what the softmax warps need to start an item
+  static constexpr int tmem_slot = item_rec + 2 * 96;
   static constexpr int abort_flag = tmem_slot + 4;
   static constexpr int total = abort_flag + 4;
 };
+static_assert(SmemLayout::item_rec % 16 == 0 && SmemLayout::bars % 8 == 0, "shared-memory records must be aligned");
 constexpr int kSmemBytes = SmemLayout::total + 1024;   // + slack for the 1024-byte alignment
 
 #ifdef DAM_PROFILE
@@ -72,6 +74,16 @@ constexpr int kSmemBytes = SmemLayout::total + 1024;   // + slack for the 1024-b
 #define PROF_LAP(k)
 #define PROF_FLUSH(base, n)
 #endif
+
+// What the producer hands to the softmax warps with every work-list position: the item record, the first tile
+// entry of each stream and the head's bit-set pointers, so that their set-up reads shared memory instead of
+// walking item -> sequence record -> tile list in global memory.
+struct ItemRec {
+  uint4 u, v;               // the two words of the DamItem
+  uint32_t eA, eB, pad0, pad1;
+  DamHeadBits hb;
+};
+static_assert(sizeof(ItemRec) == 96, "ItemRec must be 96 bytes");
 
 struct AttnParams {
   unsigned long long* prof;
@@ -104,14 +116,16 @@ struct Item {
   uint32_t a0, a1, b0, b1;      // tile list [a0, a1) of block 2p, [b0, b1) of block 2p+1
 };
 
-__device__ __forceinline__ Item load_item(const unsigned char* blob, const DamHeader* H, int w) {
-  const uint4* src = reinterpret_cast<const uint4*>(blob + H->off_work) + 2 * (size_t)w;
-  const uint4 u = __ldg(src), v = __ldg(src + 1);
+__device__ __forceinline__ Item item_from_words(const uint4& u, const uint4& v) {
   Item it;
   it.head = (int)u.x; it.tok0 = (int)u.y; it.qb0 = (int)u.z; it.S = (int)u.w;
   it.a0 = v.x; it.a1 = v.y; it.b0 = v.y; it.b1 = v.z;
   it.hasB = (int)(v.w >> 31); it.seq = (int)(v.w & 0x7FFFFFFFu);
   return it;
+}
+__device__ __forceinline__ Item load_item(const unsigned char* blob, const DamHeader* H, int w) {
+  const uint4* src = reinterpret_cast<const uint4*>(blob + H->off_work) + 2 * (size_t)w;
+  return item_from_words(__ldg(src), __ldg(src + 1));
 }
 
 // Merge of the two ascending tile lists: every step is one kv tile with the kinds it has in A and in B.
@@ -293,6 +307,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   const uint32_t bSchedFull = bOFinal + 16, bSchedEmpty = bSchedFull + 16;
   volatile int* sched_items = reinterpret_cast<volatile int*>(smem + SmemLayout::sched_items);
   volatile uint32_t* step_desc = reinterpret_cast<volatile uint32_t*>(smem + SmemLayout::step_desc);
+  ItemRec* item_rec = reinterpret_cast<ItemRec*>(smem + SmemLayout::item_rec);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + SmemLayout::tmem_slot);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + SmemLayout::abort_flag);
 
@@ -364,9 +379,22 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (w >= nitems) w = -1;
         Item it;
         bool skip = false;
+        long long gtile0 = 0;
         if (w >= 0) {
-          it = load_item(blob, H, w);
+          const uint4* src = reinterpret_cast<const uint4*>(blob + H->off_work) + 2 * (size_t)w;
+          const uint4 u = __ldg(src), v = __ldg(src + 1);
+          it = item_from_words(u, v);
           skip = it.a0 == it.b1 || !item_active(it);         // no tile in either list, or outside the row range
+          ItemRec& rec = item_rec[slot];
+          rec.u = u; rec.v = v;
+          if (!skip) {
+            const DamSeq sq = reinterpret_cast<const DamSeq*>(blob + H->off_seq)[it.seq];
+            rec.eA = it.a0 < it.a1 ? __ldg(tiles + it.a0) : 0u;
+            rec.eB = it.b0 < it.b1 ? __ldg(tiles + it.b0) : 0u;
+            rec.hb = dam_head_bits(blob, H, sq, it.head);
+            // gathered-column tiles of this (sequence, head): K tile at rows (2T) * 128, V tile at (2T + 1) * 128
+            gtile0 = (long long)sq.gath_off + (long long)it.head * sq.nL;
+          }
         }
         // the entry tells the MMA thread whether the item has steps at all, so that it never reads the work list
         sched_items[slot] = w < 0 ? w : (w | (skip ? kSchedNoSteps : 0));
@@ -384,12 +412,6 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
         ++ic;
         const int kvh = it.head / prm.group;
-        // gathered-column tiles of this (sequence, head): K tile at rows (2T) * 128, V tile at (2T + 1) * 128
-        long long gtile0 = 0;
-        if (H->flags & DAM_FLAG_GATHER) {
-          const DamSeq* sqp = reinterpret_cast<const DamSeq*>(blob + H->off_seq) + it.seq;
-          gtile0 = (long long)sqp->gath_off + (long long)it.head * sqp->nL;
-        }
         Walker wk; wk.init(tiles, it);
         int kb; uint32_t kA, kB;
         while (ok && wk.next(kb, kA, kB)) {
@@ -530,11 +552,18 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     PROF_DECL(8)
     for (uint32_t n = 0; ok; ++n) {
       const int ws = next_item_consumer(n, false);
+      if (ws < 0) {
+        __syncwarp();
+        if (lane == 0 && ws != -2) mbar_arrive(bSchedEmpty + 8 * (n & 1u));
+        ok = (ws == -1);
+        break;
+      }
+      const ItemRec& rec = item_rec[n & 1u];
+      const Item it = item_from_words(rec.u, rec.v);
+      const DamHeadBits hb = rec.hb;                         // (not meaningful for an item without steps)
+      const uint32_t e_first = X ? rec.eB : rec.eA;
       __syncwarp();
-      if (lane == 0 && ws != -2) mbar_arrive(bSchedEmpty + 8 * (n & 1u));   // the whole warp has read the entry
-      if (ws < 0) { ok = (ws == -1); break; }
-      const int w = ws & ~kSchedNoSteps;
-      const Item it = load_item(blob, H, w);
+      if (lane == 0) mbar_arrive(bSchedEmpty + 8 * (n & 1u));               // the whole warp has read the record
       if ((X == 1 && !it.hasB) || !item_active(it)) continue;
       const int qb = it.qb0 + X;
       const uint32_t t0 = X ? it.b0 : it.a0, t1 = X ? it.b1 : it.a1;
@@ -551,8 +580,6 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
         continue;
       }
-      const DamSeq sq = reinterpret_cast<const DamSeq*>(blob + H->off_seq)[it.seq];
-      const DamHeadBits hb = dam_head_bits(blob, H, sq, it.head);
       float m_ref = -CUDART_INF_F;   // reference max (scaled, log2 domain) that P and O are expressed against
       float l = 0.f;
       // the mask words of a tile come from global memory: they are fetched one tile ahead
@@ -569,7 +596,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       };
       uint32_t e_next = t0 + 1 < t1 ? __ldg(tiles + t0 + 1) : 0u;
       bool need_nx = false;
-      uint4 bits_nx = tile_bits(__ldg(tiles + t0), need_nx);
+      uint4 bits_nx = tile_bits(e_first, need_nx);
       for (uint32_t t = t0; t < t1; ++t) {
         const bool need_mask = need_nx;
         const uint4 bits = bits_nx;
