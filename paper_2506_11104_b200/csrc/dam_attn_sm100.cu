@@ -7,7 +7,8 @@
 //   warp 0      TMA producer: both Q tiles once per item, then K and V of every kv tile in the union of
 //               the two tile lists ("step") into a ring of 32 KB shared-memory slots (128-byte swizzle); for
 //               every step it leaves a descriptor word in shared memory (which streams have a tile in it, whether
-//               it is a stream's last, whether the item goes on);
+//               it is a stream's last, whether the item goes on), and for every item a record for the softmax
+//               warps (item, first tile entries, the head's bit-set pointers);
 //   warp 1      MMA issuer (one elected thread), driven by those descriptors alone (it reads no global memory):
 //               S_X = Q_X K^T into the stream's TMEM columns, then O_X += P_X V with P_X read from TMEM (it
 //               overwrites the first half of S_X); the two streams are interleaved so that one stream's softmax
