@@ -237,6 +237,55 @@ def test_mask_tile_count_is_independent_of_gathering():
     assert b["tiles"] < a["tiles"]
 
 
+@pytest.mark.parametrize("lengths,pcl,gather", [
+    ([1], 64, False), ([127, 128, 129], 128, True), ([700, 260, 5], 96, True), ([2100], 512, True),
+    ([2100], 512, False), ([640, 64], 1024, True),
+])
+def test_tile_lists_sit_at_fixed_places(lengths, pcl, gather):
+    """Every pair of adjacent query blocks owns the range of tiles[] that its rows' upper bounds add up to: the
+    ranges follow from the shapes alone, tile the whole capacity, and hold the two rows' entries back to back
+    followed by zero entries only."""
+    Hq, Hkv, d = 4, 2, 128
+    w = synth.small_case(0, Hq, Hkv, d, pcl, seed=13, dtype=torch.bfloat16, lengths=lengths)
+    shape = B.make_shape(w.cu_seqlens, Hq, Hkv, d, torch.bfloat16, DEV)
+    rule = B.make_rule(w.pcl_max, w.tau, w.mu, w.lam, w.eps, gather_columns=gather)
+    blob, _ = B.dam_build_masks(w.Q.to(DEV), w.K.to(DEV), shape, rule)
+    assert B.dam_poll_status(blob) == 0
+    mb = B.MaskBlob(blob)
+    hdr, tq = mb.hdr, int(mb.hdr["total_qblocks"])
+
+    def bound(qb, nL, L):                      # upper bound on the listed tiles of a query block (host restatement)
+        gf = (2 * L - 1 + 127) // 128
+        if gather and L > 0 and qb >= gf:
+            return nL + min(qb + 1, nL + 1)
+        return min(qb + 1, 2 * nL + 1)
+
+    cap_head = int(hdr["head_tile_cap"])
+    assert int(hdr["tile_capacity"]) == Hq * cap_head == int(mb.tile_ptr[-1])
+    assert int(hdr["bytes_used"]) == int(hdr["off_tiles"]) + 4 * Hq * cap_head
+    listed = 0
+    for h in range(Hq):
+        at = h * cap_head
+        for b, sq in enumerate(mb.seqs):
+            nq, nL, L = int(sq["nq"]), int(sq["nL"]), int(sq["L"])
+            assert at == h * cap_head + int(sq["tile_base"])
+            for qb0 in range(0, nq, 2):
+                row = h * tq + int(sq["first_qblock"]) + qb0
+                nblk = 2 if qb0 + 1 < nq else 1
+                end = at + sum(bound(qb0 + x, nL, L) for x in range(nblk))
+                assert int(mb.tile_ptr[row]) == at
+                nA = len(mb.row_entries(b, h, qb0))
+                nB = len(mb.row_entries(b, h, qb0 + 1)) if nblk == 2 else 0
+                if nblk == 2:
+                    assert int(mb.tile_ptr[row + 1]) == at + nA
+                seg = mb.tiles[at:end]
+                assert ((seg[:nA + nB] >> 28) != 0).all() and not seg[nA + nB:].any()
+                listed += nA + nB
+                at = end
+        assert at == (h + 1) * cap_head
+    assert listed == int(hdr["total_tiles"])
+
+
 def test_multi_sample_capture_masks_bit_exact():
     """Three batches of samples of mixed lengths are accumulated on the GPU; the masks built from the averaged
     maps equal, bit for bit, the oracle's masks from its own fp32 average of the same per-sample score tensors."""
