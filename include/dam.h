@@ -20,8 +20,8 @@
  *     (exceptions are stated at the function);
  *   - every function returns a dam_status_t; argument errors are detected on the host before
  *     anything is enqueued and nothing is written in that case;
- *   - problems only the device can see (a tile list that would overflow the blob, a bounded wait
- *     that expired) are recorded in the status word at the start of the mask blob / attention
+ *   - problems only the device can see (a bounded wait that expired, an attention scratch that is too
+ *     small for the blob it is used with) are recorded in the status word at the start of the mask blob / attention
  *     scratch and are read back with dam_poll_status;
  *   - layouts: Q, O are [total_tokens, num_q_heads, head_dim]; K, V are
  *     [total_tokens, num_kv_heads, head_dim]; sequences are packed back to back (token-major) and
@@ -266,7 +266,8 @@ dam_status_t dam_decode_attention(const void* q, const void* K, const void* V, c
 /*
  * Counts taken from a mask blob (DEVICE): out[0] = listed tiles (what the attention kernel executes),
  * out[1] = of those, fully active ones, out[2] = total causal tiles of the shape (for densities),
- * out[3] = bytes of the blob in use, out[4] = 128 x 128 tiles of the masks themselves that hold an
+ * out[3] = bytes of the blob in use (the tile lists have a fixed place per row, sized by the row's upper
+ * bound, so this follows from the shapes; out[0] says how many entries are real), out[4] = 128 x 128 tiles of the masks themselves that hold an
  * active cell (equals out[0] unless gathered-column tiles are listed). `out` is HOST memory
  * (5 x uint64). Synchronises `stream`. The paper reports no such counts; they feed the density and
  * active-FLOP figures of the benchmark.
