@@ -5,7 +5,7 @@ One step = one layer of the workload: `dam_build_masks` followed by `dam_sparse_
 the C ABI.  Default workload: the 32-layer stack of Llama-3-8B-shaped layers at 32768 tokens, PCL 2048
 (each step takes the next layer, its own seed and planted-pattern mix), inputs resident in HBM.
 
-Prints ONE JSON line (see README for the fields).  `--impl reference` times the CPU oracle
+Prints ONE JSON line (metric, value, roofline, cpu_baseline, e2e, clocks, ...).  `--impl reference` times the CPU oracle
 on a bounded sample of the same workload instead.
 """
 from __future__ import annotations
