@@ -367,7 +367,7 @@ def main():
                               {"layer": elem["layer"], "element_density": elem["density"],
                                "tflops": round(elem["flops"] / (total_ms_max / args.steps * 1e-3) / 1e12, 3),
                                "flops": "4*d per active cell of the masks (one layer, at the mean layer time)"}),
-           "roofline": roof, "clocks": clocks, "gpu_launches": (9 if not args.no_gather else 8) * args.steps}
+           "roofline": roof, "clocks": clocks, "gpu_launches": (8 if not args.no_gather else 7) * args.steps}   # init, score, counts, match, classify, order, [gather], attention
 
     if rank == 0 and not args.no_dense:
         # the build's own dense causal attention at the same length (all tiles listed as fully active)
