@@ -349,6 +349,9 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  // launched as a programmatic dependent of the kernel that gathers the matched columns: everything above ran
+  // under that kernel's tail; its tiles (and the cleared work counter) are visible from here on
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -746,6 +749,7 @@ __global__ void __launch_bounds__(128)
 gather_columns_kernel(const unsigned char* __restrict__ blob, const __nv_bfloat16* __restrict__ K,
                       const __nv_bfloat16* __restrict__ V, int Hq, int group, int64_t kst, int64_t ksh, int64_t vst,
                       int64_t vsh, unsigned char* scratch, unsigned long long scratch_bytes) {
+  asm volatile("griddepcontrol.launch_dependents;");     // the attention kernel behind this one may start its prologue
   const DamHeader* H = reinterpret_cast<const DamHeader*>(blob);
   if (!(H->flags & DAM_FLAG_GATHER)) return;
   if (H->attn_scratch_bytes > scratch_bytes) {
@@ -902,7 +906,12 @@ cudaError_t dam_launch_attn_sm100(const void* Q, const void* K, const void* V, c
   p.o_stride_tok = s->o_stride_tok; p.o_stride_head = s->o_stride_head;
   p.scale_log2 = scale * 1.4426950408889634f;
   const int grid = pairs < sm_count ? pairs : sm_count;
-  if (ranges) attn_sm100_kernel<true><<<grid, kThreads, kSmemBytes, st>>>(tq, tk, tv, to, tg, p);
-  else attn_sm100_kernel<false><<<grid, kThreads, kSmemBytes, st>>>(tq, tk, tv, to, tg, p);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  if (ranges) return cudaLaunchKernelEx(&cfg, attn_sm100_kernel<true>, tq, tk, tv, to, tg, p);
+  return cudaLaunchKernelEx(&cfg, attn_sm100_kernel<false>, tq, tk, tv, to, tg, p);
 }
