@@ -365,52 +365,87 @@ __global__ void classify_kernel(unsigned char* blob, unsigned char* scratch, uin
   const uint32_t pair_end = (uint32_t)(head_base + dam_row_tile_prefix(qb0 + nblk, sq.nL, sq.L, gflag));
   uint32_t base = pair_begin, a1 = pair_begin;
   int pair_total = 0, nfull = 0, mask_tiles = 0;
-  for (int x = 0; x < nblk; ++x) {
-    const int gqb = gqb0 + x;
-    const int row = h * H->total_qblocks + gqb;
-    const int qb = gqb - sq.first_qblock;
-    // candidates, ascending: [0, min(qb, nL-1)] then [max(that + 1, qb - nL), qb].  From row 2L - 1 on
-    // (gathered columns enabled) the first range is replaced by the gathered tiles and the second range
-    // is classified on the matched diagonals alone.
-    const bool gathered = gflag && sq.L > 0 && qb >= dam_gather_first_qblock(sq.L);
-    const int nV = gathered ? v.prefV[sq.W] : 0;
-    const int n1 = gathered ? (nV + DAM_TILE - 1) / DAM_TILE : min(qb, sq.nL - 1) + 1;
-    const int lo2 = gathered ? max(0, qb - sq.nL) : max(n1, qb - sq.nL);
-    const int n2 = max(0, qb - lo2 + 1);
-    // tiles of the mask itself (128 x 128 grid) with an active cell are counted in the same sweep (their loads
-    // overlap the classification's): they equal the listed tiles unless the row is served by gathered tiles
-    const int m1 = min(qb, sq.nL - 1) + 1, l2 = max(m1, qb - sq.nL), m2 = max(0, qb - l2 + 1);
-    const int ncand = n1 + n2, nmask = gathered ? m1 + m2 : 0;
-    int total = 0, nat = 0;
-    for (int c0 = 0; c0 < max(ncand, nmask); c0 += 32) {
-      int idx = c0 + lane;
-      uint32_t kind = 0, entry = 0;
-      if (idx < ncand) {
-        if (gathered && idx < n1) {
-          kind = DAM_KIND_GATHERED;
-          entry = (uint32_t)idx | ((uint32_t)(min(DAM_TILE, nV - idx * DAM_TILE) - 1) << 16) | (kind << 28);
-        } else {
-          const int kb = idx < n1 ? idx : lo2 + (idx - n1);
-          kind = gathered ? classify_band(v, qb, kb) : classify_tile(v, qb, kb);
-          entry = (uint32_t)kb | (kind << 28);
-        }
+  // Per query block: candidates, ascending: [0, min(qb, nL-1)] then [max(that + 1, qb - nL), qb].  From row 2L - 1
+  // on (gathered columns enabled) the first range is replaced by the gathered tiles and the second range is
+  // classified on the matched diagonals alone.  The tiles of the mask itself (128 x 128 grid) with an active cell
+  // are counted in the same sweep: they equal the listed tiles unless the row is served by gathered tiles.
+  struct BlockPlan { int qb, gathered, n1, lo2, ncand, m1, l2, nmask; };
+  const int nV = (gflag && sq.L > 0) ? v.prefV[sq.W] : 0;        // matched columns of the head
+  BlockPlan plan[2];
+#pragma unroll
+  for (int x = 0; x < 2; ++x) {
+    BlockPlan& p = plan[x];
+    p.qb = qb0 + x;
+    p.gathered = gflag && sq.L > 0 && p.qb >= dam_gather_first_qblock(sq.L);
+    p.n1 = p.gathered ? (nV + DAM_TILE - 1) / DAM_TILE : min(p.qb, sq.nL - 1) + 1;
+    p.lo2 = p.gathered ? max(0, p.qb - sq.nL) : max(p.n1, p.qb - sq.nL);
+    p.ncand = x < nblk ? p.n1 + max(0, p.qb - p.lo2 + 1) : 0;
+    p.m1 = min(p.qb, sq.nL - 1) + 1;
+    p.l2 = max(p.m1, p.qb - sq.nL);
+    p.nmask = (x < nblk && p.gathered) ? p.m1 + max(0, p.qb - p.l2 + 1) : 0;
+  }
+  // one candidate per lane: list entry (kind 0: not listed) and whether the mask tile has an active cell
+  auto eval = [&](const BlockPlan& p, int idx, uint32_t& kind, uint32_t& entry, bool& act) {
+    kind = 0u; entry = 0u;
+    if (idx < p.ncand) {
+      if (p.gathered && idx < p.n1) {
+        kind = DAM_KIND_GATHERED;
+        entry = (uint32_t)idx | ((uint32_t)(min(DAM_TILE, nV - idx * DAM_TILE) - 1) << 16) | (kind << 28);
+      } else {
+        const int kb = idx < p.n1 ? idx : p.lo2 + (idx - p.n1);
+        kind = p.gathered ? classify_band(v, p.qb, kb) : classify_tile(v, p.qb, kb);
+        entry = (uint32_t)kb | (kind << 28);
       }
-      const bool act = idx < nmask && classify_tile(v, qb, idx < m1 ? idx : l2 + (idx - m1)) != 0u;
-      uint32_t m = __ballot_sync(0xFFFFFFFFu, kind != 0);
-      if (kind) {
-        int rank = __popc(m & ((1u << lane) - 1u));
-        if (base + total + rank < pair_end) tiles[base + total + rank] = entry;     // always true: the range is the bound
-      }
-      nfull += __popc(__ballot_sync(0xFFFFFFFFu, kind == DAM_KIND_FULL || (kind == DAM_KIND_GATHERED && ((entry >> 16) & 0xFFu) == DAM_TILE - 1)));
-      total += __popc(m);
-      nat += __popc(__ballot_sync(0xFFFFFFFFu, act));
     }
-    if (lane == 0) tile_ptr[row] = base;
+    act = idx < p.nmask && classify_tile(v, p.qb, idx < p.m1 ? idx : p.l2 + (idx - p.m1)) != 0u;
+  };
+  int total = 0, nat = 0;
+  auto consume = [&](uint32_t kind, uint32_t entry, bool act) {
+    const uint32_t m = __ballot_sync(0xFFFFFFFFu, kind != 0);
+    if (kind) {
+      const int rank = __popc(m & ((1u << lane) - 1u));
+      if (base + total + rank < pair_end) tiles[base + total + rank] = entry;     // always true: the range is the bound
+    }
+    nfull += __popc(__ballot_sync(0xFFFFFFFFu, kind == DAM_KIND_FULL || (kind == DAM_KIND_GATHERED && ((entry >> 16) & 0xFFu) == DAM_TILE - 1)));
+    total += __popc(m);
+    nat += __popc(__ballot_sync(0xFFFFFFFFu, act));
+  };
+  auto finish_block = [&](int x) {
+    if (lane == 0) tile_ptr[h * H->total_qblocks + gqb0 + x] = base;
     base += total;
     if (x == 0) a1 = base;
     pair_total += total;
-    if (!gathered) nat = total;
-    mask_tiles += nat;
+    mask_tiles += plan[x].gathered ? nat : total;
+    total = 0; nat = 0;
+  };
+  const int span0 = max(plan[0].ncand, plan[0].nmask), span1 = max(plan[1].ncand, plan[1].nmask);
+  if (span0 <= 64 && span1 <= 64) {
+    // the usual sizes: all candidates of both blocks are looked up before any is written, so that their loads
+    // (prefix counts, bit words, tile counts) are in flight together
+    uint32_t k[4], e[4];
+    bool a[4];
+    eval(plan[0], lane, k[0], e[0], a[0]);
+    eval(plan[0], 32 + lane, k[1], e[1], a[1]);
+    eval(plan[1], lane, k[2], e[2], a[2]);
+    eval(plan[1], 32 + lane, k[3], e[3], a[3]);
+    consume(k[0], e[0], a[0]);
+    if (span0 > 32) consume(k[1], e[1], a[1]);
+    finish_block(0);
+    if (nblk == 2) {
+      consume(k[2], e[2], a[2]);
+      if (span1 > 32) consume(k[3], e[3], a[3]);
+      finish_block(1);
+    }
+  } else {
+    for (int x = 0; x < nblk; ++x) {
+      for (int c0 = 0; c0 < max(plan[x].ncand, plan[x].nmask); c0 += 32) {
+        uint32_t kind, entry;
+        bool act;
+        eval(plan[x], c0 + lane, kind, entry, act);
+        consume(kind, entry, act);
+      }
+      finish_block(x);
+    }
   }
   // zero entries up to the next pair
   for (uint32_t t = base + lane; t < pair_end; t += 32) tiles[t] = 0u;
