@@ -330,8 +330,7 @@ def main():
     # element-level density of one layer's masks (host arithmetic on the pattern bits: the paper's O(s L) figure)
     elem = None
     if rank == 0:
-        mbh = B.MaskBlob(mask)
-        nnz = sum(mbh.active_elements(b, h) for b in range(len(shape.lengths)) for h in range(w0.num_q_heads))
+        nnz = int(B.dam_mask_stats(mask, shape, active_elements=True)["active_elements"].sum().item())
         causal_elems = sum(S * (S + 1) // 2 for S in shape.lengths) * w0.num_q_heads
         elem = {"layer": int(l), "density": round(nnz / causal_elems, 5), "flops": 4.0 * w0.head_dim * nnz}
     step_tiles = [per_layer_stats[(args.warmup + i) % n_layers]["tiles"] for i in range(args.steps)]

@@ -228,8 +228,10 @@ dam_status_t dam_capture_average(const float* A, const int32_t* C, int32_t pcl_m
  * Chunked prefill: dam_sparse_attention restricted, per sequence b, to the query rows
  * [row_ranges[2b], row_ranges[2b+1]) (indices inside the sequence). The blob is the one built for the full
  * lengths (stage 1 reads only the first L_b rows of Q and K, so it can be built as soon as the window has been
- * computed); K and V must hold the keys 0 .. end-1 of every sequence; rows outside the ranges of O and LSE are
- * neither read nor written. The paper has no counterpart (its Sec. 4.3 extends the mask to "longer sequences"
+ * computed); K and V must hold the keys 0 .. end-1 of every sequence, and the rows from `end` up to the next
+ * multiple of 128 (as far as the packed buffers reach) must hold finite values: they share a 128-key tile with
+ * the last keys, take probability zero, and zero times a NaN or an infinity would still reach the output;
+ * rows outside the ranges of O and LSE are neither read nor written. The paper has no counterpart (its Sec. 4.3 extends the mask to "longer sequences"
  * without saying how they arrive); the arithmetic per row is exactly that of dam_sparse_attention.
  * Work is dealt in pairs of 128-row query blocks, so every begin must be a multiple of 256 and every end a
  * multiple of 256 or the sequence length (INVALID_ARGUMENT otherwise); an empty range skips the sequence.
@@ -269,11 +271,16 @@ dam_status_t dam_decode_attention(const void* q, const void* K, const void* V, c
  * out[3] = bytes of the blob in use (the tile lists have a fixed place per row, sized by the row's upper
  * bound, so this follows from the shapes; out[0] says how many entries are real), out[4] = 128 x 128 tiles of the masks themselves that hold an
  * active cell (equals out[0] unless gathered-column tiles are listed). `out` is HOST memory
- * (5 x uint64). Synchronises `stream`. The paper reports no such counts; they feed the density and
- * active-FLOP figures of the benchmark.
+ * (5 x uint64). Synchronises `stream` before the header is read.
+ * active_elems_dev: DEVICE uint64[num_seqs][num_q_heads], 8-byte aligned, or NULL. When given, a kernel is
+ * enqueued on `stream` (not synchronised) that writes, for every (sequence, head), the number of active cells
+ * of its S x S mask: the true mask inside the window plus, for every row below it, the matched columns and the
+ * matched diagonals with a cell that is both counted once (Sec. 4.3, Case 2; the paper's O(s L) work figure in
+ * Sec. 5.3 is this count times 4 d). UNSUPPORTED for a blob made by dam_mask_all_ones.
+ * The paper reports no tile counts; they feed the density and active-FLOP figures of the benchmark.
  */
 dam_status_t dam_mask_stats(const void* mask, const dam_shape_t* shape, uint64_t* out,
-                            void* stream);
+                            uint64_t* active_elems_dev, void* stream);
 
 /*
  * Test hook: expands rows [row_begin, row_begin + nrows) of (seq, head) of the S x S mask exactly as
@@ -302,6 +309,17 @@ dam_status_t dam_poll_status(const void* mask_or_scratch, void* stream);
  * without faulting or hanging a GPU.
  */
 dam_status_t dam_selftest_bounded_wait(void* scratch, size_t scratch_bytes, uint32_t limit_us, void* stream);
+
+/*
+ * Self-test of the per-device bookkeeping (the paper has no counterpart). The library keeps, per device
+ * ordinal, the device's properties and which one-off set-up steps (the shared-memory opt-in of the tensor-core
+ * kernels) have run there, in a table guarded by a mutex, so that one process may drive several GPUs from several
+ * threads. This call runs the same table code on a private table with a fake device query, for the `n` ordinals
+ * given (HOST int32[n]): sm_counts[i] (HOST) receives 100 + ordinal (-1 for an ordinal outside 0..63, and the call
+ * then returns INVALID_ARGUMENT), counters[0] (HOST int32[2]) the number of queries made (one per distinct valid
+ * ordinal), counters[1] the number of set-up steps run (likewise). No device is touched.
+ */
+dam_status_t dam_selftest_device_table(const int32_t* ordinals, int32_t n, int32_t* sm_counts, int32_t* counters);
 
 /*
  * Both stages from HOST buffers (pinned recommended, layouts from `shape` with dense strides): copies

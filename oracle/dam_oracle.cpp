@@ -204,10 +204,10 @@ int oracle_attention_rows(const float* Q, const float* K, const float* V,
                           double* O, double* lse) {
   if (!Q || !K || !V || !rows || !O || !lse || S < 0 || d <= 0) return 1;
   int bad = 0;
-#pragma omp parallel for schedule(dynamic, 4)
+#pragma omp parallel for schedule(dynamic, 4) reduction(| : bad)
   for (int a = 0; a < nrows; ++a) {
     int i = rows[a];
-    if (i < 0 || i >= S) { bad = 1; continue; }
+    if (i < 0 || i >= S) { bad |= 1; continue; }
     const uint8_t* mrow = mask_rows ? mask_rows + (int64_t)a * S : nullptr;
     std::vector<double> s(S);
     const double ninf = -std::numeric_limits<double>::infinity();

@@ -4,9 +4,13 @@ TEST INFRASTRUCTURE ONLY: imported by tests, the smoke check and the
 benchmark's CPU-baseline leg; the CUDA library and its Python binding never
 import this module.
 
-The C++ file holds the arithmetic.  This module only marshals numpy arrays,
-loops over (sequence, head), and offers ``build_masks`` / ``attention`` helpers
-that chain the paper's steps in order:
+The C++ file holds the arithmetic of the main path (window softmax, Box-Cox
+threshold, pattern counts, match, extension, masked attention).  This module
+marshals numpy arrays for it, loops over (sequence, head), and states in numpy
+the two side branches of the method: the other amplifications of Appendix B
+(``amplify_transform`` / ``true_mask_transform``) and the multi-sample average
+of Sec. 4.2.2 (``capture_average``).  ``build_masks`` / ``attention`` chain the
+paper's steps in order:
 
   window softmax (Sec. 3, 4.2.1) -> Box-Cox + shift (Sec. 4.2.2) -> threshold
   (Sec. 4.2.3) -> pattern counts and match (Sec. 4.2.4) -> extension (Sec. 4.3)

@@ -24,7 +24,8 @@ STATUS = {0: "DAM_OK", 1: "DAM_ERR_INVALID_ARGUMENT", 2: "DAM_ERR_UNSUPPORTED", 
 EXPORTS = ["dam_version", "dam_status_string", "dam_mask_sizes", "dam_build_masks", "dam_build_masks_from_scores",
            "dam_mask_all_ones", "dam_sparse_attention", "dam_mask_stats", "dam_mask_expand_rows", "dam_poll_status",
            "dam_prefill_host", "dam_build_masks_static", "dam_static_scratch_bytes", "dam_selftest_bounded_wait",
-           "dam_decode_attention", "dam_sparse_attention_rows", "dam_capture_accumulate", "dam_capture_average"]
+           "dam_decode_attention", "dam_sparse_attention_rows", "dam_capture_accumulate", "dam_capture_average",
+           "dam_selftest_device_table"]
 
 
 class DamError(RuntimeError):
@@ -293,12 +294,29 @@ def dam_decode_attention(q, K, V, mask, shape: Shape, positions: torch.Tensor, s
     return O, lse, scratch
 
 
-def dam_mask_stats(mask: torch.Tensor, shape: Shape) -> dict:
+def dam_mask_stats(mask: torch.Tensor, shape: Shape, active_elements: bool = False) -> dict:
+    """Counts of a mask blob; with active_elements=True also the active cells per (sequence, head), counted by
+    the library on the device (int64 tensor [num_seqs, num_q_heads], key "active_elements")."""
     out = (ctypes.c_uint64 * 5)()
-    rc = lib().dam_mask_stats(_ptr(mask), shape.ref, out, _stream(mask.device))
+    ae = torch.zeros(shape.c.num_seqs, shape.c.num_q_heads, dtype=torch.int64, device=mask.device) if active_elements else None
+    rc = lib().dam_mask_stats(_ptr(mask), shape.ref, out, _ptr(ae), _stream(mask.device))
     _check(rc, "dam_mask_stats")
-    return {"tiles": int(out[0]), "full_tiles": int(out[1]), "causal_tiles": int(out[2]), "bytes_used": int(out[3]),
-            "mask_tiles": int(out[4])}
+    st = {"tiles": int(out[0]), "full_tiles": int(out[1]), "causal_tiles": int(out[2]), "bytes_used": int(out[3]),
+          "mask_tiles": int(out[4])}
+    if active_elements:
+        st["active_elements"] = ae
+    return st
+
+
+def dam_selftest_device_table(ordinals):
+    """Runs the library's per-device table on a private table with a fake device query (no device needed).
+    Returns (status code, sm_counts, (queries, set-up steps))."""
+    n = len(ordinals)
+    arr = (ctypes.c_int32 * max(1, n))(*ordinals)
+    sm = (ctypes.c_int32 * max(1, n))()
+    cnt = (ctypes.c_int32 * 2)()
+    rc = lib().dam_selftest_device_table(arr, n, sm, cnt)
+    return int(rc), [int(x) for x in sm[:n]], (int(cnt[0]), int(cnt[1]))
 
 
 def dam_mask_expand_rows(mask: torch.Tensor, shape: Shape, seq: int, head: int, row_begin: int, nrows: int,
@@ -398,23 +416,6 @@ class MaskBlob:
         off = int(self.hdr["off_true"]) + 4 * (int(s["true_off"]) + head * L * W)
         w = np.frombuffer(self.raw, dtype="<u4", count=L * W, offset=off).reshape(L, W)
         return _unpack_bits(w, L)
-
-    def active_elements(self, seq: int, head: int) -> int:
-        """Number of active cells of the S x S mask of (seq, head): the true mask inside the window, and below
-        it, per row, the matched columns plus the matched diagonals minus the cells that are both (rows
-        L .. 2L-2 only: a correlation of the two bit sets)."""
-        s = self.seqs[seq]
-        S, L, W = int(s["S"]), int(s["L"]), int(s["W"])
-        if L == 0:
-            return 0
-        off = int(self.hdr["off_true"]) + 4 * (int(s["true_off"]) + head * L * W)
-        words = np.frombuffer(self.raw, dtype="<u4", count=L * W, offset=off)
-        n = int(np.unpackbits(words.view(np.uint8)).sum())
-        if S > L:
-            D, _, V = self.pattern_bits(seq, head)
-            both = np.convolve(V.astype(np.int64), D.astype(np.int64))     # index i = column + diagonal
-            n += (S - L) * (int(D.sum()) + int(V.sum())) - int(both[L: min(S, 2 * L - 1)].sum())
-        return n
 
     def row_tiles(self, seq: int, head: int, qb: int):
         """(kv tile indices, kinds) of query block qb of (seq, head)."""

@@ -25,17 +25,11 @@ def _stale() -> bool:
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not _stale():
         return LIB
-    extra = ["-DDAM_PROFILE"] if os.environ.get("DAM_PROFILE") else []   # cycle counters for tuning runs
-    for knob in ("DAM_DEC_KPG", "DAM_DEC_BPS"):
-        if os.environ.get(knob):
-            extra.append("-D%s=%s" % (knob, os.environ[knob]))
-    if os.environ.get("DAM_POLY_PER8"):
-        extra.append("-DDAM_POLY_PER8=" + os.environ["DAM_POLY_PER8"])
     objs = []
     procs = []
     for src in SOURCES:
         obj = os.path.join(CSRC, src.replace(".cu", ".o"))
-        cmd = ["nvcc", *NVCC_FLAGS, *extra, "-c", os.path.join(CSRC, src), "-o", obj]
+        cmd = ["nvcc", *NVCC_FLAGS, "-c", os.path.join(CSRC, src), "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas")
             cmd.insert(2, "-v")

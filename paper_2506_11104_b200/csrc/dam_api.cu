@@ -219,11 +219,56 @@ dam_status_t fill_ctx(const dam_shape_t* s, const dam_rule_t* r, void* mask, siz
   return DAM_OK;
 }
 
+std::mutex g_device_mutex;
+
+cudaError_t query_device(int device, DamDeviceInfo* out) {
+  cudaError_t e;
+  if ((e = cudaDeviceGetAttribute(&out->cc_major, cudaDevAttrComputeCapabilityMajor, device)) != cudaSuccess) return e;
+  if ((e = cudaDeviceGetAttribute(&out->sm_count, cudaDevAttrMultiProcessorCount, device)) != cudaSuccess) return e;
+  return cudaDeviceGetAttribute(&out->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
+}
+
 }  // namespace
+
+cudaError_t DamDeviceTable::info(int device, dam_device_query_fn query, DamDeviceInfo* out) {
+  if (device < 0 || device >= kMaxDevices || !query || !out) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_device_mutex);
+  Slot& s = slots_[device];
+  if (!s.filled) {
+    DamDeviceInfo di = {};
+    const cudaError_t e = query(device, &di);
+    if (e != cudaSuccess) return e;                 // nothing is remembered about a failed query
+    s.info = di;
+    s.filled = true;
+  }
+  *out = s.info;
+  return cudaSuccess;
+}
+
+cudaError_t DamDeviceTable::once(int device, int key, dam_device_setup_fn fn) {
+  if (device < 0 || device >= kMaxDevices || key < 0 || key >= kMaxSetups || !fn) return cudaErrorInvalidValue;
+  std::lock_guard<std::mutex> lock(g_device_mutex);
+  Slot& s = slots_[device];
+  if (s.done[key]) return cudaSuccess;
+  const cudaError_t e = fn();
+  if (e == cudaSuccess) s.done[key] = true;
+  return e;
+}
+
+DamDeviceTable& dam_device_table() {
+  static DamDeviceTable table;
+  return table;
+}
+
+cudaError_t dam_current_device(int* device, DamDeviceInfo* info) {
+  cudaError_t e = cudaGetDevice(device);
+  if (e != cudaSuccess) return e;
+  return dam_device_table().info(*device, query_device, info);
+}
 
 extern "C" {
 
-int32_t dam_version(void) { return 1000; }
+int32_t dam_version(void) { return 1001; }
 
 const char* dam_status_string(dam_status_t s) {
   switch (s) {
@@ -402,13 +447,22 @@ dam_status_t dam_decode_attention(const void* q, const void* K, const void* V, c
   return e == cudaSuccess ? DAM_OK : DAM_ERR_CUDA;
 }
 
-dam_status_t dam_mask_stats(const void* mask, const dam_shape_t* shape, uint64_t* out, void* stream) {
+dam_status_t dam_mask_stats(const void* mask, const dam_shape_t* shape, uint64_t* out, uint64_t* active_elems_dev,
+                            void* stream) {
   if (!mask || !out || !shape) return DAM_ERR_INVALID_ARGUMENT;
+  if (active_elems_dev && !aligned(active_elems_dev, 8)) return DAM_ERR_INVALID_ARGUMENT;
   cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
   DamHeader h;
   if (cudaMemcpyAsync(&h, mask, sizeof(h), cudaMemcpyDeviceToHost, cs) != cudaSuccess) return DAM_ERR_CUDA;
   if (cudaStreamSynchronize(cs) != cudaSuccess) return DAM_ERR_CUDA;
   if (h.magic != DAM_MAGIC) return DAM_ERR_INVALID_ARGUMENT;
+  if (active_elems_dev) {
+    if (h.flags & DAM_FLAG_ALL_ONES) return DAM_ERR_UNSUPPORTED;      // an all-ones blob has no pattern sections
+    if (h.num_seqs != shape->num_seqs || h.num_q_heads != shape->num_q_heads) return DAM_ERR_INVALID_ARGUMENT;
+    if (dam_launch_active_elems(mask, h.num_seqs, h.num_q_heads, reinterpret_cast<unsigned long long*>(active_elems_dev),
+                                cs) != cudaSuccess)
+      return DAM_ERR_CUDA;
+  }
   out[0] = h.total_tiles; out[1] = h.full_tiles; out[2] = h.causal_tiles; out[3] = h.bytes_used;
   out[4] = h.mask_tiles;
   return DAM_OK;
@@ -447,6 +501,39 @@ dam_status_t dam_selftest_bounded_wait(void* scratch, size_t scratch_bytes, uint
   cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(scratch, 0, 256, cs) != cudaSuccess) return DAM_ERR_CUDA;
   return dam_launch_bounded_wait_selftest(scratch, 1000ull * limit_us, cs) == cudaSuccess ? DAM_OK : DAM_ERR_CUDA;
+}
+
+namespace {
+int g_fake_queries = 0;
+cudaError_t fake_query(int device, DamDeviceInfo* out) {
+  ++g_fake_queries;                                  // (called under the table's lock)
+  out->cc_major = 10; out->sm_count = 100 + device; out->smem_optin = 1000 * (device + 1);
+  return cudaSuccess;
+}
+int g_fake_setups = 0;
+cudaError_t fake_setup() { ++g_fake_setups; return cudaSuccess; }
+}  // namespace
+
+dam_status_t dam_selftest_device_table(const int32_t* ordinals, int32_t n, int32_t* sm_counts, int32_t* counters) {
+  if (!ordinals || !sm_counts || !counters || n < 0) return DAM_ERR_INVALID_ARGUMENT;
+  static std::mutex selftest_mutex;
+  std::lock_guard<std::mutex> lock(selftest_mutex);
+  DamDeviceTable table;                              // a table of its own: the library's records are not touched
+  g_fake_queries = g_fake_setups = 0;
+  dam_status_t st = DAM_OK;
+  for (int i = 0; i < n; ++i) {
+    DamDeviceInfo di = {};
+    if (table.info(ordinals[i], fake_query, &di) != cudaSuccess ||
+        table.once(ordinals[i], DAM_SETUP_ATTN_SMEM, fake_setup) != cudaSuccess) {
+      sm_counts[i] = -1;
+      st = DAM_ERR_INVALID_ARGUMENT;
+      continue;
+    }
+    sm_counts[i] = di.sm_count;
+  }
+  counters[0] = g_fake_queries;
+  counters[1] = g_fake_setups;
+  return st;
 }
 
 // Streams and events of the host-buffer entry point (created on first use, one set per device).
@@ -564,6 +651,10 @@ dam_status_t dam_prefill_host(const void* Qh, const void* Kh, const void* Vh, co
   // the workspace may still be in use by earlier work of the caller's stream
   ok = cudaEventRecord(P.start, cs) == cudaSuccess && cudaStreamWaitEvent(P.h2d, P.start, 0) == cudaSuccess &&
        cudaStreamWaitEvent(P.d2h, P.start, 0) == cudaSuccess;
+  // A chunk that ends at a sequence end inside a 128-key tile makes that tile's K / V rows reach into tokens that
+  // arrive with a later chunk; their probabilities are zero, but a zero times whatever bytes the workspace held
+  // (a NaN or an infinity) is not: K and V start out as zeros.
+  ok = ok && cudaMemsetAsync(w + off_k, 0, kb, P.h2d) == cudaSuccess && cudaMemsetAsync(w + off_v, 0, kb, P.h2d) == cudaSuccess;
   // windows first, with the row ranges of all chunks
   ok = ok && cudaMemcpyAsync(w + off_r, ranges.data(), ranges.size() * sizeof(int32_t), cudaMemcpyHostToDevice, P.h2d) == cudaSuccess;
   for (int b = 0; b < nb && ok; ++b) {

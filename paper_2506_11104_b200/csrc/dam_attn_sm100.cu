@@ -43,10 +43,7 @@ constexpr int kSchedNoSteps = 1 << 30;       // work-list entry handed to the co
 // Step descriptor bits: stream A / B has a tile in the step; it is the stream's last tile of the item; the item has
 // another step.
 constexpr uint32_t kStepA = 1u, kStepB = 2u, kStepLastA = 4u, kStepLastB = 8u, kStepMore = 16u;
-#ifndef DAM_POLY_PER8
-#define DAM_POLY_PER8 2
-#endif
-constexpr int kPolyPer8 = DAM_POLY_PER8;   // of every 8 exponentials, how many use the FMA-pipe polynomial (0, 2 or 4)
+constexpr int kPolyPer8 = 2;   // of every 8 exponentials, how many use the FMA-pipe polynomial (0, 2 or 4)
 
 struct SmemLayout {
   static constexpr int q = 0;                           // Q_A, Q_B
@@ -66,16 +63,6 @@ struct SmemLayout {
 static_assert(SmemLayout::item_rec % 16 == 0 && SmemLayout::bars % 8 == 0, "shared-memory records must be aligned");
 constexpr int kSmemBytes = SmemLayout::total + 1024;   // + slack for the 1024-byte alignment
 
-#ifdef DAM_PROFILE
-#define PROF_DECL(n) long long prof_acc[n] = {0}; long long prof_t = clock64();
-#define PROF_LAP(k) { long long now_ = clock64(); prof_acc[k] += now_ - prof_t; prof_t = now_; }
-#define PROF_FLUSH(base, n) if (blockIdx.x == 0) { for (int q_ = 0; q_ < n; ++q_) prm.prof[(base) + q_] = (unsigned long long)prof_acc[q_]; }
-#else
-#define PROF_DECL(n)
-#define PROF_LAP(k)
-#define PROF_FLUSH(base, n)
-#endif
-
 // What the producer hands to the softmax warps with every work-list position: the item record, the first tile
 // entry of each stream and the head's bit-set pointers, so that their set-up reads shared memory instead of
 // walking item -> sequence record -> tile list in global memory.
@@ -87,7 +74,6 @@ struct ItemRec {
 static_assert(sizeof(ItemRec) == 96, "ItemRec must be 96 bytes");
 
 struct AttnParams {
-  unsigned long long* prof;
   const unsigned char* blob;
   __nv_bfloat16* O;
   float* lse;
@@ -123,10 +109,6 @@ __device__ __forceinline__ Item item_from_words(const uint4& u, const uint4& v) 
   it.a0 = v.x; it.a1 = v.y; it.b0 = v.y; it.b1 = v.z;
   it.hasB = (int)(v.w >> 31); it.seq = (int)(v.w & 0x7FFFFFFFu);
   return it;
-}
-__device__ __forceinline__ Item load_item(const unsigned char* blob, const DamHeader* H, int w) {
-  const uint4* src = reinterpret_cast<const uint4*>(blob + H->off_work) + 2 * (size_t)w;
-  return item_from_words(__ldg(src), __ldg(src + 1));
 }
 
 // Merge of the two ascending tile lists: every step is one kv tile with the kinds it has in A and in B.
@@ -317,8 +299,12 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   const DamHeader* H = reinterpret_cast<const DamHeader*>(blob);
   const int nitems = H->prows;
   const uint32_t* tiles = reinterpret_cast<const uint32_t*>(blob + H->off_tiles);
-  // a blob with gathered-column tiles needs the larger scratch; the gather kernel has recorded the error
-  if ((H->flags & DAM_FLAG_GATHER) && H->attn_scratch_bytes > prm.scratch_bytes) return;
+  // a blob with gathered-column tiles needs the larger scratch: nothing is computed without it, and the status
+  // word says why (the gather kernel is not even launched when the scratch holds no tile at all)
+  if ((H->flags & DAM_FLAG_GATHER) && H->attn_scratch_bytes > prm.scratch_bytes) {
+    if (blockIdx.x == 0 && tid == 0) atomicMax(prm.status, (uint32_t)DAM_ERR_BUFFER_TOO_SMALL);
+    return;
+  }
   // Dynamic scheduling: the work list is sorted longest first; the producer thread takes positions from a
   // global counter (the first one is the CTA index) and hands each to the other roles through a two-entry
   // ring in shared memory.  A negative position ends the loop.
@@ -361,12 +347,9 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 #pragma unroll
       for (int s = 0; s < kSlots; ++s) armed[s] = 2u;      // 2 = never armed
       bool ok = true;
-      PROF_DECL(4)
       auto load_tile = [&](const CUtensorMap* tm, int head, int tok) -> bool {
         const uint32_t s = sc % kSlots, ph = (sc / kSlots) & 1u;
-        PROF_LAP(0)
         if (!mbar_wait(bSlotEmpty + 8 * s, ph ^ 1u, abort_flag)) return false;
-        PROF_LAP(1)
         const uint32_t dst = sSlots + s * kSlotBytes, bar = bSlotFull + 8 * s;
         mbar_arrive_expect_tx(bar, kSlotBytes);
         tma_load_3d(dst, tm, bar, 0, head, tok);
@@ -439,8 +422,6 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           if (armed[s] != 2u) mbar_wait(bSlotFull + 8 * s, armed[s], &dummy, 20000000ull);
         mbar_wait(bQFull, (ic + 1u) & 1u, &dummy, 20000000ull);
       }
-      PROF_LAP(0)
-      PROF_FLUSH(0, 4)
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
@@ -450,7 +431,6 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       uint32_t sc = 0, ic = 0, step = 0;
       uint32_t cP[2] = {0u, 0u};           // P tiles consumed per stream (phase of p_full)
       bool ok = true;
-      PROF_DECL(6)
       // descriptors: the high words are invariant, the low words step by (byte offset >> 4)
       const uint64_t dQ = smem_desc_sw128(sQ, 16, 1024);
       const uint64_t dK = smem_desc_sw128(sSlots, 16, 1024);
@@ -469,9 +449,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         tc_commit(bSFull + 8 * X);
       };
       auto issue_pv = [&](int X, uint32_t slot, bool accumulate) -> bool {
-        PROF_LAP(0)
         if (!mbar_wait(bPFull + 8 * X, cP[X] & 1u, abort_flag)) return false;
-        PROF_LAP(1 + X)
         ++cP[X];
         tc_fence_after();
         const uint32_t b0 = dV_lo + slot * (kSlotBytes >> 4);
@@ -487,16 +465,13 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         const int w = next_item_consumer(n, true);
         if (w < 0) { ok = (w == -1); break; }
         if (w & kSchedNoSteps) continue;
-        PROF_LAP(0)
         if (!(ok = mbar_wait(bQFull, ic & 1u, abort_flag))) break;
-        PROF_LAP(3)
         ++ic;
         // S of the first step (the producer's descriptor of a step is readable once its K tile is)
         uint32_t d;
         {
           const uint32_t s = sc % kSlots;
           if (!(ok = mbar_wait(bSlotFull + 8 * s, (sc / kSlots) & 1u, abort_flag))) break;
-          PROF_LAP(4)
           d = step_desc[step & 15u];
           tc_fence_after();
           if (d & kStepA) issue_s(0, s);
@@ -509,18 +484,14 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           const bool have_nxt = (d & kStepMore) != 0u;
           if (!have_nxt) tc_commit(bQEmpty);                   // every S of this item has been issued
           const uint32_t sv = sc % kSlots;                     // V of the current step
-          PROF_LAP(0)
           if (!(ok = mbar_wait(bSlotFull + 8 * sv, (sc / kSlots) & 1u, abort_flag))) break;
-          PROF_LAP(4)
           ++sc;
           uint32_t sk = 0, dn = 0;
           // a stream's output is final right after the P V of its last listed tile
           if (d & kStepA) { if (!(ok = issue_pv(0, sv, accA))) break; accA = true; if (d & kStepLastA) tc_commit(bOFinal); }
           if (have_nxt) {                                      // K of the next step
             sk = sc % kSlots;
-            PROF_LAP(0)
             if (!(ok = mbar_wait(bSlotFull + 8 * sk, (sc / kSlots) & 1u, abort_flag))) break;
-            PROF_LAP(4)
             ++sc;
             dn = step_desc[(step + 1u) & 15u];
             tc_fence_after();
@@ -535,12 +506,6 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           d = dn;
         }
       }
-      PROF_LAP(0)
-      PROF_FLUSH(4, 6)
-#ifdef DAM_PROFILE
-      { long long tot_ = 0; for (int q_ = 0; q_ < 6; ++q_) tot_ += prof_acc[q_];
-        prm.prof[128 + 2 * blockIdx.x] = (unsigned long long)tot_; prm.prof[128 + 2 * blockIdx.x + 1] = (unsigned long long)prof_acc[0]; }
-#endif
     }
   } else {
     // ------------------------------------------------------------------ softmax / epilogue warps
@@ -553,7 +518,6 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const uint32_t stage_addr = sbase + SmemLayout::stage + X * kStageBytes + (warp & 3) * 4096;   // 32 rows x 128 B
     uint32_t cS = 0, cO = 0;
     bool ok = true;
-    PROF_DECL(8)
     for (uint32_t n = 0; ok; ++n) {
       const int ws = next_item_consumer(n, false);
       if (ws < 0) {
@@ -608,9 +572,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           bits_nx = tile_bits(e_next, need_nx);
           if (t + 2 < t1) e_next = __ldg(tiles + t + 2);
         }
-        PROF_LAP(0)
         if (!(ok = mbar_wait(bS, cS & 1u, abort_flag))) break;
-        PROF_LAP(1)
         ++cS;
         tc_fence_after();
         // ---- sweep 1: row maximum of the raw dot products.  On a masked tile the maximum over all entries is
@@ -625,7 +587,6 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           else masked_max = __any_sync(0xFFFFFFFFu, mu * prm.scale_log2 - m_ref > kRescaleThreshold);   // -inf reference: true
         }
         if (masked_max) mx = sweep_max<true>(tS, bits);
-        PROF_LAP(2)
         const float m_new = fmaxf(m_ref, mx * prm.scale_log2);
         // move the reference only on the first tile or when the max grew by more than the threshold
         bool move = (t == t0) || (m_new - m_ref > kRescaleThreshold);   // -inf reference: inf > 8 is true
@@ -639,7 +600,6 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         // ---- sweep 2: probabilities against the reference max, packed to bf16 into the first half of S
         const float tsum = need_mask ? sweep_exp<true>(tS, bits, prm.scale_log2, -mm)
                                      : sweep_exp<false>(tS, bits, prm.scale_log2, -mm);
-        PROF_LAP(3)
         l = l * alpha + tsum;
         // ---- O is complete up to the previous tile of this stream (its MMAs precede S of this tile)
         if (t > t0) {
@@ -656,18 +616,14 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             }
           }
         }
-        PROF_LAP(4)
         tc_wait_st();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bP);
-        PROF_LAP(5)
       }
       if (!ok) break;
       // ---- epilogue: O / l and the log-sum-exp
-      PROF_LAP(0)
       if (!(ok = mbar_wait(bO, cO & 1u, abort_flag))) break;
-      PROF_LAP(6)
       ++cO;
       tc_fence_after();
       const float inv = l > 0.f ? 1.0f / l : 0.f;
@@ -728,12 +684,8 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       }
       if (row_valid) *lse_p = l > 0.f ? (m_ref + log2f(l)) * 0.6931471805599453f : -CUDART_INF_F;
       tc_fence_before();
-      PROF_LAP(7)
     }
     if (lane == 0) tma_store_wait_all();                    // outstanding O stores complete before the CTA exits
-#ifdef DAM_PROFILE
-    if (tid == 64 || tid == 192) { PROF_FLUSH(10 + 8 * X, 8) }
-#endif
   }
 
   if (*abort_flag && tid == 64) atomicMax(prm.status, (uint32_t)DAM_ERR_DEVICE_TIMEOUT);
@@ -850,21 +802,18 @@ cudaError_t dam_launch_attn_sm100(const void* Q, const void* K, const void* V, c
                                   size_t scratch_bytes, const int32_t* ranges, bool run_gather, cudaStream_t st) {
   if (s->dtype != DAM_BF16 || s->head_dim != 128) return cudaErrorNotSupported;
   if (s->total_tokens == 0) return cudaSuccess;
-  static int sm_count = 0, smem_optin = 0;
-  if (sm_count == 0) {
-    int dev = 0;
-    cudaError_t e;
-    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-    int cc_major = 0;
-    cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev);
-    if (cc_major != 10) return cudaErrorNotSupported;
-    cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-    if (smem_optin < kSmemBytes) return cudaErrorNotSupported;
-    if ((e = cudaFuncSetAttribute(attn_sm100_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) != cudaSuccess ||
-        (e = cudaFuncSetAttribute(attn_sm100_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) != cudaSuccess)
-      return e;
-    cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-  }
+  int dev = 0;
+  DamDeviceInfo di;
+  cudaError_t e;
+  if ((e = dam_current_device(&dev, &di)) != cudaSuccess) return e;
+  if (di.cc_major != 10 || di.smem_optin < kSmemBytes) return cudaErrorNotSupported;
+  if ((e = dam_device_table().once(dev, DAM_SETUP_ATTN_SMEM, [](void) -> cudaError_t {
+         cudaError_t r = cudaFuncSetAttribute(attn_sm100_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+         if (r != cudaSuccess) return r;
+         return cudaFuncSetAttribute(attn_sm100_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+       })) != cudaSuccess)
+    return e;
+  const int sm_count = di.sm_count;
   // gathered-column tiles (if the blob has any) live after the 256-byte status block of the scratch buffer
   const size_t grows = scratch_bytes > 256 ? (scratch_bytes - 256) / 256 : 0;      // rows of 128 bf16
   CUtensorMap tq, tk, tv, to, tg;
@@ -899,8 +848,6 @@ cudaError_t dam_launch_attn_sm100(const void* Q, const void* K, const void* V, c
   p.work_counter = reinterpret_cast<uint32_t*>(scratch) + 2;
   p.scratch_bytes = scratch_bytes;
   p.ranges = ranges;
-  // profile builds keep their cycle counters in the last 8 KiB of the scratch buffer
-  p.prof = reinterpret_cast<unsigned long long*>(reinterpret_cast<unsigned char*>(scratch) + (scratch_bytes >= 16384 ? scratch_bytes - 8192 : 256));
   p.Hq = s->num_q_heads; p.group = s->num_q_heads / s->num_kv_heads; p.total_tokens = s->total_tokens;
   p.causal = causal;
   p.o_stride_tok = s->o_stride_tok; p.o_stride_head = s->o_stride_head;

@@ -18,14 +18,8 @@
 namespace {
 
 constexpr int kWarps = 8;
-#ifndef DAM_DEC_KPG
-#define DAM_DEC_KPG 2
-#endif
-#ifndef DAM_DEC_BPS
-#define DAM_DEC_BPS 4
-#endif
-constexpr int kKeysPerGroup = DAM_DEC_KPG;     // keys a lane group has in flight per step
-constexpr int kBlocksPerSM = DAM_DEC_BPS;      // resident blocks the register budget is sized for
+constexpr int kKeysPerGroup = 2;               // keys a lane group has in flight per step
+constexpr int kBlocksPerSM = 4;                // resident blocks the register budget is sized for
 constexpr int kRoundWords = 256;               // pattern words the block expands at a time (<= 8192 keys, 32 KB)
 
 template <typename T, int N> struct LdN;       // N consecutive elements -> float

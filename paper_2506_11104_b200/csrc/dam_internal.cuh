@@ -205,6 +205,32 @@ __device__ __forceinline__ uint4 dam_apply_bits(const DamHeadBits& hb, uint32_t 
   return b;
 }
 
+// ---- per-device state ---------------------------------------------------------------------------
+// What a launch needs to know about the device it runs on, and the one-off set-up steps that CUDA wants per
+// device (cudaFuncSetAttribute for the large dynamic shared memory of the tensor-core kernels).  Records are kept
+// per device ordinal and filled on first use under a mutex, so that one process may drive several GPUs from
+// several threads.
+struct DamDeviceInfo { int cc_major, sm_count, smem_optin; };
+typedef cudaError_t (*dam_device_query_fn)(int device, DamDeviceInfo* out);
+typedef cudaError_t (*dam_device_setup_fn)(void);
+
+class DamDeviceTable {
+ public:
+  static constexpr int kMaxDevices = 64;
+  static constexpr int kMaxSetups = 8;
+  // The record of `device`, filled by `query` the first time the ordinal is seen.
+  cudaError_t info(int device, dam_device_query_fn query, DamDeviceInfo* out);
+  // Runs `fn` (with `device` current) unless set-up step `key` already succeeded on that device.
+  cudaError_t once(int device, int key, dam_device_setup_fn fn);
+ private:
+  struct Slot { bool filled; DamDeviceInfo info; bool done[kMaxSetups]; };
+  Slot slots_[kMaxDevices] = {};
+};
+enum { DAM_SETUP_ATTN_SMEM = 0, DAM_SETUP_SCORE_SMEM = 1 };
+
+DamDeviceTable& dam_device_table();                                       // the library's own table
+cudaError_t dam_current_device(int* device, DamDeviceInfo* info);         // ordinal and record of the current device
+
 // ---- host-side launch entry points of the kernel files -----------------------------------------
 struct DamBuildCtx {
   unsigned char* blob;
@@ -233,6 +259,7 @@ cudaError_t dam_launch_rule(const DamBuildCtx& c, cudaStream_t st);
 cudaError_t dam_launch_all_ones(const dam_shape_t* shape, int causal, void* blob, cudaStream_t st);
 cudaError_t dam_launch_expand_rows(const void* blob, int seq, int head, int row_begin, int nrows, int words,
                                    int causal, uint32_t* out, cudaStream_t st);
+cudaError_t dam_launch_active_elems(const void* blob, int num_seqs, int Hq, unsigned long long* out, cudaStream_t st);
 // `ranges` (device, int32[2 * num_seqs], or NULL): only the pairs of query blocks whose first row lies in
 // [ranges[2b], ranges[2b+1]) of sequence b are computed
 cudaError_t dam_launch_attn_ref(const void* Q, const void* K, const void* V, const void* blob,

@@ -878,6 +878,52 @@ cudaError_t dam_launch_all_ones(const dam_shape_t* shape, int causal, void* blob
   return cudaGetLastError();
 }
 
+// Active cells of the S x S mask of every (sequence, head): the true mask inside the window; below it every row
+// keeps the matched columns and the matched diagonals, and a cell that is both (key j = i - r with V[j] and D[r],
+// possible on rows L .. 2L-2 only) counts once (Sec. 4.3, Case 2).  One block per (sequence, head); integer
+// arithmetic, the block's partial sums are added in a fixed order.
+__global__ void __launch_bounds__(256)
+active_elems_kernel(const unsigned char* blob, unsigned long long* __restrict__ out) {
+  const DamHeader* H = reinterpret_cast<const DamHeader*>(blob);
+  const int b = blockIdx.x / H->num_q_heads, h = blockIdx.x % H->num_q_heads;
+  const DamSeq sq = blob_seqs(blob, H)[b];
+  __shared__ unsigned long long part[256];
+  unsigned long long n = 0;
+  if (sq.L > 0) {
+    const DamHeadBits hb = dam_head_bits(blob, H, sq, h);
+    const size_t words = (size_t)sq.L * sq.W;
+    for (size_t w = threadIdx.x; w < words; w += blockDim.x) n += (unsigned long long)__popc(__ldg(hb.M + w));
+    if (sq.S > sq.L) {
+      // rows i in [L, min(S, 2L-1)): overlap(i) = #{j < L : V[j] and D[i-j]}; keys j .. j+31 read Drev bits from L-1-i+j
+      const int i_end = sq.S < 2 * sq.L - 1 ? sq.S : 2 * sq.L - 1;
+      long long both = 0;
+      for (int i = sq.L + (int)threadIdx.x; i < i_end; i += blockDim.x)
+        for (int w = 0; w < sq.W; ++w) {
+          const uint32_t v = __ldg(hb.V + w);
+          if (v) both += __popc(v & dam_window32(hb.Drev, sq.W, sq.L - 1 - i + 32 * w));
+        }
+      if (threadIdx.x == 0) {
+        long long pd = 0, pv = 0;
+        for (int w = 0; w < sq.W; ++w) { pd += __popc(__ldg(hb.D + w)); pv += __popc(__ldg(hb.V + w)); }
+        n += (unsigned long long)((long long)(sq.S - sq.L) * (pd + pv));
+      }
+      n -= (unsigned long long)both;      // (modular arithmetic: the block's total is what counts)
+    }
+  }
+  part[threadIdx.x] = n;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned long long t = 0;
+    for (int k = 0; k < 256; ++k) t += part[k];
+    out[blockIdx.x] = t;
+  }
+}
+
+cudaError_t dam_launch_active_elems(const void* blob, int num_seqs, int Hq, unsigned long long* out, cudaStream_t st) {
+  active_elems_kernel<<<num_seqs * Hq, 256, 0, st>>>(reinterpret_cast<const unsigned char*>(blob), out);
+  return cudaGetLastError();
+}
+
 cudaError_t dam_launch_expand_rows(const void* blob, int seq, int head, int row_begin, int nrows, int words,
                                    int causal, uint32_t* out, cudaStream_t st) {
   expand_rows_kernel<<<nrows, 128, 0, st>>>(reinterpret_cast<const unsigned char*>(blob), seq, head, row_begin, nrows,

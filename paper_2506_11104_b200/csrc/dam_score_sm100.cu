@@ -375,18 +375,16 @@ cudaError_t dam_launch_scores_sm100(const void* Q, const void* K, const dam_shap
                                     float* dump, cudaStream_t st) {
   if (s->dtype != DAM_BF16 || s->head_dim != 128) return cudaErrorNotSupported;
   if (c.max_nL == 0) return cudaSuccess;
-  static int sm_count = 0;
-  if (sm_count == 0) {
-    int dev = 0, cc_major = 0, smem_optin = 0;
-    cudaError_t e;
-    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-    cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev);
-    cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-    if (cc_major != 10 || smem_optin < kSmemBytes) return cudaErrorNotSupported;
-    if ((e = cudaFuncSetAttribute(score_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) != cudaSuccess)
-      return e;
-    cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-  }
+  int dev = 0;
+  DamDeviceInfo di;
+  cudaError_t e;
+  if ((e = dam_current_device(&dev, &di)) != cudaSuccess) return e;
+  if (di.cc_major != 10 || di.smem_optin < kSmemBytes) return cudaErrorNotSupported;
+  if ((e = dam_device_table().once(dev, DAM_SETUP_SCORE_SMEM, [](void) -> cudaError_t {
+         return cudaFuncSetAttribute(score_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+       })) != cudaSuccess)
+    return e;
+  const int sm_count = di.sm_count;
   CUtensorMap tq, tk;
   if (!dam_make_tmap_bf16(&tq, Q, 128, s->num_q_heads, s->total_tokens, s->q_stride_tok, s->q_stride_head) ||
       !dam_make_tmap_bf16(&tk, K, 128, s->num_kv_heads, s->total_tokens, s->k_stride_tok, s->k_stride_head))

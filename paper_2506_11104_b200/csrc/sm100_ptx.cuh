@@ -61,42 +61,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
-__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-
-// The same bounded wait for a whole warp of a role that is off the critical path: one lane polls without
-// blocking in the barrier unit and sleeps between polls, the other lanes wait at the warp barrier, so that the
-// waiting warp leaves the issue slots and the shared-memory port to the others.
-__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                                  uint64_t limit_ns = 2000000000ull) {
-  uint32_t ok = 1u;
-  if ((threadIdx.x & 31u) == 0u) {
-    uint64_t t0 = 0;
-    for (uint32_t it = 1; !mbar_test_wait(bar, parity); ++it) {
-      __nanosleep(100);
-      if ((it & 255u) == 0) {
-        if (*abort_flag) { ok = 0u; break; }
-        uint64_t now = globaltimer_ns();
-        if (t0 == 0) t0 = now;
-        else if (now - t0 > limit_ns) { *abort_flag = 1u; ok = 0u; break; }
-      }
-    }
-  }
-  ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
-  // the other lanes take the acquire of the completed phase themselves
-  if (ok) { while (!mbar_test_wait(bar, parity)) {} }
-  return ok != 0u;
-}
-
 // ---- TMA ----------------------------------------------------------------------------------------
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* m) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
@@ -126,12 +90,6 @@ __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {   // whole warp
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
 }
-// Register reallocation between warpgroups (whole warpgroup, same value in every warp).
-template <int N>
-__device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
-template <int N>
-__device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
-
 __device__ __forceinline__ void tmem_relinquish() {                               // whole warp
   asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
 }

@@ -97,3 +97,22 @@ def test_null_and_misaligned_pointers_rejected_before_any_launch():
     n = ctypes.c_size_t(0)
     rc = lib.dam_prefill_host(null, null, null, sh.ref, ctypes.byref(rule), 1, null, null, null, ctypes.byref(n), null)
     assert rc == 0 and n.value > 0            # size query only
+
+
+def test_per_device_table_keeps_one_record_per_ordinal():
+    """The table behind the tensor-core launches (device properties and one-off set-up steps per device ordinal),
+    driven with a fake device query for two fake ordinals and from several threads at once."""
+    rc, sm, (queries, setups) = B.dam_selftest_device_table([0, 1, 0, 1, 1, 0])
+    assert rc == 0 and sm == [100, 101, 100, 101, 101, 100]
+    assert queries == 2 and setups == 2                      # once per device, not once per process or per call
+    rc, sm, (queries, setups) = B.dam_selftest_device_table([5, 64, -1, 5])
+    assert rc == 1 and sm == [105, -1, -1, 105] and queries == 1 and setups == 1
+    import threading
+    results = []
+    ts = [threading.Thread(target=lambda k=k: results.append(B.dam_selftest_device_table([k % 3, (k + 1) % 3] * 50)))
+          for k in range(8)]
+    for t in ts:
+        t.start()
+    for t in ts:
+        t.join()
+    assert len(results) == 8 and all(r[0] == 0 and r[2] == (2, 2) for r in results)

@@ -17,11 +17,26 @@ def _shape(w):
     return B.make_shape(w.cu_seqlens, w.num_q_heads, w.num_kv_heads, w.head_dim, w.Q.dtype, DEV)
 
 
-def _run(w, blob, shape, causal=True):
+def _run(w, blob, shape, causal=True, sentinel=False):
     Q, K, V = w.Q.to(DEV), w.K.to(DEV), w.V.to(DEV)
-    O, lse, scratch = B.dam_sparse_attention(Q, K, V, blob, shape, causal=causal)
+    O = lse = None
+    if sentinel:
+        # every row of every head must be written: a work item that was dropped would leave the NaN fill behind
+        O = torch.full_like(Q, float("nan"))
+        lse = torch.full((w.num_q_heads, Q.shape[0]), float("nan"), dtype=torch.float32, device=DEV)
+    O, lse, scratch = B.dam_sparse_attention(Q, K, V, blob, shape, causal=causal, O=O, lse=lse)
     assert B.dam_poll_status(scratch) == 0
+    if sentinel:
+        _assert_every_row_written(O, lse)
     return O, lse
+
+
+def _assert_every_row_written(O, lse):
+    """No fill value left: O finite everywhere, LSE finite or -inf, and O = 0 exactly on the rows whose LSE is -inf."""
+    assert torch.isfinite(O).all(), "rows of O were not written"
+    assert not torch.isnan(lse).any() and not torch.isposinf(lse).any(), "rows of LSE were not written"
+    empty = torch.isneginf(lse).transpose(0, 1)                       # [T, Hq]
+    assert (O[empty] == 0).all()
 
 
 def _check(w, O, lse, masks, rows_for, heads=None, causal=True, all_ones=False):
@@ -42,13 +57,21 @@ def _all_rows(S):
     return list(range(S))
 
 
-def _sample_rows(L):
+def _sample_rows(L, n_random=256, n_blocks=8):
+    """The rows around the window edges and the first row without overlap of columns and diagonals, both edge rows
+    of `n_blocks` random 128-row query blocks, and `n_random` random rows."""
     def f(S, L=L):
         rng = np.random.default_rng(S)
         fixed = [0, L - 1, L, L + 1, 2 * L - 2, 2 * L - 1, S - 1, 127, 128, S - 129]
-        rows = set(r for r in fixed if 0 <= r < S) | set(int(x) for x in rng.choice(S, size=min(S, 40), replace=False))
+        nq = (S + 127) // 128
+        for qb in rng.choice(nq, size=min(nq, n_blocks), replace=False):
+            fixed += [int(qb) * 128, min(S - 1, int(qb) * 128 + 127)]
+        rows = set(r for r in fixed if 0 <= r < S) | set(int(x) for x in rng.choice(S, size=min(S, n_random), replace=False))
         return sorted(rows)
     return f
+
+
+HEADS8 = [0, 5, 9, 13, 18, 22, 27, 31]
 
 
 @pytest.mark.parametrize("lengths,Hq,Hkv,d,dtype,causal", [
@@ -67,7 +90,7 @@ def test_all_ones_mask_is_dense_attention(lengths, Hq, Hkv, d, dtype, causal):
     _check(w, O, lse, None, _all_rows, causal=causal, all_ones=True)
 
 
-def _masked_case(w, rows_for, heads=None, gather=False):
+def _masked_case(w, rows_for, heads=None, gather=False, sentinel=False):
     shape = _shape(w)
     rule = B.make_rule(w.pcl_max, w.tau, w.mu, w.lam, w.eps, gather_columns=gather)
     n = sum(w.num_q_heads * min(S, w.pcl_max) ** 2 for S in shape.lengths)
@@ -75,7 +98,7 @@ def _masked_case(w, rows_for, heads=None, gather=False):
     blob, _ = B.dam_build_masks(w.Q.to(DEV), w.K.to(DEV), shape, rule, scores_dump=dump)
     assert B.dam_poll_status(blob) == 0
     masks = H.oracle_masks_from_dump(w, dump.cpu().numpy(), heads=heads)      # identical mask on both sides
-    O, lse = _run(w, blob, shape)
+    O, lse = _run(w, blob, shape, sentinel=sentinel)
     worst = _check(w, O, lse, masks, rows_for, heads=heads)
     return blob, shape, masks, O, lse, worst
 
@@ -110,7 +133,7 @@ def test_empty_rows_and_no_patterns():
 @pytest.mark.parametrize("gather", [False, True])
 def test_config1_sampled_rows(gather):
     w = synth.config1()
-    _masked_case(w, _sample_rows(1024), heads=[0, 5, 13, 22, 31], gather=gather)
+    _masked_case(w, _sample_rows(1024), heads=HEADS8, gather=gather, sentinel=True)
 
 
 def test_config1_dense_causal_sampled_rows():
@@ -124,13 +147,13 @@ def test_config1_dense_causal_sampled_rows():
 @pytest.mark.parametrize("gather", [False, True])
 def test_config4_varlen_sampled_rows(gather):
     w = synth.config4()
-    _masked_case(w, _sample_rows(1024), heads=[2, 17], gather=gather)
+    _masked_case(w, _sample_rows(1024), heads=HEADS8, gather=gather, sentinel=True)
 
 
 def test_config2_layer_sampled_rows():
     """One layer of the 32-layer stack (32768 tokens, PCL 2048), in the launch configuration the benchmark times."""
     w = synth.config2_layer(5, DEV)
-    blob, shape, masks, O, lse, worst = _masked_case(w, _sample_rows(2048), heads=[1, 12, 27], gather=True)
+    blob, shape, masks, O, lse, worst = _masked_case(w, _sample_rows(2048), heads=HEADS8, gather=True, sentinel=True)
     st = B.dam_mask_stats(blob, shape)
     assert 0.01 <= st["tiles"] / st["causal_tiles"] <= 0.30
 
@@ -138,20 +161,25 @@ def test_config2_layer_sampled_rows():
 def test_config3_sampled_rows():
     """131072 tokens, PCL 4096: sampled rows of a few heads against the oracle over all 131072 keys."""
     w = synth.config3(DEV)
-    _masked_case(w, _sample_rows(4096), heads=[4, 19], gather=True)
+    _masked_case(w, _sample_rows(4096), heads=HEADS8, gather=True, sentinel=True)
 
 
 def test_gathered_blob_with_small_scratch_reports_error():
-    """A blob with gathered-column tiles needs the larger scratch; a 256-byte scratch is refused on the device."""
+    """A blob with gathered-column tiles needs the larger scratch; a scratch that holds some tiles but not all, and
+    the 256-byte scratch that is enough for every other blob, are both refused on the device: O and LSE stay as
+    they were and the status word says BUFFER_TOO_SMALL."""
     w = synth.small_case(0, 4, 2, 128, 128, seed=4, lengths=[900])
     shape = _shape(w)
     rule = B.make_rule(w.pcl_max, w.tau, w.mu, gather_columns=True)
     blob, _ = B.dam_build_masks(w.Q.to(DEV), w.K.to(DEV), shape, rule)
     assert B.dam_mask_sizes(shape, rule)[2] > 256
-    small = torch.zeros(256 + 70000, dtype=torch.uint8, device=DEV)[:256 + 65536]
-    O, lse, scr = B.dam_sparse_attention(w.Q.to(DEV), w.K.to(DEV), w.V.to(DEV), blob, shape, scratch=small)
-    torch.cuda.synchronize()
-    assert B.dam_poll_status(scr) == 3
+    for nbytes in (256 + 65536, 256):
+        small = torch.zeros(256 + 70000, dtype=torch.uint8, device=DEV)[:nbytes]
+        O = torch.full_like(w.Q.to(DEV), 7.0)
+        O, lse, scr = B.dam_sparse_attention(w.Q.to(DEV), w.K.to(DEV), w.V.to(DEV), blob, shape, scratch=small, O=O)
+        torch.cuda.synchronize()
+        assert B.dam_poll_status(scr) == 3
+        assert (O == 7.0).all()
 
 
 def test_bounded_wait_times_out_cleanly():
@@ -207,13 +235,16 @@ def test_degenerate_lengths(gather):
     ([900, 512], 2, 2, 64, torch.float32, False),
 ])
 def test_chunked_prefill_equals_one_call(lengths, Hq, Hkv, d, dtype, gather):
-    """Row ranges: chunks of 256 / 512 rows, with the cache beyond each chunk's end poisoned, give bit for bit the
-    output of the single call (the arithmetic per row is the same and no row reads a key beyond itself)."""
+    """Row ranges: chunks of 256 / 512 rows, with the cache beyond each chunk's end poisoned, give the oracle's
+    O and LSE on every row (Sec. 4.3, Case 2, applied to rows that arrive in chunks) and, bit for bit, the output of
+    the single call (the arithmetic per row is the same and no row reads a key beyond itself)."""
     w = synth.small_case(0, Hq, Hkv, d, 128, seed=21, dtype=dtype, lengths=lengths)
     shape = _shape(w)
     rule = B.make_rule(w.pcl_max, w.tau, w.mu, w.lam, w.eps, gather_columns=gather)
     Q, K, V = w.Q.to(DEV), w.K.to(DEV), w.V.to(DEV)
-    blob, _ = B.dam_build_masks(Q, K, shape, rule)
+    dump = torch.zeros(sum(Hq * min(S, w.pcl_max) ** 2 for S in lengths), dtype=torch.float32, device=DEV)
+    blob, _ = B.dam_build_masks(Q, K, shape, rule, scores_dump=dump)
+    masks = H.oracle_masks_from_dump(w, dump.cpu().numpy())
     O_ref, lse_ref, _ = B.dam_sparse_attention(Q, K, V, blob, shape, causal=True)
     O = torch.full_like(O_ref, 7.0)
     lse = torch.full_like(lse_ref, 7.0)
@@ -230,6 +261,7 @@ def test_chunked_prefill_equals_one_call(lengths, Hq, Hkv, d, dtype, gather):
             done[b] = max(done[b], r1)
         scratch = B.dam_sparse_attention_rows(Q, Kc, Vc, blob, shape, ranges, O, lse)
         assert B.dam_poll_status(scratch) == 0
+    _check(w, O, lse, masks, _all_rows)                      # the chunked output itself against the oracle
     assert torch.equal(O, O_ref)
     assert torch.equal(lse, lse_ref)
 

@@ -208,12 +208,20 @@ def test_config2_layer_masks():
     blob, shape, masks, dump = _build_and_check(w, qblocks=10, gather=True)
     st = B.dam_mask_stats(blob, shape)
     assert 0.01 <= st["tiles"] / st["causal_tiles"] <= 0.30
+    # the scoring kernel's own map at PCL 2048 (16 kv tiles per query block, all four softmax groups and their
+    # merge) against the float64 map
+    flipped, total = _score_closeness(w, dump, masks, [2, 11, 20, 29])
+    print(f"config 2: {flipped} of {total} window cells decided differently from the float64 map")
+    assert flipped <= 1e-3 * total
 
 
 @pytest.mark.parametrize("gather", GATHER)
 def test_config4_varlen_masks(gather):
     w = synth.config4(lengths=(4096, 16384, 32768, 65536))
-    _build_and_check(w, qblocks=8, gather=gather)
+    blob, shape, masks, dump = _build_and_check(w, qblocks=8, gather=gather)
+    flipped, total = _score_closeness(w, dump, masks, [1, 14, 30])          # every sequence, three heads
+    print(f"config 4: {flipped} of {total} window cells decided differently from the float64 map")
+    assert flipped <= 1e-3 * total
 
 
 def test_config3_shape_masks():
@@ -222,6 +230,10 @@ def test_config3_shape_masks():
     blob, shape, masks, dump = _build_and_check(w, qblocks=8)
     st = B.dam_mask_stats(blob, shape)
     assert 0.005 <= st["tiles"] / st["causal_tiles"] <= 0.08
+    # PCL 4096: a query block sweeps up to 32 kv tiles; the map itself against the float64 map
+    flipped, total = _score_closeness(w, dump, masks, [0, 13, 26])
+    print(f"config 3: {flipped} of {total} window cells decided differently from the float64 map")
+    assert flipped <= 1e-3 * total
 
 
 def test_mask_tile_count_is_independent_of_gathering():
@@ -363,16 +375,19 @@ def test_other_amplifications_bit_exact_from_scores(transform, lam, tau):
 
 
 def test_active_element_count_matches_the_extended_mask():
-    """MaskBlob.active_elements (host arithmetic on the pattern bits, used for the element-level density of the
-    bench line) against the sum of the oracle's extended-mask rows."""
-    w = synth.small_case(0, 4, 2, 64, 96, seed=50, dtype=torch.bfloat16, lengths=[400, 150, 60])
+    """dam_mask_stats' per-(sequence, head) active-cell counts (a kernel of the library working on the pattern
+    bits) against the sum of the oracle's extended-mask rows, with and without gathered-column tile lists."""
+    w = synth.small_case(0, 4, 2, 64, 96, seed=50, dtype=torch.bfloat16, lengths=[400, 150, 60, 96, 191])
     shape = B.make_shape(w.cu_seqlens, 4, 2, 64, w.Q.dtype, DEV)
     rule = B.make_rule(96, w.tau, w.mu)
     n = sum(4 * min(S, 96) ** 2 for S in shape.lengths)
     dump = torch.zeros(n, dtype=torch.float32, device=DEV)
     blob, _ = B.dam_build_masks(w.Q.to(DEV), w.K.to(DEV), shape, rule, scores_dump=dump)
     masks = H.oracle_masks_from_dump(w, dump.cpu().numpy())
-    mb = B.MaskBlob(blob)
+    got = B.dam_mask_stats(blob, shape, active_elements=True)["active_elements"].cpu().numpy()
     for b, S in enumerate(shape.lengths):
         for h in range(4):
-            assert mb.active_elements(b, h) == int(masks[b][h].rows(list(range(S))).sum())
+            assert int(got[b, h]) == int(masks[b][h].rows(list(range(S))).sum()), (b, h)
+    # an all-ones blob has no pattern sections to count from
+    with pytest.raises(B.DamError):
+        B.dam_mask_stats(B.dam_mask_all_ones(shape, True, DEV), shape, active_elements=True)

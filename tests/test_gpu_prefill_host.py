@@ -1,10 +1,29 @@
-"""The host-buffer entry point (uploads, mask construction, attention and downloads pipelined over row chunks)
-returns exactly what the two device calls return on the same inputs."""
+"""The host-buffer entry point (uploads, mask construction, attention and downloads pipelined over row chunks):
+its O and LSE against the float64 oracle (masks from the shared fp32 score tensor), and bit for bit against the two
+device calls on the same inputs."""
+import numpy as np
 import pytest
 import torch
 
 from paper_2506_11104_b200 import binding as B
 from paper_2506_11104_b200 import synth
+from tests import helpers as H
+
+TOL = {torch.bfloat16: (2e-2, 2e-3, 1e-3), torch.float32: (1e-4, 1e-5, 1e-5)}
+
+
+def _oracle_check(w, Oh, lh, masks, causal):
+    """Sampled rows of every (sequence, head) of the host-side result against the oracle (Sec. 4.3)."""
+    mx, mn, le = TOL[w.Q.dtype]
+    for b in range(len(w.cu_seqlens) - 1):
+        S = w.cu_seqlens[b + 1] - w.cu_seqlens[b]
+        rng = np.random.default_rng(S)
+        L = min(S, w.pcl_max)
+        fixed = [0, L - 1, L, L + 1, 2 * L - 2, 2 * L - 1, S - 1, 255, 256, 2047, 2048, 4095, 4096]
+        rows = sorted(set(r for r in fixed if 0 <= r < S) | set(int(x) for x in rng.choice(S, size=min(S, 256), replace=False)))
+        for h in range(w.num_q_heads):
+            e = H.attention_errors(Oh, lh, w, masks, b, h, rows, causal=causal)
+            assert e[0] <= mx and e[1] <= mn and e[2] <= le, (b, h, e)
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -22,7 +41,9 @@ def test_prefill_host_equals_device_calls(lengths, Hq, Hkv, d, dtype, pcl, gathe
     shape = B.make_shape(w.cu_seqlens, Hq, Hkv, d, dtype, DEV)
     rule = B.make_rule(w.pcl_max, w.tau, w.mu, w.lam, w.eps, gather_columns=gather)
     Q, K, V = w.Q.to(DEV), w.K.to(DEV), w.V.to(DEV)
-    blob, _ = B.dam_build_masks(Q, K, shape, rule)
+    dump = torch.zeros(sum(Hq * min(S, pcl) ** 2 for S in lengths), dtype=torch.float32, device=DEV)
+    blob, _ = B.dam_build_masks(Q, K, shape, rule, scores_dump=dump)
+    masks = H.oracle_masks_from_dump(w, dump.cpu().numpy())
     # (the masks keep no key beyond the query either way, so a chunk never needs keys past its end)
     O, lse, scratch = B.dam_sparse_attention(Q, K, V, blob, shape, causal=causal)
     assert B.dam_poll_status(blob) == 0 and B.dam_poll_status(scratch) == 0
@@ -31,8 +52,10 @@ def test_prefill_host_equals_device_calls(lengths, Hq, Hkv, d, dtype, pcl, gathe
     lh = torch.full(tuple(lse.shape), 7.0, dtype=torch.float32).pin_memory()
     n = B.dam_prefill_host(Qh, Kh, Vh, shape, rule, Oh, lh, None, DEV)
     ws = torch.empty(n, dtype=torch.uint8, device=DEV)
-    for _ in range(2):                                            # the second call reuses the workspace
+    for it in range(2):                                           # the second call reuses the workspace
         B.dam_prefill_host(Qh, Kh, Vh, shape, rule, Oh, lh, ws, DEV, causal=causal)
+        if it == 0:
+            _oracle_check(w, Oh, lh, masks, causal)
         assert torch.equal(Oh.view(torch.uint8), O.cpu().view(torch.uint8))
         assert torch.equal(lh.view(torch.uint8), lse.cpu().view(torch.uint8))
         Oh.fill_(7.0); lh.fill_(7.0)
