@@ -215,6 +215,169 @@ def decode_leg(dev, num_seqs=64, capacity=32768, pcl=2048, iters=16):
                          "requested_gbs": round(keys_all * row_bytes / (us * 1e-6) / 1e9, 1)}}
 
 
+def per_head_listed_tiles(mask, Hq):
+    """Listed (non-padding) entries of tiles[] per query head, read from the blob on the device."""
+    from paper_2506_11104_b200 import binding as B
+    hdr = np.frombuffer(mask[:256].cpu().numpy().tobytes(), dtype=B._HDR)[0]
+    off_tiles, cap_head = int(hdr["off_tiles"]), int(hdr["head_tile_cap"])
+    t = mask[off_tiles: off_tiles + 4 * Hq * cap_head].view(torch.int32).view(Hq, cap_head)
+    return (t != 0).sum(dim=1).cpu().numpy()
+
+
+def run_config(cfg, steps, warmup, gather, rank, world, local_rank, dev, pk, B, want_dense, long_warm=True):
+    """Times `steps` layers of configuration `cfg` (stage 1 + stage 2 per step) and returns the figures of one
+    benchmark line: executed-tile FLOPs over whole-step device time, per-stage times, densities, roofline."""
+    import torch.distributed as dist
+    n_distinct = {1: 32, 2: 32, 3: 2, 4: 1}[cfg]
+    n_layers = min(n_distinct, steps + warmup)
+    layers = [make_layer(cfg, l, dev) for l in layer_ids_for_rank(rank, n_layers)]
+    w0 = layers[0]
+    shape = B.make_shape(w0.cu_seqlens, w0.num_q_heads, w0.num_kv_heads, w0.head_dim, w0.Q.dtype, dev)
+    rule = B.make_rule(w0.pcl_max, w0.tau, w0.mu, w0.lam, w0.eps, gather_columns=gather)
+    rule_plain = B.make_rule(w0.pcl_max, w0.tau, w0.mu, w0.lam, w0.eps, gather_columns=False)
+    mb, sb, ab = B.dam_mask_sizes(shape, rule)
+    mbp, sbp, _ = B.dam_mask_sizes(shape, rule_plain)
+    mask = torch.empty(max(mb, mbp), dtype=torch.uint8, device=dev)
+    bscr = torch.empty(max(sb, sbp), dtype=torch.uint8, device=dev)
+    ascr = torch.empty(max(256, ab), dtype=torch.uint8, device=dev)
+    O = torch.empty_like(w0.Q)
+    lse = torch.empty(w0.num_q_heads, shape.c.total_tokens, dtype=torch.float32, device=dev)
+
+    def step(l, ev=None):
+        w = layers[l % n_layers]
+        if ev:
+            ev[0].record()
+        B.dam_build_masks(w.Q, w.K, shape, rule, mask, bscr)
+        if ev:
+            ev[1].record()
+        B.dam_sparse_attention(w.Q, w.K, w.V, mask, shape, True, 0.0, O, lse, ascr)
+        if ev:
+            ev[2].record()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(3, warmup)):
+        step(i)
+    torch.cuda.synchronize()
+    assert B.dam_poll_status(mask) == 0 and B.dam_poll_status(ascr) == 0
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    if long_warm:
+        # a longer loaded stretch before the timed region so that the clock sampler sees the GPU under this load
+        t_end = time.perf_counter() + 1.0
+        i = 0
+        while time.perf_counter() < t_end:
+            step(i)
+            i += 1
+            if i % 8 == 0:
+                torch.cuda.synchronize()
+
+    # ---- timed region: exactly `steps` steps, device-timed, per-stage events inside
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    start.record()
+    for i in range(steps):
+        step(warmup + i, evs[i])
+    end.record()
+    barrier()
+    clocks = sampler.stop()
+    total_ms = start.elapsed_time(end)
+    assert B.dam_poll_status(mask) == 0 and B.dam_poll_status(ascr) == 0
+    s1 = [e[0].elapsed_time(e[1]) for e in evs]
+    s2 = [e[1].elapsed_time(e[2]) for e in evs]
+
+    # ---- statistics of the timed layers (outside the timed region: rebuild and read the blob)
+    timed = sorted(set((warmup + i) % n_layers for i in range(steps)))
+    Hq = w0.num_q_heads
+    per_layer, head_exec, head_mask, elem_nnz = {}, [], [], {}
+    for l in timed:
+        w = layers[l]
+        B.dam_build_masks(w.Q, w.K, shape, rule, mask, bscr)
+        st = B.dam_mask_stats(mask, shape, active_elements=True)
+        elem_nnz[l] = int(st.pop("active_elements").sum().item())
+        per_layer[l] = st
+        head_exec.append(per_head_listed_tiles(mask, Hq))
+        if gather:
+            B.dam_build_masks(w.Q, w.K, shape, rule_plain, mask, bscr)      # tiles of the masks themselves, per head
+            head_mask.append(per_head_listed_tiles(mask, Hq))
+        else:
+            head_mask.append(head_exec[-1])
+    causal_tiles = per_layer[timed[0]]["causal_tiles"]
+    causal_head = causal_tiles / Hq
+    hm = np.concatenate(head_mask) / causal_head
+    he = np.concatenate(head_exec) / causal_head
+    flops_tile = 4.0 * TILE * TILE * w0.head_dim
+    step_tiles = [per_layer[(warmup + i) % n_layers]["tiles"] for i in range(steps)]
+    step_mask_tiles = [per_layer[(warmup + i) % n_layers]["mask_tiles"] for i in range(steps)]
+    total_ms_max, flops_exec = aggregate_over_ranks(total_ms, flops_tile * sum(step_tiles), world, dev)
+    _, flops_mask = aggregate_over_ranks(total_ms, flops_tile * sum(step_mask_tiles), world, dev)
+    _, flops_elem = aggregate_over_ranks(total_ms, 4.0 * w0.head_dim * sum(elem_nnz[(warmup + i) % n_layers] for i in range(steps)),
+                                         world, dev)
+    sec = total_ms_max * 1e-3
+    causal_elems = sum(S * (S + 1) // 2 for S in shape.lengths) * Hq
+
+    # ---- roofline of the dominant kernel (sparse attention incl. the column gather), from the per-launch events
+    attn_ms = sum(s2) / len(s2)
+    attn_tflops = flops_tile * (sum(step_tiles) / len(step_tiles)) / (attn_ms * 1e-3) / 1e12
+    roof = {"bound": "tensor", "kernel": "attn_sm100_kernel", "achieved": round(attn_tflops, 2), "peak": pk["bf16"],
+            "peak_kind": f"cuBLAS bf16 burst, {pk['which']} (the attention call is timed by itself, {attn_ms:.2f} ms per launch)",
+            "unit": "TFLOP/s", "frac": round(attn_tflops / pk["bf16"], 4),
+            "frac_of_sustained": round(attn_tflops / (pk["bf16_sustained"] or pk["bf16"]), 4),
+            "frac_of_nominal_2250": round(attn_tflops / 2250.0, 4),
+            "sm_mhz_sampled": clocks.get("sm_mhz"),
+            "algorithmic_flops_per_launch": flops_tile * (sum(step_tiles) / len(step_tiles)),
+            "traffic": measured_traffic("attn_sm100_kernel", cfg) if gather else None,
+            "avg_launch_ms": round(attn_ms, 4)}
+    res = {"value": round(flops_exec / sec / 1e12, 3), "ms_per_step": round(total_ms_max / steps, 4),
+           "stage1_ms": round(sum(s1) / len(s1), 4), "stage2_ms": round(attn_ms, 4),
+           "value_definition": "4*128*128*d FLOP per tile the attention kernel executed (listed tiles), over the device "
+                               "time of the whole steps (stage 1 + stage 2)",
+           "effective_mask_tile_tflops": round(flops_mask / sec / 1e12, 3),
+           "effective_mask_tile_definition": "4*128*128*d per 128x128 tile of the masks that holds an active cell (more "
+                                             "than the kernel executes when matched columns are served by gathered tiles)",
+           "element_active_tflops": round(flops_elem / sec / 1e12, 3),
+           "element_density": round(sum(elem_nnz.values()) / len(elem_nnz) / causal_elems, 5),
+           "tile_density": round(sum(step_mask_tiles) / len(step_mask_tiles) / causal_tiles, 4),
+           "executed_tile_density": round(sum(step_tiles) / len(step_tiles) / causal_tiles, 4),
+           "tile_density_per_layer_min_max": [round(min(step_mask_tiles) / causal_tiles, 4),
+                                              round(max(step_mask_tiles) / causal_tiles, 4)],
+           "tile_density_per_head": {"heads": int(hm.size), "min": round(float(hm.min()), 4),
+                                     "median": round(float(np.median(hm)), 4), "max": round(float(hm.max()), 4),
+                                     "executed_min": round(float(he.min()), 4), "executed_median": round(float(np.median(he)), 4),
+                                     "executed_max": round(float(he.max()), 4)},
+           "roofline": roof, "clocks": clocks, "distinct_layers": n_layers,
+           "gpu_launches": (8 if gather else 7) * steps}      # init, score, counts, match, classify, order, [gather], attention
+    if want_dense and rank == 0:
+        # the build's own dense causal attention at the same length (all tiles listed as fully active)
+        dmb, _, _ = B.dam_mask_sizes(shape, None, True)
+        dmask = torch.empty(dmb, dtype=torch.uint8, device=dev)
+        B.dam_mask_all_ones(shape, True, dev, dmask)
+        for _ in range(2):
+            B.dam_sparse_attention(w0.Q, w0.K, w0.V, dmask, shape, True, 0.0, O, lse, ascr)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        nd = 3 if cfg != 3 else 1
+        e0.record()
+        for i in range(nd):
+            w = layers[i % n_layers]
+            B.dam_sparse_attention(w.Q, w.K, w.V, dmask, shape, True, 0.0, O, lse, ascr)
+        e1.record()
+        torch.cuda.synchronize()
+        dense_ms = e0.elapsed_time(e1) / nd
+        res["dense_causal"] = {"ms": round(dense_ms, 3), "tflops": round(flops_tile * causal_tiles / (dense_ms * 1e-3) / 1e12, 1),
+                               "frac_of_burst": round(flops_tile * causal_tiles / (dense_ms * 1e-3) / 1e12 / pk["bf16"], 4),
+                               "speedup_sparse_stage2": round(dense_ms / attn_ms, 2),
+                               "speedup_sparse_layer": round(dense_ms / (total_ms_max / steps), 2)}
+        del dmask
+    ctx = dict(layers=layers, shape=shape, rule=rule, w0=w0, lse=lse, per_layer=per_layer, n_layers=n_layers,
+               flops_tile=flops_tile, barrier=barrier)
+    return res, ctx
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -226,6 +389,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-dense", action="store_true")
     ap.add_argument("--no-decode", action="store_true", help="skip the generation-time (KV cache) measurement")
+    ap.add_argument("--no-configs", action="store_true", help="skip the short runs of the other configurations")
     ap.add_argument("--only-decode", type=int, default=0, metavar="SEQS",
                     help="run only the generation-time measurement on SEQS sequences and print its object (for profiling)")
     ap.add_argument("--no-gather", action="store_true", help="list one tile per matched column stripe instead of gathered-column tiles")
@@ -258,181 +422,72 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
     pk = peaks()
     cfg = args.config
-    n_distinct = {1: 32, 2: 32, 3: 2, 4: 1}[cfg]
-    n_layers = min(n_distinct, args.steps + args.warmup)
-    # each rank owns its own layers (independent problems: no data-path collective)
-    layers = [make_layer(cfg, l, dev) for l in layer_ids_for_rank(rank, n_layers)]
-    w0 = layers[0]
-    shape = B.make_shape(w0.cu_seqlens, w0.num_q_heads, w0.num_kv_heads, w0.head_dim, w0.Q.dtype, dev)
-    rule = B.make_rule(w0.pcl_max, w0.tau, w0.mu, w0.lam, w0.eps, gather_columns=not args.no_gather)
-    mb, sb, ab = B.dam_mask_sizes(shape, rule)
-    mask = torch.empty(mb, dtype=torch.uint8, device=dev)
-    bscr = torch.empty(sb, dtype=torch.uint8, device=dev)
-    ascr = torch.empty(max(256, ab), dtype=torch.uint8, device=dev)
-    O = torch.empty_like(w0.Q)
-    lse = torch.empty(w0.num_q_heads, shape.c.total_tokens, dtype=torch.float32, device=dev)
+    gather = not args.no_gather
+    res, ctx = run_config(cfg, args.steps, args.warmup, gather, rank, world, local_rank, dev, pk, B, not args.no_dense)
+    layers, shape, rule, w0, lse = ctx["layers"], ctx["shape"], ctx["rule"], ctx["w0"], ctx["lse"]
+    per_layer, n_layers, flops_tile, barrier = ctx["per_layer"], ctx["n_layers"], ctx["flops_tile"], ctx["barrier"]
 
-    def step(l, ev=None):
-        w = layers[l % n_layers]
-        if ev:
-            ev[0].record()
-        B.dam_build_masks(w.Q, w.K, shape, rule, mask, bscr)
-        if ev:
-            ev[1].record()
-        B.dam_sparse_attention(w.Q, w.K, w.V, mask, shape, True, 0.0, O, lse, ascr)
-        if ev:
-            ev[2].record()
-
-    def barrier():
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    for i in range(max(3, args.warmup)):
-        step(i)
-    torch.cuda.synchronize()
-    assert B.dam_poll_status(mask) == 0 and B.dam_poll_status(ascr) == 0
-    # a longer loaded stretch before the timed region so that the clock sampler sees the GPU under this load
-    sampler = ClockSampler(local_rank)
-    sampler.start()
-    t_end = time.perf_counter() + 1.0
-    i = 0
-    while time.perf_counter() < t_end:
-        step(i)
-        i += 1
-        if i % 8 == 0:
-            torch.cuda.synchronize()
-
-    # ---- timed region: exactly K steps, device-timed, per-stage events inside
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
-    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    start.record()
-    for i in range(args.steps):
-        step(args.warmup + i, evs[i])
-    end.record()
-    barrier()
-    clocks = sampler.stop()
-    total_ms = start.elapsed_time(end)
-    assert B.dam_poll_status(mask) == 0 and B.dam_poll_status(ascr) == 0
-    s1 = [e[0].elapsed_time(e[1]) for e in evs]
-    s2 = [e[1].elapsed_time(e[2]) for e in evs]
-    # tile statistics per timed layer (outside the timed region: rebuild and read the header)
-    per_layer_stats = {}
-    for l in sorted(set((args.warmup + i) % n_layers for i in range(args.steps))):
-        w = layers[l]
-        B.dam_build_masks(w.Q, w.K, shape, rule, mask, bscr)
-        per_layer_stats[l] = B.dam_mask_stats(mask, shape)
-    flops_tile = 4.0 * TILE * TILE * w0.head_dim
-    # executed tiles (what the tensor cores ran) and mask tiles (128 x 128 tiles of the masks with an active
-    # cell; the two differ when matched columns are served by gathered-column tiles)
-    # element-level density of one layer's masks (host arithmetic on the pattern bits: the paper's O(s L) figure)
-    elem = None
-    if rank == 0:
-        nnz = int(B.dam_mask_stats(mask, shape, active_elements=True)["active_elements"].sum().item())
-        causal_elems = sum(S * (S + 1) // 2 for S in shape.lengths) * w0.num_q_heads
-        elem = {"layer": int(l), "density": round(nnz / causal_elems, 5), "flops": 4.0 * w0.head_dim * nnz}
-    step_tiles = [per_layer_stats[(args.warmup + i) % n_layers]["tiles"] for i in range(args.steps)]
-    step_mask_tiles = [per_layer_stats[(args.warmup + i) % n_layers]["mask_tiles"] for i in range(args.steps)]
-    total_flops = flops_tile * sum(step_mask_tiles)
-    causal_tiles = per_layer_stats[next(iter(per_layer_stats))]["causal_tiles"]
-    total_ms_max, flops_all = aggregate_over_ranks(total_ms, total_flops, world, dev)
-    value = flops_all / (total_ms_max * 1e-3) / 1e12
-
-    # ---- roofline of the dominant kernel (sparse attention), from the per-launch events
-    attn_ms = sum(s2) / len(s2)
-    attn_tflops = flops_tile * (sum(step_tiles) / len(step_tiles)) / (attn_ms * 1e-3) / 1e12
-    peak = pk["bf16_sustained"] or pk["bf16"]
-    roof = {"bound": "tensor", "kernel": "attn_sm100_kernel", "achieved": round(attn_tflops, 2), "peak": peak,
-            "peak_kind": f"sustained cuBLAS bf16, {pk['which']}", "unit": "TFLOP/s", "frac": round(attn_tflops / peak, 4),
-            "frac_of_burst": round(attn_tflops / pk["bf16"], 4), "traffic": None if args.no_gather else measured_traffic("attn_sm100_kernel", cfg),   # captured with gathered tiles
-            "avg_launch_ms": round(attn_ms, 4)}
-
-    out = {"metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
-           "warmup": args.warmup, "ms_per_step": round(total_ms_max / args.steps, 4), "higher_is_better": True,
+    out = {"metric": METRIC, "value": res.pop("value"), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+           "warmup": args.warmup, "ms_per_step": res.pop("ms_per_step"), "higher_is_better": True,
            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
            "config": {"workload": workload_name(cfg), "pcl": w0.pcl_max, "tau": w0.tau, "mu": w0.mu,
                       "l2": "inputs larger than L2: every step reads a different layer's Q/K/V (384 MiB at C2)",
-                      "distinct_layers": n_layers, "gathered_column_tiles": not args.no_gather},
-           "stage1_ms": round(sum(s1) / len(s1), 4), "stage2_ms": round(attn_ms, 4),
-           "active_flops": "4*128*128*d per 128x128 tile of the mask that holds an active cell",
-           "tile_density": round(sum(step_mask_tiles) / len(step_mask_tiles) / causal_tiles, 4),
-           "tile_density_min_max": [round(min(step_mask_tiles) / causal_tiles, 4),
-                                    round(max(step_mask_tiles) / causal_tiles, 4)],
-           "executed_tile_density": round(sum(step_tiles) / len(step_tiles) / causal_tiles, 4),
-           "executed_tflops": round(flops_tile * sum(step_tiles) / (total_ms_max * 1e-3) / 1e12 * world, 3),
-           "element_active": (None if elem is None else
-                              {"layer": elem["layer"], "element_density": elem["density"],
-                               "tflops": round(elem["flops"] / (total_ms_max / args.steps * 1e-3) / 1e12, 3),
-                               "flops": "4*d per active cell of the masks (one layer, at the mean layer time)"}),
-           "roofline": roof, "clocks": clocks, "gpu_launches": (8 if not args.no_gather else 7) * args.steps}   # init, score, counts, match, classify, order, [gather], attention
-
-    if rank == 0 and not args.no_dense:
-        # the build's own dense causal attention at the same length (all tiles listed as fully active)
-        dmb, _, _ = B.dam_mask_sizes(shape, None, True)
-        dmask = torch.empty(dmb, dtype=torch.uint8, device=dev)
-        B.dam_mask_all_ones(shape, True, dev, dmask)
-        for _ in range(2):
-            B.dam_sparse_attention(w0.Q, w0.K, w0.V, dmask, shape, True, 0.0, O, lse, ascr)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        nd = 3
-        e0.record()
-        for i in range(nd):
-            w = layers[i % n_layers]
-            B.dam_sparse_attention(w.Q, w.K, w.V, dmask, shape, True, 0.0, O, lse, ascr)
-        e1.record()
-        torch.cuda.synchronize()
-        dense_ms = e0.elapsed_time(e1) / nd
-        out["dense_causal"] = {"ms": round(dense_ms, 3), "tflops": round(flops_tile * causal_tiles / (dense_ms * 1e-3) / 1e12, 1),
-                               "speedup_sparse_stage2": round(dense_ms / attn_ms, 2),
-                               "speedup_sparse_layer": round(dense_ms / (total_ms_max / args.steps), 2)}
-        del dmask
+                      "distinct_layers": res.pop("distinct_layers"), "gathered_column_tiles": gather,
+                      "tile_density_per_head": res.pop("tile_density_per_head")}}
+    out.update(res)
 
     if rank == 0 and world == 1 and not args.no_decode:
         out["decode"] = decode_leg(dev)
 
     if not args.no_e2e:
-        # end to end through the host-buffer entry point: H2D of Q, K, V and D2H of O, LSE inside the timed region
+        # end to end through the host-buffer entry point: H2D of Q, K, V and D2H of O, LSE inside the timed region;
+        # the layers are the first timed ones, so that their executed-tile counts are the measured ones
         n_e2e = min(args.steps, 4)
-        hosts = []
-        for l in range(min(n_layers, n_e2e)):
-            w = layers[l]
-            hosts.append(tuple(x.cpu().pin_memory() for x in (w.Q, w.K, w.V)))
+        e2e_layers = [(args.warmup + i) % n_layers for i in range(n_e2e)]
+        hosts = [tuple(x.cpu().pin_memory() for x in (layers[l].Q, layers[l].K, layers[l].V)) for l in e2e_layers]
         Oh = torch.empty(w0.Q.shape, dtype=w0.Q.dtype).pin_memory()
         lh = torch.empty(lse.shape, dtype=torch.float32).pin_memory()
         nbytes = B.dam_prefill_host(hosts[0][0], hosts[0][1], hosts[0][2], shape, rule, Oh, lh, None, dev)
         ws = torch.empty(nbytes, dtype=torch.uint8, device=dev)
         B.dam_prefill_host(hosts[0][0], hosts[0][1], hosts[0][2], shape, rule, Oh, lh, ws, dev)
         barrier()
-        t0 = time.perf_counter()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        for i in range(n_e2e):
-            q, k, v = hosts[i % len(hosts)]
+        for q, k, v in hosts:
             B.dam_prefill_host(q, k, v, shape, rule, Oh, lh, ws, dev)
         e1.record()
         barrier()
-        e2e_ms = e0.elapsed_time(e1)
-        te = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(te, op=dist.ReduceOp.MAX)
-        e2e_flops = flops_tile * sum(per_layer_stats.get(i % n_layers, per_layer_stats[next(iter(per_layer_stats))])["mask_tiles"]
-                                     for i in range(n_e2e)) * world
+        e2e_ms, e2e_flops = aggregate_over_ranks(e0.elapsed_time(e1), flops_tile * sum(per_layer[l]["tiles"] for l in e2e_layers),
+                                                 world, dev)
         es = w0.Q.element_size()
-        out["e2e"] = {"value": round(e2e_flops / (float(te.item()) * 1e-3) / 1e12, 3), "unit": UNIT,
-                      "ms_per_step": round(float(te.item()) / n_e2e, 3), "steps": n_e2e,
+        out["e2e"] = {"value": round(e2e_flops / (e2e_ms * 1e-3) / 1e12, 3), "unit": UNIT,
+                      "ms_per_step": round(e2e_ms / n_e2e, 3), "steps": n_e2e, "layers": e2e_layers,
                       "h2d_bytes_per_step": int((w0.Q.numel() + w0.K.numel() + w0.V.numel()) * es),
                       "d2h_bytes_per_step": int(w0.Q.numel() * es + lse.numel() * 4),
-                      "api": "dam_prefill_host (pinned host buffers in and out)"}
+                      "api": "dam_prefill_host (pinned host buffers in and out); executed-tile FLOPs of the layers it ran"}
         del ws, hosts
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        layer_s, info = oracle_sample(layers[args.warmup % n_layers], n_rows=6144, heads=tuple(range(w0.num_q_heads)))
         l = args.warmup % n_layers
-        info["value"] = round(flops_tile * per_layer_stats.get(l, next(iter(per_layer_stats.values())))["mask_tiles"] / layer_s / 1e12, 6)
+        layer_s, info = oracle_sample(layers[l], n_rows=6144, heads=tuple(range(w0.num_q_heads)))
+        info["value"] = round(flops_tile * per_layer[l]["tiles"] / layer_s / 1e12, 6)
         info["unit"] = UNIT
         out["cpu_baseline"] = info
+
+    del layers, ctx
+    torch.cuda.empty_cache()
+    if rank == 0 and world == 1 and not args.no_configs:
+        # the other full-size configurations, one short run each, same fields
+        others = {}
+        for c in (1, 3, 4):
+            if c == cfg:
+                continue
+            r, cx = run_config(c, 8 if c != 3 else 4, 3, gather, rank, world, local_rank, dev, pk, B, c != 3, long_warm=False)
+            r["workload"] = workload_name(c)
+            others[f"C{c}"] = r
+            del cx
+            torch.cuda.empty_cache()
+        out["configs"] = others
 
     if rank == 0:
         print(json.dumps(out))

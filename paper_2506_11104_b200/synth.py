@@ -148,14 +148,15 @@ def make_sequence(S: int, Hq: int, Hkv: int, d: int, pcl: int, plans: Sequence[H
 
 
 def _draw_plans(Hq: int, pcl: int, seed_words, band_m_choices: Sequence[int], max_stripes: int,
-                sink_prob: float = 1.0) -> List[HeadPlan]:
+                sink_prob: float = 1.0, stripe_span: float = 0.5, stripe_skew: float = 1.0) -> List[HeadPlan]:
     gen = _gen(list(seed_words) + [7777], "cpu")
     plans = []
     for h in range(Hq):
         u = torch.rand(4, generator=gen)
         bm = band_m_choices[int(u[0] * len(band_m_choices)) % len(band_m_choices)]
-        ns = int(u[1] * (max_stripes + 1)) % (max_stripes + 1)
-        pos = torch.randperm(max(1, pcl // 2 - 1), generator=gen)[:ns] + 1     # stripes inside the first half
+        ns = int(float(u[1]) ** stripe_skew * (max_stripes + 1)) % (max_stripes + 1)   # skew > 1: mostly few, sometimes many
+        # stripes inside the first `stripe_span` of the window (0.5: the first half)
+        pos = torch.randperm(max(1, int(pcl * stripe_span) - 1), generator=gen)[:ns] + 1
         plans.append(HeadPlan(sink=bool(u[2] < sink_prob), band_m=int(bm), stripes=sorted(int(p) for p in pos)))
     return plans
 
@@ -191,23 +192,32 @@ def config0(device="cpu") -> Workload:
 
 
 def llama_layer(S: int, pcl: int, cfg: int, layer: int = 0, device="cpu", band_m_choices=(0, 2, 3, 4, 6, 8, 12, 16, 24, 40),
-                max_stripes: int = 16, dtype=torch.bfloat16, name: Optional[str] = None) -> Workload:
-    """Llama-3-8B-shaped layer: 32 query heads, 8 KV heads, d 128, one sequence of S tokens."""
+                max_stripes: int = 16, dtype=torch.bfloat16, name: Optional[str] = None, sink_prob: float = 1.0,
+                stripe_span: float = 0.5, stripe_skew: float = 1.0, lone_stripe_heads: Sequence[int] = ()) -> Workload:
+    """Llama-3-8B-shaped layer: 32 query heads, 8 KV heads, d 128, one sequence of S tokens.
+    `lone_stripe_heads`: heads that attend to their first one or two stripe keys only (the sparsest masks)."""
     Hq, Hkv, d = 32, 8, 128
     r = CONFIG_RULE[cfg]
-    plans = _draw_plans(Hq, pcl, [0, cfg, layer, 0], band_m_choices, max_stripes)
+    plans = _draw_plans(Hq, pcl, [0, cfg, layer, 0], band_m_choices, max_stripes, sink_prob, stripe_span, stripe_skew)
+    for k, h in enumerate(lone_stripe_heads):
+        keys = plans[h].stripes[:1 + k % 2] or [pcl // 3 + 7 * k]
+        plans[h] = HeadPlan(sink=False, band_m=0, stripes=keys)
     seq = make_sequence(S, Hq, Hkv, d, pcl, plans, r["amp"], [0, cfg, layer, 0], device)
     return _pack(name or f"C{cfg} layer {layer} S={S} PCL={pcl}", [seq], [0, S], pcl, r["tau"], r["mu"], dtype, [plans])
 
 
 def config1(device="cpu") -> Workload:
-    return llama_layer(8192, 1024, 1, 0, device)
+    """Heads from a lone stripe or sink (a few per cent of the causal tiles) to the widest band the threshold
+    keeps plus stripes all over the window (about 40 %)."""
+    return llama_layer(8192, 1024, 1, 0, device, band_m_choices=(0, 0, 2, 2, 3, 4, 6, 8, 12, 16, 24, 40), max_stripes=32,
+                       sink_prob=0.8, stripe_span=0.95, stripe_skew=3.0, lone_stripe_heads=(3, 14, 25))
 
 
 def config2_layer(layer: int, device="cpu", S: int = 32768, pcl: int = 2048) -> Workload:
     """One layer of the 32-layer stack; the band/stripe mix is re-drawn per layer."""
-    choices = [(2, 3, 4, 6), (8, 12, 16, 24, 40), (2, 4, 8, 16, 40), (24, 40)][layer % 4]
-    return llama_layer(S, pcl, 2, layer, device, band_m_choices=choices, max_stripes=(4, 16, 8, 2)[layer % 4])
+    choices = [(0, 2, 2, 3, 4, 6), (0, 8, 12, 16, 24, 40), (2, 2, 4, 8, 16, 40), (0, 0, 24, 40)][layer % 4]
+    return llama_layer(S, pcl, 2, layer, device, band_m_choices=choices, max_stripes=(8, 40, 64, 2)[layer % 4],
+                       sink_prob=0.85, stripe_span=0.95, stripe_skew=(1.0, 1.0, 0.5, 1.0)[layer % 4])
 
 
 def config3(device="cpu", S: int = 131072, pcl: int = 4096) -> Workload:

@@ -391,3 +391,25 @@ def test_active_element_count_matches_the_extended_mask():
     # an all-ones blob has no pattern sections to count from
     with pytest.raises(B.DamError):
         B.dam_mask_stats(B.dam_mask_all_ones(shape, True, DEV), shape, active_elements=True)
+
+
+def _per_head_tile_density(w):
+    shape, rule = _shape(w), _rule(w)
+    blob, _ = B.dam_build_masks(w.Q.to(DEV), w.K.to(DEV), shape, rule)
+    mb = B.MaskBlob(blob)
+    Hq, cap = int(mb.hdr["num_q_heads"]), int(mb.hdr["head_tile_cap"])
+    listed = (mb.tiles.reshape(Hq, cap) != 0).sum(axis=1)
+    return listed / (int(mb.hdr["causal_tiles"]) / Hq)
+
+
+def test_per_head_densities_are_heterogeneous():
+    """The planted-pattern draw gives per-head tile densities (tiles with an active cell over causal tiles) that
+    span what the configurations ask for: a few per cent to about 40 % over the heads of the 8192-token layer, about
+    1 % to the cap the threshold allows (a row keeps at most 1 / p* = 1587 keys at tau 0.05, so a band is at most a
+    dozen tiles wide next to the 16 column tiles of the window) over the heads of the 32-layer stack."""
+    d1 = _per_head_tile_density(synth.config1(DEV))
+    assert d1.min() <= 0.06 and d1.max() >= 0.33 and 0.15 <= np.median(d1) <= 0.33, (d1.min(), np.median(d1), d1.max())
+    d2 = np.concatenate([_per_head_tile_density(synth.config2_layer(l, DEV)) for l in (2, 3, 4, 5)])
+    assert d2.min() <= 0.025 and d2.max() >= 0.15 and d2.max() <= 0.30, (d2.min(), d2.max())
+    # heads of one layer differ by a large factor, which is what the longest-first work list has to balance
+    assert d2.max() / d2.min() >= 6
