@@ -205,7 +205,7 @@ def decode_leg(dev, num_seqs=64, capacity=32768, pcl=2048, iters=16):
             "us_per_launch": round(us, 1), "tokens_per_s": round(num_seqs / (us * 1e-6)),
             "keys_per_query_head": round(keys_all / (num_seqs * Hq), 1),
             "unique_keys_per_kv_head": round(keys_unique / (num_seqs * Hkv), 1),
-            "roofline": {"bound": "hbm", "kernel": "decode_kernel", "achieved": round(gbs, 1), "peak": peak,
+            "roofline": {"bound": "hbm", "kernel": "decode_group_kernel", "achieved": round(gbs, 1), "peak": peak,
                          "peak_kind": "copy bandwidth, " + pk["which"], "unit": "GB/s", "frac": round(gbs / peak, 4),
                          "traffic": (lambda t: int(t * num_seqs) if t else None)(
                              (json.load(open(os.path.join(ROOT, "profiles", "traffic.json")))

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdam_b200.so")
 SOURCES = ["dam_api.cu", "dam_mask_kernels.cu", "dam_ref_kernels.cu", "dam_attn_sm100.cu", "dam_score_sm100.cu", "dam_static_scratch.cu",
-           "dam_decode_kernels.cu"]
+           "dam_decode_kernels.cu", "dam_decode_mma.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-ffp-contract=off", "--fmad=true", "-cudart", "static"]
 

@@ -281,6 +281,9 @@ decode_kernel(const T* __restrict__ q, const T* __restrict__ K, const T* __restr
 
 cudaError_t dam_launch_decode(const void* q, const void* K, const void* V, const void* blob, const dam_shape_t* s,
                               const int32_t* pos_dev, float scale, void* O, float* lse, void* scratch, cudaStream_t st) {
+  // bf16 with a GQA group of at most 8 heads: one block per (sequence, KV head) on the tensor cores
+  const cudaError_t ge = dam_launch_decode_group(q, K, V, blob, s, pos_dev, scale, O, lse, scratch, st);
+  if (ge != cudaErrorNotSupported) return ge;
   const dim3 grid((unsigned)s->num_q_heads, (unsigned)s->num_seqs);
   const int group = s->num_q_heads / s->num_kv_heads;
   const float sl2 = scale * 1.4426950408889634f;

@@ -226,7 +226,7 @@ class DamDeviceTable {
   struct Slot { bool filled; DamDeviceInfo info; bool done[kMaxSetups]; };
   Slot slots_[kMaxDevices] = {};
 };
-enum { DAM_SETUP_ATTN_SMEM = 0, DAM_SETUP_SCORE_SMEM = 1 };
+enum { DAM_SETUP_ATTN_SMEM = 0, DAM_SETUP_SCORE_SMEM = 1, DAM_SETUP_DECODE_SMEM = 2 };
 
 DamDeviceTable& dam_device_table();                                       // the library's own table
 cudaError_t dam_current_device(int* device, DamDeviceInfo* info);         // ordinal and record of the current device
@@ -276,6 +276,8 @@ cudaError_t dam_launch_capture_accumulate(const float* P, const dam_shape_t* sha
                                           cudaStream_t st);
 cudaError_t dam_launch_capture_average(const float* A, const int32_t* C, int Lmax, float eps, const dam_shape_t* shape,
                                        float* P_out, cudaStream_t st);
+cudaError_t dam_launch_decode_group(const void* q, const void* K, const void* V, const void* blob, const dam_shape_t* shape,
+                                    const int32_t* pos_dev, float scale, void* O, float* lse, void* scratch, cudaStream_t st);
 cudaError_t dam_launch_decode(const void* q, const void* K, const void* V, const void* blob, const dam_shape_t* shape,
                               const int32_t* pos_dev, float scale, void* O, float* lse, void* scratch, cudaStream_t st);
 

@@ -70,6 +70,9 @@ def _decode_and_check(w, blob, masks, positions):
     ([1024, 700], [512, 700], 8, 2, 128, torch.bfloat16, 128),
     ([900], [300], 4, 1, 64, torch.bfloat16, 96),
     ([640, 640, 130], [640, 200, 130], 4, 2, 128, torch.float32, 160),
+    ([700], [700], 2, 2, 128, torch.bfloat16, 128),          # one head per KV head on the grouped tensor-core kernel
+    ([5000], [5000], 8, 1, 64, torch.bfloat16, 2112),        # eight heads per KV head; 132 pattern words: two rounds
+    ([600], [600], 16, 1, 64, torch.bfloat16, 96),           # sixteen heads per KV head: the one-head-per-block kernel
 ])
 def test_decode_matches_oracle(cache_lengths, build_lengths, Hq, Hkv, d, dtype, pcl):
     w = synth.small_case(0, Hq, Hkv, d, pcl, seed=11, dtype=dtype, lengths=cache_lengths)
