@@ -209,7 +209,7 @@ def decode_leg(dev, num_seqs=64, capacity=32768, pcl=2048, iters=16):
                          "peak_kind": "copy bandwidth, " + pk["which"], "unit": "GB/s", "frac": round(gbs / peak, 4),
                          "traffic": (lambda t: int(t * num_seqs) if t else None)(
                              (json.load(open(os.path.join(ROOT, "profiles", "traffic.json")))
-                              .get("decode_kernel", {}).get("per_sequence"))
+                              .get("decode_group_kernel", {}).get("per_sequence"))
                              if os.path.exists(os.path.join(ROOT, "profiles", "traffic.json")) else None),
                          "algorithmic_bytes": keys_unique * row_bytes,
                          "requested_gbs": round(keys_all * row_bytes / (us * 1e-6) / 1e9, 1)}}
@@ -476,6 +476,13 @@ def main():
 
     del layers, ctx
     torch.cuda.empty_cache()
+    if rank == 0 and world == 1 and gather and not args.no_configs:
+        # the same workload with one listed tile per matched-column stripe (no gathered-column tiles): more tiles, longer
+        # lists, a slower layer and a higher rate on the executed tiles
+        r, cx = run_config(cfg, 8, 3, False, rank, world, local_rank, dev, pk, B, False, long_warm=False)
+        out["no_gather"] = {k: r[k] for k in ("value", "ms_per_step", "stage1_ms", "stage2_ms", "executed_tile_density", "roofline")}
+        del cx
+        torch.cuda.empty_cache()
     if rank == 0 and world == 1 and not args.no_configs:
         # the other full-size configurations, one short run each, same fields
         others = {}
