@@ -61,7 +61,7 @@ typedef struct dam_shape_t {
   int32_t max_seqlen;             /* >= every sequence length                                       */
   int32_t num_q_heads;            /* Hq                                                             */
   int32_t num_kv_heads;           /* Hkv, Hq % Hkv == 0                                             */
-  int32_t head_dim;               /* d; multiple of 8, <= 256 (tensor-core path: bf16, d = 128)     */
+  int32_t head_dim;               /* d; multiple of 8, <= 256 (tensor-core path: bf16, d = 128 or 64) */
   int32_t dtype;                  /* dam_dtype_t of Q, K, V, O                                      */
   int64_t q_stride_tok, q_stride_head; /* elements                                                  */
   int64_t k_stride_tok, k_stride_head;
@@ -119,7 +119,7 @@ typedef enum dam_transform_t {
  * can be copied once per (sequence, head) into dense tiles of 128 keys that every such query block
  * visits as fully active tiles, instead of one mostly-empty tile per stripe. The mask content is
  * unchanged; only the tile lists differ, and dam_sparse_attention needs the larger scratch that
- * dam_mask_sizes then reports. Honoured for the tensor-core shapes (bf16, head_dim 128); ignored otherwise.
+ * dam_mask_sizes then reports. Honoured for the tensor-core shapes (bf16, head_dim 128 or 64); ignored otherwise.
  */
 #define DAM_RULE_GATHER_COLUMNS 1u
 
@@ -194,8 +194,9 @@ dam_status_t dam_mask_all_ones(const dam_shape_t* shape, int32_t causal, void* m
  * same shape; O: DEVICE, written for every token and head; lse: DEVICE float [Hq][total_tokens].
  * gqa_group must equal num_q_heads / num_kv_heads; softmax_scale 0 selects 1 / sqrt(head_dim).
  * scratch: DEVICE, >= attn_scratch_bytes, 256-byte aligned; it begins with a status word.
- * Tensor-core path (tcgen05 + TMA): dtype bf16, head_dim 128, 16-byte aligned strides; other
- * shapes run a plain CUDA-core kernel.
+ * Tensor-core path (tcgen05 + TMA): dtype bf16, head_dim 128 or 64, 16-byte aligned strides; other
+ * shapes run a plain CUDA-core kernel. (Word 4 of the scratch block, i.e. bytes 16..19, is 1 after a call the
+ * tensor-core kernel served and 0 otherwise: a hook for tests.)
  * Errors: INVALID_ARGUMENT, UNSUPPORTED, BUFFER_TOO_SMALL, CUDA; DEVICE_TIMEOUT via the status word.
  */
 dam_status_t dam_sparse_attention(const void* Q, const void* K, const void* V, const void* mask,

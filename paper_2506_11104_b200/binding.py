@@ -330,6 +330,11 @@ def dam_mask_expand_rows(mask: torch.Tensor, shape: Shape, seq: int, head: int, 
     return out
 
 
+def attention_ran_on_tensor_cores(scratch: torch.Tensor) -> bool:
+    """Test hook: word 4 of the attention scratch block says whether the tcgen05 kernel served the last call."""
+    return int(scratch[16:20].cpu().numpy().view(np.uint32)[0]) == 1
+
+
 def dam_poll_status(buf: torch.Tensor) -> int:
     return int(lib().dam_poll_status(_ptr(buf), _stream(buf.device)))
 
@@ -400,6 +405,11 @@ class MaskBlob:
         # every row owns a fixed range of tiles[]: its entries, then possibly zero entries (kind 0) as padding
         self.tiles = np.frombuffer(self.raw, dtype="<u4", count=int(self.tile_ptr[rows]),
                                    offset=int(self.hdr["off_tiles"]))
+
+    @property
+    def scored_on_tensor_cores(self) -> bool:
+        """Test hook: the window map of this blob was computed by the tcgen05 scoring kernel."""
+        return int(self.hdr["reserved"][0]) == 1
 
     def pattern_bits(self, seq: int, head: int):
         """(D, Drev, V) as uint8 [L]."""

@@ -52,7 +52,7 @@ dam_status_t check_rule(const dam_rule_t* r) {
   return DAM_OK;
 }
 
-bool sm100_shape(const dam_shape_t* s) { return s->dtype == DAM_BF16 && s->head_dim == 128; }
+bool sm100_shape(const dam_shape_t* s) { return s->dtype == DAM_BF16 && (s->head_dim == 128 || s->head_dim == 64); }
 
 // Gathered-column tiles: asked for by the rule, tensor-core shape, window small enough for the gather kernel.
 bool gather_enabled(const dam_shape_t* s, const dam_rule_t* r) {

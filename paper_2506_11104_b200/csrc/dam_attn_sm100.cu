@@ -1,4 +1,4 @@
-// Sparse flash attention on the 5th-generation tensor cores (sm_100a): bf16 inputs, head_dim 128.
+// Sparse flash attention on the 5th-generation tensor cores (sm_100a): bf16 inputs, head_dim 128 or 64.
 //
 // One persistent CTA per SM walks the work list of the mask blob.  A work item is a pair of adjacent
 // 128-row query blocks (2p, 2p+1) of one (sequence, head): two query tiles ("streams" A and B) share every
@@ -273,7 +273,9 @@ __device__ __forceinline__ float sweep_exp(uint32_t tS, const uint4& bits, float
 }
 
 // RANGED: only the work items whose first row lies in the row range of their sequence are processed.
-template <bool RANGED>
+// D: head_dim, 128 or 64.  With 64 a Q / K / V tile is one 16 KB box of the tensor maps (the slots keep their size),
+// S = Q K^T takes four MMAs instead of eight and O has 64 columns.
+template <bool RANGED, int D>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                   const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
@@ -351,9 +353,9 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         const uint32_t s = sc % kSlots, ph = (sc / kSlots) & 1u;
         if (!mbar_wait(bSlotEmpty + 8 * s, ph ^ 1u, abort_flag)) return false;
         const uint32_t dst = sSlots + s * kSlotBytes, bar = bSlotFull + 8 * s;
-        mbar_arrive_expect_tx(bar, kSlotBytes);
+        mbar_arrive_expect_tx(bar, DAM_TILE * D * 2);
         tma_load_3d(dst, tm, bar, 0, head, tok);
-        tma_load_3d(dst + 16384, tm, bar, 64, head, tok);
+        if (D == 128) tma_load_3d(dst + 16384, tm, bar, 64, head, tok);
         armed[s] = ph;
         ++sc;
         return true;
@@ -390,12 +392,12 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (skip) continue;
         if (!(ok = mbar_wait(bQEmpty, (ic & 1u) ^ 1u, abort_flag))) break;
         const int tokq = it.tok0 + it.qb0 * DAM_TILE;
-        mbar_arrive_expect_tx(bQFull, it.hasB ? 2 * kSlotBytes : kSlotBytes);
+        mbar_arrive_expect_tx(bQFull, (it.hasB ? 2 : 1) * DAM_TILE * D * 2);
         tma_load_3d(sQ, &tmQ, bQFull, 0, it.head, tokq);
-        tma_load_3d(sQ + 16384, &tmQ, bQFull, 64, it.head, tokq);
+        if (D == 128) tma_load_3d(sQ + 16384, &tmQ, bQFull, 64, it.head, tokq);
         if (it.hasB) {
           tma_load_3d(sQ + 32768, &tmQ, bQFull, 0, it.head, tokq + DAM_TILE);
-          tma_load_3d(sQ + 49152, &tmQ, bQFull, 64, it.head, tokq + DAM_TILE);
+          if (D == 128) tma_load_3d(sQ + 49152, &tmQ, bQFull, 64, it.head, tokq + DAM_TILE);
         }
         ++ic;
         const int kvh = it.head / prm.group;
@@ -427,7 +429,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       const uint32_t idesc_qk = idesc_bf16_f32(128, 128, 0);
-      const uint32_t idesc_pv = idesc_bf16_f32(128, 128, 1);
+      const uint32_t idesc_pv = idesc_bf16_f32(128, D, 1);
       uint32_t sc = 0, ic = 0, step = 0;
       uint32_t cP[2] = {0u, 0u};           // P tiles consumed per stream (phase of p_full)
       bool ok = true;
@@ -442,7 +444,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         const uint32_t a0 = dQ_lo + X * (kSlotBytes >> 4), b0 = dK_lo + slot * (kSlotBytes >> 4);
         const uint32_t d = tmem + kColS + X * 128;
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
+        for (int ks = 0; ks < D / 16; ++ks) {
           const uint32_t off = ((ks >> 2) * 16384 + (ks & 3) * 32) >> 4;
           mma_ss_lh(d, a0 + off, dQ_hi, b0 + off, dK_hi, idesc_qk, ks > 0 ? 1u : 0u);
         }
@@ -543,7 +545,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (row_valid) {
           const uint4 z = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-          for (int c = 0; c < 16; ++c) reinterpret_cast<uint4*>(orow)[c] = z;
+          for (int c = 0; c < D / 8; ++c) reinterpret_cast<uint4*>(orow)[c] = z;
           *lse_p = -CUDART_INF_F;
         }
         continue;
@@ -606,7 +608,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           const bool resc = alpha != 1.f;
           if (__any_sync(0xFFFFFFFFu, resc)) {
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < D / 32; ++c) {
               uint32_t rr[32];
               tmem_ld32(tO + c * 32, rr);
               tc_wait_ld();
@@ -631,7 +633,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         // whole tile inside the sequence: through shared memory (128-byte swizzle) and TMA stores
         const int tok = it.tok0 + qb * DAM_TILE;
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
+        for (int half = 0; half < D / 64; ++half) {
           uint32_t pk[32];
 #pragma unroll
           for (int c = 0; c < 2; ++c) {
@@ -663,7 +665,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
       } else {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < D / 32; ++c) {
           uint32_t rr[32];
           tmem_ld32(tO + c * 32, rr);
           tc_wait_ld();
@@ -689,17 +691,18 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   }
 
   if (*abort_flag && tid == 64) atomicMax(prm.status, (uint32_t)DAM_ERR_DEVICE_TIMEOUT);
+  if (blockIdx.x == 0 && tid == 64) prm.status[3] = 1u;      // word 4 of the scratch block: which kernel served the call
   tc_fence_before();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem, kTmemCols);
 }
 
 // Copies the K and V rows of the matched columns of every (sequence, head) into dense tiles of 128 keys in
-// the scratch buffer (K tile at rows (2T) * 128, V tile at rows (2T + 1) * 128 of a [rows][128] bf16 array;
+// the scratch buffer (K tile at rows (2T) * 128, V tile at rows (2T + 1) * 128 of a [rows][head_dim] bf16 array;
 // T = gath_off + head * nL + g).  Rows past the last matched column are zero.  One block per tile, grid-stride.
 __global__ void __launch_bounds__(128)
 gather_columns_kernel(const unsigned char* __restrict__ blob, const __nv_bfloat16* __restrict__ K,
-                      const __nv_bfloat16* __restrict__ V, int Hq, int group, int64_t kst, int64_t ksh, int64_t vst,
+                      const __nv_bfloat16* __restrict__ V, int Hq, int group, int d, int64_t kst, int64_t ksh, int64_t vst,
                       int64_t vsh, unsigned char* scratch, unsigned long long scratch_bytes) {
   asm volatile("griddepcontrol.launch_dependents;");     // the attention kernel behind this one may start its prologue
   const DamHeader* H = reinterpret_cast<const DamHeader*>(blob);
@@ -756,16 +759,17 @@ gather_columns_kernel(const unsigned char* __restrict__ blob, const __nv_bfloat1
     __syncthreads();
     const __nv_bfloat16* Kh = K + (int64_t)sq.tok_start * kst + (int64_t)(h / group) * ksh;
     const __nv_bfloat16* Vh = V + (int64_t)sq.tok_start * vst + (int64_t)(h / group) * vsh;
-    const int part = tid & 15, r0 = tid >> 4;                   // 16 threads x 16 bytes per 256-byte row
-    for (int r = r0; r < DAM_TILE; r += 8) {
+    const int ppr = d >> 3;                                      // 16-byte pieces per row (16 at head_dim 128, 8 at 64)
+    const int part = tid % ppr, r0 = tid / ppr;
+    for (int r = r0; r < DAM_TILE; r += 128 / ppr) {
       const int c = col[r];
       uint4 kv = make_uint4(0u, 0u, 0u, 0u), vv = kv;
       if (c >= 0) {
         kv = __ldg(reinterpret_cast<const uint4*>(Kh + (int64_t)c * kst) + part);
         vv = __ldg(reinterpret_cast<const uint4*>(Vh + (int64_t)c * vst) + part);
       }
-      out[((size_t)(2 * T) * DAM_TILE + r) * 16 + part] = kv;
-      out[((size_t)(2 * T + 1) * DAM_TILE + r) * 16 + part] = vv;
+      out[((size_t)(2 * T) * DAM_TILE + r) * ppr + part] = kv;
+      out[((size_t)(2 * T + 1) * DAM_TILE + r) * ppr + part] = vv;
     }
   }
 }
@@ -800,7 +804,8 @@ cudaError_t dam_launch_bounded_wait_selftest(void* scratch, unsigned long long l
 cudaError_t dam_launch_attn_sm100(const void* Q, const void* K, const void* V, const void* blob,
                                   const dam_shape_t* s, int causal, float scale, void* O, float* lse, void* scratch,
                                   size_t scratch_bytes, const int32_t* ranges, bool run_gather, cudaStream_t st) {
-  if (s->dtype != DAM_BF16 || s->head_dim != 128) return cudaErrorNotSupported;
+  const int d = s->head_dim;
+  if (s->dtype != DAM_BF16 || (d != 128 && d != 64)) return cudaErrorNotSupported;
   if (s->total_tokens == 0) return cudaSuccess;
   int dev = 0;
   DamDeviceInfo di;
@@ -808,30 +813,32 @@ cudaError_t dam_launch_attn_sm100(const void* Q, const void* K, const void* V, c
   if ((e = dam_current_device(&dev, &di)) != cudaSuccess) return e;
   if (di.cc_major != 10 || di.smem_optin < kSmemBytes) return cudaErrorNotSupported;
   if ((e = dam_device_table().once(dev, DAM_SETUP_ATTN_SMEM, [](void) -> cudaError_t {
-         cudaError_t r = cudaFuncSetAttribute(attn_sm100_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-         if (r != cudaSuccess) return r;
-         return cudaFuncSetAttribute(attn_sm100_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+         cudaError_t r;
+         if ((r = cudaFuncSetAttribute(attn_sm100_kernel<false, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) != cudaSuccess) return r;
+         if ((r = cudaFuncSetAttribute(attn_sm100_kernel<true, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) != cudaSuccess) return r;
+         if ((r = cudaFuncSetAttribute(attn_sm100_kernel<false, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) != cudaSuccess) return r;
+         return cudaFuncSetAttribute(attn_sm100_kernel<true, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
        })) != cudaSuccess)
     return e;
   const int sm_count = di.sm_count;
   // gathered-column tiles (if the blob has any) live after the 256-byte status block of the scratch buffer
-  const size_t grows = scratch_bytes > 256 ? (scratch_bytes - 256) / 256 : 0;      // rows of 128 bf16
+  const size_t grows = scratch_bytes > 256 ? (scratch_bytes - 256) / (size_t)(d * 2) : 0;      // rows of head_dim bf16
   CUtensorMap tq, tk, tv, to, tg;
   const bool has_g = grows >= 2 * DAM_TILE;
-  if (!dam_make_tmap_bf16(&tg, has_g ? reinterpret_cast<const unsigned char*>(scratch) + 256 : Q, 128, 1,
-                          has_g ? (int64_t)grows : DAM_TILE, 128, 128))
+  if (!dam_make_tmap_bf16(&tg, has_g ? reinterpret_cast<const unsigned char*>(scratch) + 256 : Q, d, 1,
+                          has_g ? (int64_t)grows : DAM_TILE, d, d))
     return cudaErrorInvalidValue;
   if (has_g && run_gather) {
     gather_columns_kernel<<<sm_count * 4, 128, 0, st>>>(
         reinterpret_cast<const unsigned char*>(blob), reinterpret_cast<const __nv_bfloat16*>(K),
-        reinterpret_cast<const __nv_bfloat16*>(V), s->num_q_heads, s->num_q_heads / s->num_kv_heads, s->k_stride_tok,
+        reinterpret_cast<const __nv_bfloat16*>(V), s->num_q_heads, s->num_q_heads / s->num_kv_heads, d, s->k_stride_tok,
         s->k_stride_head, s->v_stride_tok, s->v_stride_head, reinterpret_cast<unsigned char*>(scratch),
         (unsigned long long)scratch_bytes);
   }
-  if (!dam_make_tmap_bf16(&to, O, 128, s->num_q_heads, s->total_tokens, s->o_stride_tok, s->o_stride_head, 32) ||
-      !dam_make_tmap_bf16(&tq, Q, 128, s->num_q_heads, s->total_tokens, s->q_stride_tok, s->q_stride_head) ||
-      !dam_make_tmap_bf16(&tk, K, 128, s->num_kv_heads, s->total_tokens, s->k_stride_tok, s->k_stride_head) ||
-      !dam_make_tmap_bf16(&tv, V, 128, s->num_kv_heads, s->total_tokens, s->v_stride_tok, s->v_stride_head))
+  if (!dam_make_tmap_bf16(&to, O, d, s->num_q_heads, s->total_tokens, s->o_stride_tok, s->o_stride_head, 32) ||
+      !dam_make_tmap_bf16(&tq, Q, d, s->num_q_heads, s->total_tokens, s->q_stride_tok, s->q_stride_head) ||
+      !dam_make_tmap_bf16(&tk, K, d, s->num_kv_heads, s->total_tokens, s->k_stride_tok, s->k_stride_head) ||
+      !dam_make_tmap_bf16(&tv, V, d, s->num_kv_heads, s->total_tokens, s->v_stride_tok, s->v_stride_head))
     return cudaErrorInvalidValue;
   int pairs = 0;
   for (int b = 0; b < s->num_seqs; ++b) {
@@ -859,6 +866,10 @@ cudaError_t dam_launch_attn_sm100(const void* Q, const void* K, const void* V, c
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = 1;
-  if (ranges) return cudaLaunchKernelEx(&cfg, attn_sm100_kernel<true>, tq, tk, tv, to, tg, p);
-  return cudaLaunchKernelEx(&cfg, attn_sm100_kernel<false>, tq, tk, tv, to, tg, p);
+  if (d == 128) {
+    if (ranges) return cudaLaunchKernelEx(&cfg, attn_sm100_kernel<true, 128>, tq, tk, tv, to, tg, p);
+    return cudaLaunchKernelEx(&cfg, attn_sm100_kernel<false, 128>, tq, tk, tv, to, tg, p);
+  }
+  if (ranges) return cudaLaunchKernelEx(&cfg, attn_sm100_kernel<true, 64>, tq, tk, tv, to, tg, p);
+  return cudaLaunchKernelEx(&cfg, attn_sm100_kernel<false, 64>, tq, tk, tv, to, tg, p);
 }

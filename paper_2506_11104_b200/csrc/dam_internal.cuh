@@ -64,7 +64,7 @@ struct DamHeader {
   uint64_t attn_scratch_bytes;   // scratch dam_sparse_attention needs for this blob
   uint64_t mask_tiles;      // 128 x 128 tiles of the masks that hold an active cell (= total_tiles unless gathered)
   uint64_t head_tile_cap;   // entries of tiles[] every head owns (sum of the row bounds of all sequences)
-  uint64_t reserved[11];
+  uint64_t reserved[11];    // [0]: 1 when the window map was scored by the tensor-core kernel (test hook)
 };
 static_assert(sizeof(DamHeader) == 256, "DamHeader must be 256 bytes");
 

@@ -1,4 +1,5 @@
-// Window scoring on the 5th-generation tensor cores (sm_100a): bf16 inputs, head_dim 128.
+// Window scoring on the 5th-generation tensor cores (sm_100a): bf16 inputs, head_dim 128 or 64 (template parameter:
+// with 64 a Q / K tile is one 16 KB box of the tensor maps and S = Q K^T takes four MMAs instead of eight).
 //
 // For every (sequence, query head) the causal softmax map over the first L tokens is computed tile by
 // tile and thresholded straight into the bit-packed true mask (paper Sec. 4.2.1 - 4.2.3); the map itself
@@ -84,6 +85,7 @@ __device__ __forceinline__ Item decode_item(const unsigned char* blob, const Dam
   return it;
 }
 
+template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                    const ScoreParams prm) {
@@ -130,6 +132,7 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   const uint32_t tmem = *tmem_slot;
   // everything above is independent of the kernel before this one; the blob it initialises is read from here on
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (blockIdx.x == 0 && tid == 0) const_cast<DamHeader*>(H)->reserved[0] = 1ull;   // the map of this blob was scored on the tensor cores
 
   if (warp == 0) {
     if (lane == 0) {
@@ -149,10 +152,10 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         const Item it = decode_item(blob, H, prm, w);
         if (!it.valid) continue;
         if (!(ok = mbar_wait(bQEmpty, (ic & 1u) ^ 1u, abort_flag))) break;
-        mbar_arrive_expect_tx(bQFull, kSlotBytes);
+        mbar_arrive_expect_tx(bQFull, DAM_TILE * D * 2);
         const int tokq = it.sq.tok_start + it.qb * DAM_TILE;
         tma_load_3d(sQ, &tmQ, bQFull, 0, it.h, tokq);
-        tma_load_3d(sQ + 16384, &tmQ, bQFull, 64, it.h, tokq);
+        if (D == 128) tma_load_3d(sQ + 16384, &tmQ, bQFull, 64, it.h, tokq);
         ++ic;
         const int kvh = it.h / prm.group;
         const int ntile = 2 * (it.qb + 1);
@@ -161,9 +164,9 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           const uint32_t s = sc % kSlots, ph = (sc / kSlots) & 1u;
           if (!(ok = mbar_wait(bSlotEmpty + 8 * s, ph ^ 1u, abort_flag))) break;
           const uint32_t dst = sSlots + s * kSlotBytes, bar = bSlotFull + 8 * s;
-          mbar_arrive_expect_tx(bar, kSlotBytes);
+          mbar_arrive_expect_tx(bar, DAM_TILE * D * 2);
           tma_load_3d(dst, &tmK, bar, 0, kvh, it.sq.tok_start + kb * DAM_TILE);
-          tma_load_3d(dst + 16384, &tmK, bar, 64, kvh, it.sq.tok_start + kb * DAM_TILE);
+          if (D == 128) tma_load_3d(dst + 16384, &tmK, bar, 64, kvh, it.sq.tok_start + kb * DAM_TILE);
           armed[s] = ph;
           ++sc;
         }
@@ -198,7 +201,7 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           tc_fence_after();
           const uint32_t b0 = dK_lo + s * (kSlotBytes >> 4);
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {
+          for (int ks = 0; ks < D / 16; ++ks) {
             const uint32_t off = ((ks >> 2) * 16384 + (ks & 3) * 32) >> 4;
             mma_ss_lh(tmem + buf * 128, dQ_lo + off, dQ_hi, b0 + off, dK_hi, idesc, ks > 0 ? 1u : 0u);
           }
@@ -373,7 +376,8 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 
 cudaError_t dam_launch_scores_sm100(const void* Q, const void* K, const dam_shape_t* s, const DamBuildCtx& c,
                                     float* dump, cudaStream_t st) {
-  if (s->dtype != DAM_BF16 || s->head_dim != 128) return cudaErrorNotSupported;
+  const int d = s->head_dim;
+  if (s->dtype != DAM_BF16 || (d != 128 && d != 64)) return cudaErrorNotSupported;
   if (c.max_nL == 0) return cudaSuccess;
   int dev = 0;
   DamDeviceInfo di;
@@ -381,13 +385,15 @@ cudaError_t dam_launch_scores_sm100(const void* Q, const void* K, const dam_shap
   if ((e = dam_current_device(&dev, &di)) != cudaSuccess) return e;
   if (di.cc_major != 10 || di.smem_optin < kSmemBytes) return cudaErrorNotSupported;
   if ((e = dam_device_table().once(dev, DAM_SETUP_SCORE_SMEM, [](void) -> cudaError_t {
-         return cudaFuncSetAttribute(score_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+         cudaError_t r = cudaFuncSetAttribute(score_sm100_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+         if (r != cudaSuccess) return r;
+         return cudaFuncSetAttribute(score_sm100_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
        })) != cudaSuccess)
     return e;
   const int sm_count = di.sm_count;
   CUtensorMap tq, tk;
-  if (!dam_make_tmap_bf16(&tq, Q, 128, s->num_q_heads, s->total_tokens, s->q_stride_tok, s->q_stride_head) ||
-      !dam_make_tmap_bf16(&tk, K, 128, s->num_kv_heads, s->total_tokens, s->k_stride_tok, s->k_stride_head))
+  if (!dam_make_tmap_bf16(&tq, Q, d, s->num_q_heads, s->total_tokens, s->q_stride_tok, s->q_stride_head) ||
+      !dam_make_tmap_bf16(&tk, K, d, s->num_kv_heads, s->total_tokens, s->k_stride_tok, s->k_stride_head))
     return cudaErrorInvalidValue;
   ScoreParams p;
   p.blob = c.blob; p.dump = dump;
@@ -408,5 +414,6 @@ cudaError_t dam_launch_scores_sm100(const void* Q, const void* K, const dam_shap
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, score_sm100_kernel, tq, tk, p);
+  if (d == 128) return cudaLaunchKernelEx(&cfg, score_sm100_kernel<128>, tq, tk, p);
+  return cudaLaunchKernelEx(&cfg, score_sm100_kernel<64>, tq, tk, p);
 }

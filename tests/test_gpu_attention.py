@@ -26,6 +26,8 @@ def _run(w, blob, shape, causal=True, sentinel=False):
         lse = torch.full((w.num_q_heads, Q.shape[0]), float("nan"), dtype=torch.float32, device=DEV)
     O, lse, scratch = B.dam_sparse_attention(Q, K, V, blob, shape, causal=causal, O=O, lse=lse)
     assert B.dam_poll_status(scratch) == 0
+    # bf16 with head_dim 128 or 64 is served by the tcgen05 kernel, everything else by the CUDA-core kernel
+    assert B.attention_ran_on_tensor_cores(scratch) == (w.Q.dtype == torch.bfloat16 and w.head_dim in (64, 128))
     if sentinel:
         _assert_every_row_written(O, lse)
     return O, lse
@@ -115,6 +117,7 @@ def test_config0_every_row():
     ([333, 1000, 64], 200, 4, 1, 64, torch.bfloat16),
     ([1500, 130], 256, 8, 2, 128, torch.bfloat16),
     ([513], 300, 2, 2, 32, torch.float32),
+    ([2100, 700], 384, 8, 2, 64, torch.bfloat16),            # head_dim 64 on the tensor cores, several tiles and a ragged tail
 ])
 @pytest.mark.parametrize("gather", [False, True])
 def test_masked_small_cases_every_row(lengths, pcl, Hq, Hkv, d, dtype, gather):

@@ -110,6 +110,8 @@ def _build_and_check(w, qblocks=None, gather=False):
     blob, _ = B.dam_build_masks(Q, K, shape, rule, scores_dump=dump)
     assert B.dam_poll_status(blob) == 0
     masks = H.oracle_masks_from_dump(w, dump.cpu().numpy())
+    # bf16 with head_dim 128 or 64 is scored by the tcgen05 kernel, everything else by the CUDA-core kernel
+    assert B.MaskBlob(blob).scored_on_tensor_cores == (w.Q.dtype == torch.bfloat16 and w.head_dim in (64, 128))
     H.check_blob_against_oracle(blob, shape, masks, qblocks_per_head=qblocks)
     # a second build without the dump gives the identical blob (dump does not change decisions; deterministic)
     blob2, _ = B.dam_build_masks(Q, K, shape, rule)
@@ -182,6 +184,7 @@ def test_config0_full():
     ([700], 256, 4, 2, 128, torch.bfloat16),
     ([333, 1000, 64], 200, 4, 1, 64, torch.bfloat16),
     ([513], 300, 2, 2, 32, torch.float32),
+    ([2100, 700], 384, 8, 2, 64, torch.bfloat16),
 ])
 @pytest.mark.parametrize("gather", GATHER)
 def test_small_cases_scored_on_gpu(lengths, pcl, Hq, Hkv, d, dtype, gather):
