@@ -98,9 +98,12 @@ typedef struct dam_rule_t {
  * ZSCORE and MINMAX normalise each map by its own statistics over all L x L cells of X (cells above the diagonal
  * count as eps): (X - mean) / (std + eps) with the population deviation, and (X - min) / (max - min + eps). After
  * the minimum is subtracted they read (X - eps) / (std + eps) >= tau and (X - eps) / (max - eps + eps) >= tau, a
- * threshold per map, decided in double precision. They need a pass over the finished map, so only
- * dam_build_masks_from_scores offers them (dam_build_masks returns UNSUPPORTED). The raw sum (Appendix B,
- * method 1) is the average times the sample count and is not offered separately.
+ * threshold per map, decided in double precision. They need a pass over the finished map:
+ * dam_build_masks_from_scores offers them, and dam_build_masks does when it is given a scores_dump buffer (the
+ * map is written there and thresholded from there; without the buffer it returns UNSUPPORTED).
+ *   SUM         the raw sum of Appendix B (method 1): the map handed in is used as it is, like AVERAGE. With one
+ *               input the sum is the map itself; with several, pass the accumulated A of dam_capture_accumulate
+ *               (not divided by the counts) to dam_build_masks_from_scores.
  */
 typedef enum dam_transform_t {
   DAM_TRANSFORM_BOXCOX = 0,
@@ -110,7 +113,8 @@ typedef enum dam_transform_t {
   DAM_TRANSFORM_YEO_JOHNSON = 4,
   DAM_TRANSFORM_AVERAGE = 5,
   DAM_TRANSFORM_ZSCORE = 6,
-  DAM_TRANSFORM_MINMAX = 7
+  DAM_TRANSFORM_MINMAX = 7,
+  DAM_TRANSFORM_SUM = 8
 } dam_transform_t;
 
 /*

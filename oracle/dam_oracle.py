@@ -190,7 +190,7 @@ def amplify_transform(P: np.ndarray, method: str, lam: float, eps: float) -> np.
         T = np.log(X + np.sqrt(X * X + 1.0))
     elif method == "yeo_johnson":                       # X >= 0 branch only: X = max(P, eps) > 0
         T = np.log(X + 1.0) if lam == 0 else (np.power(X + 1.0, lam) - 1.0) / lam
-    elif method == "average":
+    elif method in ("average", "sum"):                  # the map as it is: the average, or (method 1) the raw sum
         T = X.copy()
     elif method == "zscore":                            # statistics over every cell of the map, population deviation
         T = (X - X.mean()) / (X.std() + np.float64(eps))

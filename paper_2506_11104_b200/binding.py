@@ -53,7 +53,7 @@ class dam_rule_t(ctypes.Structure):
                 ("transform", ctypes.c_int32)]
 
 
-TRANSFORMS = {"boxcox": 0, "log": 1, "sqrt": 2, "arcsinh": 3, "yeo_johnson": 4, "average": 5, "zscore": 6, "minmax": 7}
+TRANSFORMS = {"boxcox": 0, "log": 1, "sqrt": 2, "arcsinh": 3, "yeo_johnson": 4, "average": 5, "zscore": 6, "minmax": 7, "sum": 8}
 
 
 _lib = None

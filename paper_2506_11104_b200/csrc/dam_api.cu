@@ -47,7 +47,7 @@ dam_status_t check_rule(const dam_rule_t* r) {
   if (!(r->tau > 0.f) || !(r->eps > 0.f) || !(r->mu == r->mu)) return DAM_ERR_INVALID_ARGUMENT;
   if (r->min_support < 1 || (r->flags & ~DAM_RULE_GATHER_COLUMNS) != 0 || r->softmax_scale < 0.f)
     return DAM_ERR_INVALID_ARGUMENT;
-  if (r->transform < DAM_TRANSFORM_BOXCOX || r->transform > DAM_TRANSFORM_MINMAX) return DAM_ERR_INVALID_ARGUMENT;
+  if (r->transform < DAM_TRANSFORM_BOXCOX || r->transform > DAM_TRANSFORM_SUM) return DAM_ERR_INVALID_ARGUMENT;
   if (!(r->lambda == r->lambda) || fabsf(r->lambda) > 64.f) return DAM_ERR_INVALID_ARGUMENT;
   return DAM_OK;
 }
@@ -207,7 +207,7 @@ dam_status_t fill_ctx(const dam_shape_t* s, const dam_rule_t* r, void* mask, siz
   c->num_seqs = s->num_seqs; c->Hq = s->num_q_heads; c->Hkv = s->num_kv_heads; c->d = s->head_dim; c->dtype = s->dtype;
   c->total_qblocks = y->hdr.total_qblocks; c->rows = y->hdr.rows; c->prows = y->hdr.prows;
   c->max_L = y->max_L; c->max_W = y->max_W; c->max_nL = y->max_nL; c->max_nq = y->max_nq;
-  c->per_map = r->transform >= DAM_TRANSFORM_ZSCORE ? r->transform : 0;
+  c->per_map = (r->transform == DAM_TRANSFORM_ZSCORE || r->transform == DAM_TRANSFORM_MINMAX) ? r->transform : 0;
   c->tau = r->tau; c->eps = r->eps;
   c->pstar = c->per_map ? INFINITY : find_pstar(r);
   c->mu = r->mu; c->min_support = r->min_support;
@@ -306,7 +306,9 @@ dam_status_t dam_build_masks(const void* Q, const void* K, const dam_shape_t* sh
   if (!Q || !K || !aligned(Q, 16) || !aligned(K, 16) || (scores_dump && !aligned(scores_dump, 16)))
     return DAM_ERR_INVALID_ARGUMENT;
   cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
-  if (c.per_map) return DAM_ERR_UNSUPPORTED;     // per-map statistics need the finished map: dam_build_masks_from_scores
+  // thresholds from a map's own statistics need the finished map: with a dump buffer the map is written there first
+  // and thresholded in a second pass; without one the caller has to go through dam_build_masks_from_scores
+  if (c.per_map && !scores_dump) return DAM_ERR_UNSUPPORTED;
   if (dam_launch_rule_prepare(c, cs) != cudaSuccess) return DAM_ERR_CUDA;
   if (dam_launch_init_blob(shape, rule->pcl_max, y.hdr.flags, mask, y.hdr, cs) != cudaSuccess)
     return DAM_ERR_CUDA;
@@ -314,6 +316,7 @@ dam_status_t dam_build_masks(const void* Q, const void* K, const dam_shape_t* sh
   if (sm100_shape(shape)) e = dam_launch_scores_sm100(Q, K, shape, c, scores_dump, cs);
   if (e == cudaErrorNotSupported) e = dam_launch_scores_ref(Q, K, shape, c, scores_dump, cs);
   if (e != cudaSuccess) return DAM_ERR_CUDA;
+  if (c.per_map && dam_launch_bits_from_scores(scores_dump, c, cs) != cudaSuccess) return DAM_ERR_CUDA;
   if (dam_launch_rule(c, cs) != cudaSuccess) return DAM_ERR_CUDA;
   return DAM_OK;
 }

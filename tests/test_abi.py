@@ -61,7 +61,7 @@ def test_mask_sizes_bounds():
     (lambda s, r: setattr(r, "eps", 0.0), 1),
     (lambda s, r: setattr(r, "pcl_max", 0), 1),
     (lambda s, r: setattr(r, "lambda_", float("nan")), 1),
-    (lambda s, r: setattr(r, "transform", 8), 1),
+    (lambda s, r: setattr(r, "transform", 9), 1),
     (lambda s, r: setattr(r, "transform", -1), 1),
     (lambda s, r: setattr(r, "min_support", 0), 1),
     (lambda s, r: setattr(r, "struct_size", 4), 1),

@@ -347,7 +347,7 @@ def test_multi_sample_capture_masks_bit_exact():
 @pytest.mark.parametrize("transform,lam,tau", [
     ("log", 0.0, 13.0), ("sqrt", 0.0, 0.1), ("arcsinh", 0.0, 0.01), ("average", 0.0, 0.01),
     ("boxcox", 0.25, 1.5), ("boxcox", 0.0, 13.0), ("yeo_johnson", 0.5, 0.01), ("yeo_johnson", 0.0, 0.01),
-    ("zscore", 0.0, 1.0), ("minmax", 0.0, 0.02),
+    ("zscore", 0.0, 1.0), ("minmax", 0.0, 0.02), ("sum", 0.0, 0.03),
 ])
 def test_other_amplifications_bit_exact_from_scores(transform, lam, tau):
     """The Appendix-B amplifications through the C ABI: the same fp32 score tensor on both sides, masks bit-exact
@@ -358,16 +358,24 @@ def test_other_amplifications_bit_exact_from_scores(transform, lam, tau):
     dump = torch.zeros(n, dtype=torch.float32, device=DEV)
     B.dam_build_masks(w.Q.to(DEV), w.K.to(DEV), shape, B.make_rule(160, w.tau, w.mu), scores_dump=dump)
     rule = B.make_rule(160, tau, w.mu, lam, w.eps, transform=transform)
-    blob, _ = B.dam_build_masks_from_scores(dump, shape, rule)
-    assert B.dam_poll_status(blob) == 0
-    if transform in ("zscore", "minmax"):
-        # thresholds that depend on the finished map are not offered by the fused path
+    if transform == "sum":
+        # the raw sum of three inputs' maps (here three times the same map), handed in as it is
+        dump = dump * 3.0
+        blob, _ = B.dam_build_masks_from_scores(dump, shape, rule)
+        blob2 = blob
+    elif transform in ("zscore", "minmax"):
+        blob, _ = B.dam_build_masks_from_scores(dump, shape, rule)
+        # thresholds that depend on the finished map: the scoring path takes them when it gets a buffer for the map
         with pytest.raises(B.DamError):
             B.dam_build_masks(w.Q.to(DEV), w.K.to(DEV), shape, rule)
-        blob2 = blob
+        dump2 = torch.zeros_like(dump)
+        blob2, _ = B.dam_build_masks(w.Q.to(DEV), w.K.to(DEV), shape, rule, scores_dump=dump2)
+        assert torch.equal(dump2, dump)
     else:
+        blob, _ = B.dam_build_masks_from_scores(dump, shape, rule)
         # and the fused scoring path decides on the same values
         blob2, _ = B.dam_build_masks(w.Q.to(DEV), w.K.to(DEV), shape, rule)
+    assert B.dam_poll_status(blob) == 0 and B.dam_poll_status(blob2) == 0
     P = H.split_dump(dump.cpu().numpy(), shape.lengths, 4, 160)
     masks = [[orc.head_mask_from_probs(np.ascontiguousarray(P[b][h]), S, tau, w.mu, lam, w.eps, method=transform)
               for h in range(4)] for b, S in enumerate(shape.lengths)]

@@ -378,7 +378,7 @@ def _inverse_threshold(method, tau, lam, eps):
         return (tau + math.sqrt(eps)) ** 2
     if method == "arcsinh":
         return math.sinh(tau + math.asinh(eps))
-    if method == "average":
+    if method in ("average", "sum"):
         return tau + eps
     if method == "boxcox":
         return eps * math.exp(tau) if lam == 0 else (lam * tau + eps ** lam) ** (1.0 / lam)
@@ -390,7 +390,7 @@ def _inverse_threshold(method, tau, lam, eps):
 @pytest.mark.parametrize("method,lam,tau", [
     ("log", 0.0, 12.0), ("sqrt", 0.0, 0.15), ("arcsinh", 0.0, 0.02), ("average", 0.0, 0.03),
     ("boxcox", 0.5, 0.3), ("boxcox", 0.25, 1.0), ("boxcox", 0.0, 12.0), ("boxcox", 1.0, 0.03),
-    ("yeo_johnson", 0.5, 0.02), ("yeo_johnson", 0.0, 0.02), ("yeo_johnson", 2.0, 0.05),
+    ("yeo_johnson", 0.5, 0.02), ("yeo_johnson", 0.0, 0.02), ("yeo_johnson", 2.0, 0.05), ("sum", 0.0, 0.03),
 ])
 def test_transform_mask_is_threshold_at_inverse(method, lam, tau):
     eps = 1e-8
@@ -421,6 +421,22 @@ def test_transform_boxcox_half_equals_the_default_path_and_sqrt_is_its_half():
         assert T.min() == 0.0
         order = np.argsort(P, axis=None)
         assert np.all(np.diff(T.reshape(-1)[order]) >= -1e-15)
+
+
+def test_raw_sum_of_samples_is_the_average_with_the_threshold_scaled_by_the_count():
+    """Appendix B, method 1 (raw sum) against method 2 (average): for n samples that all cover the window the sum is
+    n times the average, so thresholding the sum at n * tau keeps the cells the average keeps at tau (eps scaled
+    alike); worked out by hand, not through the oracle's own formula."""
+    rng = np.random.default_rng(14)
+    L, n = 48, 4
+    samples = []
+    for _ in range(n):
+        P = np.tril(rng.random((L, L)) ** 5)
+        samples.append(P / P.sum(axis=1, keepdims=True))
+    total = np.sum(samples, axis=0)
+    M_sum = orc.true_mask_transform(total, n * 0.03, "sum", 0.0, n * 1e-8)
+    M_avg = orc.true_mask_transform(total / n, 0.03, "average", 0.0, 1e-8)
+    assert np.array_equal(M_sum, M_avg) and 0 < M_sum.sum() < L * (L + 1) // 2
 
 
 def test_zscore_and_minmax_masks_are_thresholds_on_the_map_statistics():
