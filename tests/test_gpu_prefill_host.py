@@ -71,3 +71,29 @@ def test_prefill_host_workspace_too_small():
     ws = torch.empty(n - 256, dtype=torch.uint8, device=DEV)
     with pytest.raises(B.DamError):
         B.dam_prefill_host(w.Q, w.K, w.V, shape, rule, Oh, lh, ws, DEV)
+
+
+def test_prefill_host_with_a_poisoned_workspace():
+    """A chunk that ends at a sequence end inside a 128-key tile makes that tile's K / V rows reach into tokens
+    of the next sequence that arrive with a later chunk (here the windows are shorter than a tile, so they are not
+    among the rows that go up first).  Their probabilities are zero, and the workspace starts out as NaN bit
+    patterns: the result must still be the device calls' result, bit for bit, and pass the oracle."""
+    lengths, Hq, Hkv, d, pcl = [2100, 2300, 2500], 4, 2, 128, 48
+    w = synth.small_case(0, Hq, Hkv, d, pcl, seed=23, dtype=torch.bfloat16, lengths=lengths)
+    shape = B.make_shape(w.cu_seqlens, Hq, Hkv, d, torch.bfloat16, DEV)
+    rule = B.make_rule(w.pcl_max, w.tau, w.mu, w.lam, w.eps, gather_columns=True)
+    Q, K, V = w.Q.to(DEV), w.K.to(DEV), w.V.to(DEV)
+    dump = torch.zeros(sum(Hq * min(S, pcl) ** 2 for S in lengths), dtype=torch.float32, device=DEV)
+    blob, _ = B.dam_build_masks(Q, K, shape, rule, scores_dump=dump)
+    masks = H.oracle_masks_from_dump(w, dump.cpu().numpy())
+    O, lse, scratch = B.dam_sparse_attention(Q, K, V, blob, shape, causal=True)
+    Qh, Kh, Vh = (x.contiguous().pin_memory() for x in (w.Q, w.K, w.V))
+    Oh = torch.full(w.Q.shape, 7.0, dtype=torch.bfloat16).pin_memory()
+    lh = torch.full(tuple(lse.shape), 7.0, dtype=torch.float32).pin_memory()
+    n = B.dam_prefill_host(Qh, Kh, Vh, shape, rule, Oh, lh, None, DEV)
+    ws = torch.full((n,), 0xFF, dtype=torch.uint8, device=DEV)       # every bf16 of the workspace is a NaN
+    B.dam_prefill_host(Qh, Kh, Vh, shape, rule, Oh, lh, ws, DEV)
+    assert torch.isfinite(Oh.float()).all()
+    assert torch.equal(Oh.view(torch.uint8), O.cpu().view(torch.uint8))
+    assert torch.equal(lh.view(torch.uint8), lse.cpu().view(torch.uint8))
+    _oracle_check(w, Oh, lh, masks, True)
