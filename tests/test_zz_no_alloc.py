@@ -41,9 +41,9 @@ def test_static_scratch_matches_regular_entry_point_twice_in_a_row():
         # run yet): that is the documented set-up call.  From then on the free memory the driver reports must
         # not move across a call: torch's own counters would not see a cudaMalloc made inside the library.
         B.dam_build_masks_static(Q, K, shape, rule, mask)
+        mask.zero_()                                                 # (torch loads its own fill kernel on first use)
         torch.cuda.synchronize()
         free_before, _ = torch.cuda.mem_get_info(DEV)
-        mask.zero_()
         B.dam_build_masks_static(Q, K, shape, rule, mask)
         torch.cuda.synchronize()
         free_after, _ = torch.cuda.mem_get_info(DEV)
