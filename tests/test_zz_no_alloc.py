@@ -2,7 +2,6 @@
 whose memory pool owns the whole GPU, a loop that must not call cudaMalloc).  It takes its scratch from a
 fixed array inside the library.  Checked here through the C ABI against dam_build_masks, bit for bit, on
 two calls in a row with different inputs (the second call meets the first call's leftovers in the array)."""
-import numpy as np
 import pytest
 import torch
 
