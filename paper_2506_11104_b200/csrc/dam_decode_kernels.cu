@@ -19,7 +19,7 @@ namespace {
 
 constexpr int kWarps = 8;
 constexpr int kKeysPerGroup = 2;               // keys a lane group has in flight per step
-constexpr int kBlocksPerSM = 4;                // resident blocks the register budget is sized for
+constexpr int kBlocksPerSM = 4;                // resident blocks the register limit is sized for
 constexpr int kRoundWords = 256;               // pattern words the block expands at a time (<= 8192 keys, 32 KB)
 
 template <typename T, int N> struct LdN;       // N consecutive elements -> float

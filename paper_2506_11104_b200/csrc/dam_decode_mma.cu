@@ -23,7 +23,7 @@ namespace {
 constexpr int kGWarps = 4;            // warps per block
 constexpr int kGStages = 1;           // chunks of 16 keys a warp holds in shared memory; with 1 a warp waits for its own copy and
                                       // the other 15 warps of the SM cover the wait (measured faster than 2 stages at half the occupancy)
-constexpr int kGMinBlocks = 4;         // resident blocks per SM the register budget is sized for
+constexpr int kGMinBlocks = 4;         // resident blocks per SM the register limit is sized for
 constexpr int kGChunk = 16;           // keys per chunk (the K dimension of the P V instruction)
 constexpr int kGRoundWords = 128;     // pattern words expanded per round (at most 4096 keys)
 constexpr int kGMaxGroup = 8;         // query heads per KV head this kernel takes (rows 0..7 of the m16 tile)
