@@ -335,6 +335,8 @@ def run_config(cfg, steps, warmup, gather, rank, world, local_rank, dev, pk, B, 
             "avg_launch_ms": round(attn_ms, 4)}
     res = {"value": round(flops_exec / sec / 1e12, 3), "ms_per_step": round(total_ms_max / steps, 4),
            "stage1_ms": round(sum(s1) / len(s1), 4), "stage2_ms": round(attn_ms, 4),
+           "median_ms": {"stage1": round(statistics.median(s1), 4), "stage2": round(statistics.median(s2), 4),
+                         "layer": round(statistics.median([a + b for a, b in zip(s1, s2)]), 4)},
            "value_definition": "4*128*128*d FLOP per tile the attention kernel executed (listed tiles), over the device "
                                "time of the whole steps (stage 1 + stage 2)",
            "effective_mask_tile_tflops": round(flops_mask / sec / 1e12, 3),
@@ -382,7 +384,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=32)
-    ap.add_argument("--warmup", type=int, default=4)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4])
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -20,7 +20,7 @@
 
 namespace {
 
-constexpr int kGWarps = 4;            // warps per block
+constexpr int kGWarps = 5;            // warps per block
 constexpr int kGStages = 1;           // chunks of 16 keys a warp holds in shared memory; with 1 a warp waits for its own copy and
                                       // the other 15 warps of the SM cover the wait (measured faster than 2 stages at half the occupancy)
 constexpr int kGMinBlocks = 4;         // resident blocks per SM the register limit is sized for
@@ -91,12 +91,9 @@ decode_group_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
   const int kvh = blockIdx.x, b = blockIdx.y, h0 = kvh * G;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, row = lane >> 2, quad = lane & 3;
   const DamHeader* H = reinterpret_cast<const DamHeader*>(blob);
-  bool bad = H->magic != DAM_MAGIC || H->num_seqs != num_seqs || H->num_q_heads != Hq;
-  int pos = 0;
-  if (!bad) {
-    pos = pos_dev[b];
-    bad = pos < 0 || pos >= cu[b + 1] - cu[b];
-  }
+  // the header, the position and the sequence bounds are requested together (one round trip to memory, not three)
+  const int pos = __ldg(pos_dev + b), cu0 = __ldg(cu + b), cu1 = __ldg(cu + b + 1);
+  const bool bad = H->magic != DAM_MAGIC || H->num_seqs != num_seqs || H->num_q_heads != Hq || pos < 0 || pos >= cu1 - cu0;
   if (bad) {
     if (tid == 0) atomicMax(status, (uint32_t)DAM_ERR_INVALID_ARGUMENT);
     for (int t = tid; t < G * D; t += kThreads) O[((int64_t)b * Hq + h0) * D + t] = __float2bfloat16_rn(0.f);
@@ -109,8 +106,8 @@ decode_group_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
   // index space of pattern words: [0, W) the row of the true mask (inside the window) or the matched columns;
   // [W, 2W) the matched diagonals (below the window only)
   const int nwords = in_window ? W : 2 * W;
-  const __nv_bfloat16* Kb = K + (int64_t)cu[b] * kst + (int64_t)kvh * ksh;
-  const __nv_bfloat16* Vb = V + (int64_t)cu[b] * vst + (int64_t)kvh * vsh;
+  const __nv_bfloat16* Kb = K + (int64_t)cu0 * kst + (int64_t)kvh * ksh;
+  const __nv_bfloat16* Vb = V + (int64_t)cu0 * vst + (int64_t)kvh * vsh;
 
   // the group's queries as B fragments of Q^T (k = dimension, n = head h0 + n; columns G..7 are zero)
   uint32_t qa0[KS], qa2[KS];
