@@ -33,8 +33,32 @@ __device__ __forceinline__ float g_ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+// K / V rows are read once per launch: they are marked to leave L2 first, so that the few lines every launch reads
+// again (blob header, sequence records, pattern words, queries) are still there next time
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t l2_evict_last_policy() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint32_t ldg_keep(const uint32_t* ptr, uint64_t policy) {
+  uint32_t v;
+  asm volatile("ld.global.nc.L2::cache_hint.u32 %0, [%1], %2;" : "=r"(v) : "l"(ptr), "l"(policy));
+  return v;
+}
+// bits [x, x + 32) of a bit array of nwords words, zero outside it (x may be negative)
+__device__ __forceinline__ uint32_t window32_keep(const uint32_t* bits, int nwords, int x, uint64_t policy) {
+  const int w = x >> 5, sh = x & 31;
+  const uint32_t lo = (w >= 0 && w < nwords) ? ldg_keep(bits + w, policy) : 0u;
+  const uint32_t hi = (w + 1 >= 0 && w + 1 < nwords) ? ldg_keep(bits + w + 1, policy) : 0u;
+  return __funnelshift_r(lo, hi, sh);
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint64_t policy) {
+  asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "l"(policy) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
@@ -126,6 +150,7 @@ decode_group_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
   for (int t = 0; t < KS; ++t) { oacc[t][0] = oacc[t][1] = oacc[t][2] = oacc[t][3] = 0.f; }
 
   const uint32_t stage0 = static_cast<uint32_t>(__cvta_generic_to_shared(gsm)) + warp * (kGStages * LY::stage_bytes);
+  const uint64_t stream_policy = l2_evict_first_policy(), keep_policy = l2_evict_last_policy();
   for (int w0 = 0; w0 < nwords; w0 += kGRoundWords) {
     // ---- one key list for the whole group: a thread per pattern word, the words of all heads OR-ed.  A listed key
     //      is stored as (word, bit) of the round; which heads keep it is read back from the round's words
@@ -137,14 +162,14 @@ decode_group_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
       if (g < G && tid < kGRoundWords && wi < nwords) {
         const DamHeadBits hb = dam_head_bits(blob, H, sq, h0 + g);
         if (in_window) {
-          wh[g] = __ldg(hb.M + (size_t)pos * W + wi);
+          wh[g] = ldg_keep(hb.M + (size_t)pos * W + wi, keep_policy);
         } else if (wi < W) {
-          wh[g] = __ldg(hb.V + wi);
+          wh[g] = ldg_keep(hb.V + wi, keep_policy);
         } else {
           // diagonal r = 32 (wi - W) + k selects key pos - r; dropped when that key is a matched column of the head
           // (then it is in the list already): bit k of the reversed 32-bit window of V that ends at key pos - 32 (wi - W)
           const int r0 = 32 * (wi - W);
-          wh[g] = __ldg(hb.D + (wi - W)) & ~__brev(dam_window32(hb.V, W, pos - r0 - 31));
+          wh[g] = ldg_keep(hb.D + (wi - W), keep_policy) & ~__brev(window32_keep(hb.V, W, pos - r0 - 31, keep_policy));
         }
         uni |= wh[g];
       }
@@ -194,8 +219,8 @@ decode_group_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
         const int idx = c * kGChunk + r;
         const int j = key_of(codes[idx < total ? idx : c * kGChunk]);  // rows past the end repeat the chunk's first key (masked below)
         const uint32_t at = r * LY::row_bytes + ((piece ^ (r & 7)) << 4);
-        cp_async16(dstK + at, Kb + (int64_t)j * kst + piece * 8);
-        cp_async16(dstV + at, Vb + (int64_t)j * vst + piece * 8);
+        cp_async16(dstK + at, Kb + (int64_t)j * kst + piece * 8, stream_policy);
+        cp_async16(dstV + at, Vb + (int64_t)j * vst + piece * 8, stream_policy);
       }
     };
     // (a group is committed every time, also when there is no chunk left to copy, so that "all but the newest
