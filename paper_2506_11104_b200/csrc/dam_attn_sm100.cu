@@ -760,16 +760,29 @@ gather_columns_kernel(const unsigned char* __restrict__ blob, const __nv_bfloat1
     const __nv_bfloat16* Kh = K + (int64_t)sq.tok_start * kst + (int64_t)(h / group) * ksh;
     const __nv_bfloat16* Vh = V + (int64_t)sq.tok_start * vst + (int64_t)(h / group) * vsh;
     const int ppr = d >> 3;                                      // 16-byte pieces per row (16 at head_dim 128, 8 at 64)
-    const int part = tid % ppr, r0 = tid / ppr;
-    for (int r = r0; r < DAM_TILE; r += 128 / ppr) {
-      const int c = col[r];
-      uint4 kv = make_uint4(0u, 0u, 0u, 0u), vv = kv;
-      if (c >= 0) {
-        kv = __ldg(reinterpret_cast<const uint4*>(Kh + (int64_t)c * kst) + part);
-        vv = __ldg(reinterpret_cast<const uint4*>(Vh + (int64_t)c * vst) + part);
+    const int part = tid % ppr, r0 = tid / ppr, step = 128 / ppr;
+    // eight rows of K and of V per thread are requested before the first is stored (the block is one dependent
+    // chain of loads as it is; one round trip per row would be most of its time)
+    for (int rb = r0; rb < DAM_TILE; rb += 8 * step) {
+      uint4 kv[8], vv[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int r = rb + u * step;
+        const int c = r < DAM_TILE ? col[r] : -1;
+        kv[u] = make_uint4(0u, 0u, 0u, 0u); vv[u] = kv[u];
+        if (c >= 0) {
+          kv[u] = __ldg(reinterpret_cast<const uint4*>(Kh + (int64_t)c * kst) + part);
+          vv[u] = __ldg(reinterpret_cast<const uint4*>(Vh + (int64_t)c * vst) + part);
+        }
       }
-      out[((size_t)(2 * T) * DAM_TILE + r) * ppr + part] = kv;
-      out[((size_t)(2 * T + 1) * DAM_TILE + r) * ppr + part] = vv;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int r = rb + u * step;
+        if (r < DAM_TILE) {
+          out[((size_t)(2 * T) * DAM_TILE + r) * ppr + part] = kv[u];
+          out[((size_t)(2 * T + 1) * DAM_TILE + r) * ppr + part] = vv[u];
+        }
+      }
     }
   }
 }
