@@ -13,7 +13,8 @@
 //               S_X = Q_X K^T into the stream's TMEM columns, then O_X += P_X V with P_X read from TMEM (it
 //               overwrites the first half of S_X); the two streams are interleaved so that one stream's softmax
 //               runs under the other stream's MMAs;
-//   warps 2-5   softmax of stream A, warps 6-9 of stream B: one thread per query row reads its S row from
+//   warps 2-3   idle: they fill the first warpgroup, which gives most of its registers to the other two;
+//   warps 4-7   softmax of stream A, warps 8-11 of stream B: one thread per query row reads its S row from
 //               TMEM (twice: running max, then probabilities), applies the tile's mask bits where the tile
 //               is not fully active, writes P (bf16) back to TMEM, rescales O in TMEM when the running max
 //               moved by more than 2^8, and finally normalises and stores O and the log-sum-exp.
@@ -33,7 +34,7 @@ namespace {
 constexpr int kSlots = 4;
 constexpr int kStageBytes = 16384;   // per-stream staging of one 64-column half of the O tile
 constexpr int kSlotBytes = 32768;
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;   // three warpgroups: {producer, MMA issuer, two idle warps}, softmax of stream A, softmax of stream B
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0;      // S_A at 0, S_B at 128 (P_X overwrites columns [0, 64) of S_X)
 constexpr uint32_t kColO = 256;    // O_A at 256, O_B at 384
@@ -341,6 +342,12 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   // under that kernel's tail; its tiles (and the cleared work counter) are visible from here on
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
+  // Registers are handed out per warpgroup: the first one (one producer thread, one issuing thread) keeps 72 per
+  // thread and the two softmax warpgroups take 216 each (72 * 128 + 216 * 256 = the 168 * 384 the CTA starts with).
+  // With 56 the issuing thread spills and the kernel is 6 % slower; with 88 or 104 the softmax warps lose more
+  // than the first warpgroup gains.
+  if (warp < 4) {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -509,9 +516,11 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
       }
     }
+  }
   } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
     // ------------------------------------------------------------------ softmax / epilogue warps
-    const int X = (warp - 2) >> 2;                           // stream: 0 = block 2p, 1 = block 2p+1
+    const int X = (warp - 4) >> 2;                           // stream: 0 = block 2p, 1 = block 2p+1
     const int r = (warp & 3) * 32 + lane;                    // row of the tile = TMEM lane
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t tS = tmem + lane_addr + kColS + X * 128;
